@@ -1,0 +1,219 @@
+"""Pins for the oracle's full optimizer step (Sec. 3.1 Eq. 2-4, Sec. 3.4).
+
+Textbook Adam / AdamW through the full-precision switch, the first step from a
+zero state, per-block scales / quantile / codes re-derived with numpy, tails,
+all-zero blocks, zeros inside a block, threading and the random stream.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2505_00347_b200 import synth
+
+
+def rand_inputs(n, seed, gscale=1e-3):
+    rng = np.random.default_rng(seed)
+    p = rng.normal(0, 0.02, n).astype(np.float32)
+    g = torch.from_numpy(rng.normal(0, gscale, n).astype(np.float32)).to(torch.bfloat16)
+    return p, synth.bf16_bits(g), g.float().numpy()
+
+
+@pytest.mark.parametrize("adamw", [1, 0])
+def test_full_precision_switch_is_textbook_adam(adamw):
+    """With quantization switched off the same EMA / update lines must reproduce
+    torch.optim.AdamW (decoupled decay) and torch.optim.Adam (L2 in the gradient)."""
+    n, steps = 1000, 10
+    p0, _, _ = rand_inputs(n, 1)
+    h = oracle.hyper(lr=1e-2, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.1, adamw=adamw)
+    tp = torch.nn.Parameter(torch.from_numpy(p0.copy()).double())
+    cls = torch.optim.AdamW if adamw else torch.optim.Adam
+    opt = cls([tp], lr=1e-2, betas=(float(np.float32(0.9)), float(np.float32(0.999))), eps=1e-8,
+              weight_decay=float(np.float32(0.1)))
+    p = p0.copy()
+    st = oracle.State(n, 4, 4, 128)
+    m32, v32 = np.zeros(n, np.float32), np.zeros(n, np.float32)
+    for t in range(1, steps + 1):
+        _, gb, gf = rand_inputs(n, 100 + t)
+        tp.grad = torch.from_numpy(gf).double()
+        opt.step()
+        oracle.step(p, gb, st, h, t, m32=m32, v32=v32)
+        ref = tp.detach().numpy()
+        # binary32 storage of p: half an ulp of |p| <= 0.1 per step, plus 1e-6 relative
+        assert np.all(np.abs(p - ref) <= 1e-6 * np.abs(ref) + 4e-9 * t), t
+    assert np.allclose(m32, opt.state[tp]["exp_avg"].numpy(), rtol=1e-5, atol=1e-9)
+    assert np.allclose(v32, opt.state[tp]["exp_avg_sq"].numpy(), rtol=1e-5, atol=1e-15)
+    assert np.all(st.codes_m == 0) and np.all(st.scale_m == 0)      # packed state untouched
+
+
+def test_first_step_from_zero_state():
+    """From the zero state the EMA sees no quantization: m^ = (1-b1) g, v^ = (1-b2) g^2 and the
+    parameter moves by the bias-corrected AdamW step."""
+    n = 128 * 5 + 17
+    p, gb, gf = rand_inputs(n, 2)
+    p0 = p.copy()
+    h = oracle.hyper(lr=1e-3, beta1=0.8, beta2=0.999, weight_decay=0.01)
+    st = oracle.State(n, 4, 4, 128)
+    mh, vh, _ = oracle.step(p, gb, st, h, 1, want_hat=True)
+    b1, b2 = np.float32(0.8), np.float32(0.999)
+    assert np.allclose(mh, (1 - b1) * gf, rtol=1e-6, atol=0)
+    assert np.allclose(vh, (1 - b2) * gf * gf, rtol=1e-6, atol=0)
+    g64 = gf.astype(np.float64)
+    ref = p0 * (1 - 1e-3 * 0.01) - 1e-3 * g64 / (np.abs(g64) + 1e-8)   # m^/bc1 = g, sqrt(v^/bc2) = |g|
+    assert np.allclose(p, ref, rtol=2e-6, atol=1e-9)
+
+
+@pytest.mark.parametrize("bits_m,bits_v,block", [(4, 4, 128), (2, 3, 128), (3, 3, 64), (8, 8, 256),
+                                                 (4, 2, 2048)])
+def test_block_quantities_rederived(bits_m, bits_v, block):
+    """After a few steps: scales are block maxima, the base puts level K-1 on the p-quantile,
+    codes are the nearest levels (re-derived with numpy in binary64)."""
+    n = block * 6 + block // 3 + 1
+    p, _, _ = rand_inputs(n, 3)
+    h = oracle.hyper(beta1=0.8, seed=99)
+    st = oracle.State(n, bits_m, bits_v, block)
+    Km, Kv = 1 << bits_m, 1 << bits_v
+    ym = oracle.codebook(oracle.DE_SIGNED, bits_m).astype(np.float64)
+    mids = 0.5 * (ym[:-1] + ym[1:])
+    for t in range(1, 5):
+        _, gb, _ = rand_inputs(n, 30 + t, gscale=1e-3 * t)
+        mh, vh, fl = oracle.step(p, gb, st, h, t, tensor=2, want_hat=True, want_flags=True)
+        dm, dv = oracle.dequant(st, 0), oracle.dequant(st, 1)
+        for j in range(st.nblk):
+            sl = slice(j * block, min(n, (j + 1) * block))
+            nb = sl.stop - sl.start
+            assert st.scale_m[j] == np.abs(mh[sl]).max() and st.scale_v[j] == vh[sl].max()
+            k = max(1, math.ceil(float(np.float32(0.1)) * nb))
+            x_p = np.sort(vh[sl])[k - 1]
+            rho = min(max(float(x_p) / float(st.scale_v[j]), 2.0 ** -48), 1 - 2.0 ** -10)
+            a = float(st.alpha[j])
+            assert 0 < a < 1 and a ** (Kv - 1) == pytest.approx(rho, rel=2e-4)
+            # first moment: nearest level
+            r = mh[sl].astype(np.float64) / float(st.scale_m[j])
+            q_ref = (r[:, None] > mids[None, :]).sum(1)
+            q = np.array([oracle.get_code(st.codes_m[j * (block * bits_m // 8):], e, bits_m) for e in range(nb)])
+            near = np.min(np.abs(r[:, None] - mids[None, :]), axis=1) < 1e-6
+            assert np.all((q == q_ref) | near)
+            # second moment: Eq. 6 with the element's own xi
+            rv = vh[sl].astype(np.float64) / float(st.scale_v[j])
+            qv = np.array([oracle.get_code(st.codes_v[j * (block * bits_v // 8):], e, bits_v) for e in range(nb)])
+            for e in range(nb):
+                w = oracle.philox_word(99, t, 2, sl.start + e, 0)
+                tt = math.log(rv[e]) / math.log(a) + oracle.xi(w) if rv[e] > 0 else Kv
+                q_ref_v = int(min(max(round(tt), 0), Kv - 1))
+                assert qv[e] == q_ref_v or abs(tt - math.floor(tt) - 0.5) < 2e-4, (j, e, tt, qv[e])
+            # dequantized state: sign / positivity, never above the scale
+            assert np.all(dv[sl] > 0) and np.all(dv[sl] <= st.scale_v[j])
+            assert np.all((dm[sl] == 0) | (np.sign(dm[sl]) == np.sign(mh[sl])))
+            assert np.all(np.abs(dm[sl]) <= st.scale_m[j])
+        # bf16 gradients make exact ties (e.g. g_i / g_max = -11/40 on the 2-bit midpoint
+        # -0.275) possible at step 1; they are rare
+        assert fl.mean() < 0.01
+
+
+def test_zero_gradients_and_zero_blocks():
+    n, block = 128 * 3 + 5, 128
+    p, gb, _ = rand_inputs(n, 4)
+    gb[128:256] = 0                      # one all-zero block
+    gb[300] = 0                          # a zero inside a non-zero block
+    h = oracle.hyper(weight_decay=0.0)
+    st = oracle.State(n, 2, 3, block)
+    p0 = p.copy()
+    oracle.step(p, gb, st, h, 1)
+    assert st.scale_m[1] == 0 and st.scale_v[1] == 0 and st.alpha[1] == 0.5
+    assert np.all(st.codes_m[32:64] == 0) and np.all(st.codes_v[48:96] == 0)
+    assert np.array_equal(p[128:256], p0[128:256])          # no gradient, no decay: unchanged
+    dv, dm = oracle.dequant(st, 1), oracle.dequant(st, 0)
+    assert np.all(dv[128:256] == 0) and np.all(dm[128:256] == 0)
+    assert oracle.get_code(st.codes_v[2 * 48:], 300 - 256, 3) == 7   # zero element -> smallest level
+    assert dv[300] > 0 and dm[300] == 0
+    # >= 10 % zeros in a block: the quantile is 0 and the base is clamped, not 0
+    gb2 = gb.copy()
+    gb2[0:20] = 0
+    st2 = oracle.State(n, 2, 3, block)
+    oracle.step(p0.copy(), gb2, st2, h, 1)
+    assert st2.alpha[0] == pytest.approx(2.0 ** (-48 / 7), rel=1e-6)
+    # a block that goes quiet decays; its scale shrinks by beta each step, never negative
+    zeros = np.zeros(n, np.uint16)
+    before = oracle.dequant(st, 1).copy()
+    for t in range(2, 6):
+        oracle.step(p, zeros, st, h, t)
+    after = oracle.dequant(st, 1)
+    assert np.all(after >= 0) and after[:128].max() == pytest.approx(before[:128].max() * 0.999 ** 4, rel=1e-5)
+
+
+@pytest.mark.parametrize("n", [1, 2, 63, 64, 65, 127, 129])
+def test_tiny_and_ragged_tensors(n):
+    p, gb, gf = rand_inputs(n, 5 + n)
+    h = oracle.hyper()
+    st = oracle.State(n, 4, 4, 128)
+    assert st.nblk == (n + 127) // 128 and st.codes_m.size == st.nblk * 64
+    for t in range(1, 4):
+        mh, vh, _ = oracle.step(p, gb, st, h, t, want_hat=True)
+    assert st.scale_m[0] == np.abs(mh[:128]).max()
+    assert np.all(np.isfinite(p))
+    tail = n % 128
+    if tail:    # padding codes of the tail block stay zero
+        last = st.codes_m[(st.nblk - 1) * 64:]
+        assert all(oracle.get_code(last, e, 4) == 0 for e in range(tail, 128))
+    if n == 1:  # a single element is its own maximum and its own quantile
+        assert oracle.get_code(st.codes_m, 0, 4) in (0, 15)
+        assert oracle.get_code(st.codes_v, 0, 4) in (0, 1)
+        assert st.alpha[0] == pytest.approx((1 - 2.0 ** -10) ** (1 / 15), rel=1e-6)
+
+
+def test_threads_slices_and_stream():
+    n, block = 128 * 37 + 11, 128
+    p, gb, _ = rand_inputs(n, 6)
+    h = oracle.hyper(seed=7)
+    runs = []
+    for nthreads in (1, 4):
+        pp, st = p.copy(), oracle.State(n, 3, 3, block)
+        for t in range(1, 4):
+            oracle.step(pp, gb, st, h, t, nthreads=nthreads)
+        runs.append((pp, st))
+    for k in ("codes_m", "codes_v", "scale_m", "scale_v", "alpha"):
+        assert np.array_equal(getattr(runs[0][1], k), getattr(runs[1][1], k))
+    assert np.array_equal(runs[0][0], runs[1][0])
+    # a slice that starts at block 5 with elem_offset set reproduces the full run's blocks
+    full_p, full = p.copy(), oracle.State(n, 3, 3, block)
+    oracle.step(full_p, gb, full, h, 1, tensor=4)
+    lo = 5 * block
+    sl_p, sl = p[lo:].copy(), oracle.State(n - lo, 3, 3, block)
+    oracle.step(sl_p, gb[lo:].copy(), sl, h, 1, tensor=4, elem_offset=lo)
+    assert np.array_equal(sl.codes_v, full.codes_v[5 * 48:]) and np.array_equal(sl_p, full_p[lo:])
+    # the stream depends on seed, step and tensor
+    other = oracle.State(n, 3, 3, block)
+    oracle.step(p.copy(), gb, other, h, 1, tensor=5)
+    assert not np.array_equal(other.codes_v, full.codes_v)
+    assert np.array_equal(other.codes_m, full.codes_m)          # nearest rounding draws nothing
+    det = oracle.State(n, 3, 3, block)
+    oracle.step(p.copy(), gb, det, oracle.hyper(seed=7, round_v=0), 1, tensor=5)
+    det2 = oracle.State(n, 3, 3, block)
+    oracle.step(p.copy(), gb, det2, oracle.hyper(seed=8, round_v=0), 1, tensor=9)
+    assert np.array_equal(det.codes_v, det2.codes_v)            # xi = 0: no randomness
+
+
+def test_bf16_parameters_and_stochastic_m():
+    n = 128 * 4
+    p, gb, _ = rand_inputs(n, 8)
+    pb = synth.bf16_bits(torch.from_numpy(p).to(torch.bfloat16))
+    pf = synth.bits_to_bf16(pb).float().numpy().copy()
+    h16 = oracle.hyper(param_dtype=1, lr=1e-2)
+    h32 = oracle.hyper(param_dtype=0, lr=1e-2)
+    s16, s32 = oracle.State(n, 4, 4, 128), oracle.State(n, 4, 4, 128)
+    oracle.step(pb, gb, s16, h16, 1)
+    oracle.step(pf, gb, s32, h32, 1)
+    want = synth.bf16_bits(torch.from_numpy(pf).to(torch.bfloat16))     # torch rounds to nearest even
+    assert np.array_equal(pb, want)
+    assert np.array_equal(s16.codes_v, s32.codes_v)
+    # stochastic first moment: codes bracket the nearest ones and differ somewhere
+    hs = oracle.hyper(round_m=1, seed=3)
+    ss, sn = oracle.State(n, 4, 4, 128), oracle.State(n, 4, 4, 128)
+    oracle.step(p.copy(), gb, ss, hs, 1)
+    oracle.step(p.copy(), gb, sn, oracle.hyper(seed=3), 1)
+    a = np.array([oracle.get_code(ss.codes_m, e, 4) for e in range(128)])
+    b = np.array([oracle.get_code(sn.codes_m, e, 4) for e in range(128)])
+    assert np.max(np.abs(a - b)) <= 1 and np.any(a != b)
