@@ -1,0 +1,185 @@
+/*
+ * solo.h -- C ABI of the B200 (sm_100a) fused low-bit optimizer step.
+ *
+ * The operation is the block-wise quantized Adam(W) step of "Pushing the Limits
+ * of Low-Bit Optimizers: A Focus on EMA Dynamics" (SOLO): Sec. 3.1 Eq. 2-4
+ * (dequantize, EMA, quantize), Sec. 3.2.2 Eq. 6 (logarithmic quantizer with a
+ * quantile-derived base for the second moment), Sec. 3.3 / Appendix A (signed
+ * dynamic-exponent codebook and a precision-specific beta1 for the first moment),
+ * Sec. 3.4 (4/2-bit and 2-bit Adam(W), block size 128).
+ *
+ * Conventions
+ *   - Every pointer named *_dev or documented "device" is a CUDA device pointer
+ *     of the current device; everything else is host memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     All device work is enqueued on it; no call synchronizes unless it says so.
+ *   - Functions return SOLO_OK (0) or a negative solo_status_t.  Nothing throws,
+ *     aborts or traps on the device.  Arguments are validated on the host before
+ *     anything is launched; a rejected call has no effect.
+ *   - Gradients are bf16.  Parameters are fp32 or bf16 and are updated in place.
+ *   - bits is 2, 3, 4 or 8 independently for the two moments; block is 64, 128,
+ *     256 or 2048 elements.
+ *
+ * State layout (device memory owned by the solo_state_t), n_blk blocks in total,
+ * tensors laid out one after the other, every tensor starting on a new block:
+ *   codes_m  n_blk * block*bits_m/8 bytes   element e of a block occupies bits
+ *   codes_v  n_blk * block*bits_v/8 bytes   [e*b, e*b+b) of the block's slot read
+ *                                           as a little-endian bit string; a short
+ *                                           last block keeps a whole slot, padding
+ *                                           codes are 0
+ *   scale_m  n_blk fp32   Delta of the first moment  (max |m| of the block)
+ *   scale_v  n_blk fp32   Delta of the second moment (max v of the block)
+ *   alpha    n_blk fp32   base of the block's logarithmic codebook, in (0,1)
+ * The zero state (all codes 0, Delta = 0, alpha = 0.5) dequantizes to exact zeros.
+ */
+#ifndef SOLO_H_
+#define SOLO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SOLO_OK = 0,
+    SOLO_EINVAL = -1,   /* bad argument value (bits, block, numel, null pointer, ...) */
+    SOLO_EALIGN = -2,   /* a parameter / gradient pointer is not 16-byte aligned */
+    SOLO_ENOMEM = -3,   /* device or host allocation failed */
+    SOLO_ECUDA = -4,    /* a CUDA runtime call or the kernel launch failed */
+    SOLO_ESTATE = -5    /* the state does not match the call (sizes, tensor count) */
+} solo_status_t;
+
+/* Constants of the quantizers that the paper leaves open. */
+#define SOLO_TINY_EXP (-100)      /* a block scale below 2^-100 is stored as 0 */
+#define SOLO_RHO_MIN_EXP (-48)    /* x_p / Delta is clamped to [2^-48, 1 - 2^-10] */
+#define SOLO_RHO_MAX_EXP (-10)
+
+typedef struct solo_state solo_state_t; /* opaque; owns its device buffers */
+
+/* Hyper-parameters of one step; plain data, read at the call and not retained. */
+typedef struct {
+    float lr;
+    float beta1;           /* momentum of the signed EMA: the precision-specific beta' of Eq. 7 */
+    float beta2;           /* momentum of the unsigned EMA (unchanged, e.g. 0.999) */
+    float eps;
+    float weight_decay;
+    float p_quantile;      /* p of the base alpha = (x_p/Delta)^(1/(2^b-1)); 0.1 in the paper; [0,1) */
+    int32_t adamw;         /* 1: decoupled decay (AdamW); 0: decay added to the gradient (Adam) */
+    int32_t bias_correction; /* 1: divide by 1-beta^t; 0: no correction */
+    int32_t round_m;       /* 0: nearest level (Eq. 1); 1: stochastic rounding (Eq. 5) */
+    int32_t round_v;       /* 1: xi ~ U(-1/2,1/2) in Eq. 6; 0: xi = 0 (deterministic) */
+    int32_t param_dtype;   /* 0: fp32 parameters; 1: bf16 parameters */
+    uint64_t seed;         /* Philox key of the rounding noise */
+} solo_hyper_t;
+
+/*
+ * Packed tensor list for solo_multi_step.  The struct itself is host memory; the
+ * three arrays it points to are DEVICE memory and stay owned by the caller:
+ *   param[t], grad[t]  device pointers of tensor t, each 16-byte aligned
+ *   numel[t]           its element count (must equal what the state was created with)
+ * `state` must come from solo_state_create_multi with the same sizes.
+ */
+typedef struct {
+    int32_t num_tensors;
+    void* const* param;          /* device array [num_tensors] of device pointers */
+    const void* const* grad;     /* device array [num_tensors] of device pointers (bf16) */
+    const int64_t* numel;        /* device array [num_tensors] */
+    solo_state_t* state;
+} solo_tensor_list_t;
+
+/*
+ * Sec. 3.4 (block-wise state of 4/2-bit and 2-bit Adam(W)).  Allocates the zero
+ * state for one tensor of `numel` > 0 elements on the current device and returns
+ * it in *out.  Synchronous (cudaMalloc + cudaMemset).
+ */
+int solo_state_create(int64_t numel, int bits_m, int bits_v, int block, solo_state_t** out);
+
+/*
+ * Same for a list of `num_tensors` tensors; numel_host is a HOST array.  Tensor t
+ * owns blocks [block_start[t], block_start[t+1]) of the state, block_start being
+ * the running sum of ceil(numel[t] / block).
+ */
+int solo_state_create_multi(const int64_t* numel_host, int num_tensors, int bits_m, int bits_v,
+                            int block, solo_state_t** out);
+
+/* Frees the state's device and host memory (synchronous).  NULL is accepted. */
+int solo_state_destroy(solo_state_t* state);
+
+/*
+ * Memory accounting of Sec. 5.2 ("Block size") / Table 2: bytes of state for one
+ * tensor = codes of both moments (whole slots) + 12 bytes per block.  Host only.
+ */
+int solo_state_bytes(int64_t numel, int bits_m, int bits_v, int block, size_t* out);
+
+/*
+ * One fused optimizer step on a single tensor (Eq. 2-4 + Adam(W), one pass over
+ * HBM): per element dequantize m and v, m^ = beta1 m~ + (1-beta1) g,
+ * v^ = beta2 v~ + (1-beta2) g^2, p <- p (1 - lr wd) - (lr/bc1) m^ / (sqrt(v^)/sqrt(bc2) + eps),
+ * then per block the new scales, the base from the p-quantile of v^, and the new
+ * codes (Eq. 1 or 5 for m, Eq. 6 for v), packed and stored.
+ *   param  device, fp32 or bf16 per hyper->param_dtype, numel elements, in/out
+ *   grad   device, bf16, numel elements, read only
+ *   step   1-based step count t (bias corrections, Philox counter)
+ * Asynchronous on `stream`.
+ */
+int solo_step(void* param_dev, const void* grad_dev, solo_state_t* state,
+              const solo_hyper_t* hyper, int64_t step, void* stream);
+
+/*
+ * The same step over every tensor of the list in ONE kernel launch, ragged block
+ * tails included.  Tensor t uses Philox stream t.  Asynchronous on `stream`.
+ */
+int solo_multi_step(const solo_tensor_list_t* list, const solo_hyper_t* hyper, int64_t step,
+                    void* stream);
+
+/*
+ * Eq. 2 for inspection: writes the dequantized moment of every element, tensors
+ * concatenated without padding (sum of numel floats).
+ *   which  0: first moment y[q] * Delta_m;  1: second moment alpha^q * Delta_v
+ *   out_dev  device, fp32
+ * Asynchronous on `stream`.
+ */
+int solo_dequant(const solo_state_t* state, int which, float* out_dev, void* stream);
+
+/*
+ * Raw access to the state's device buffers (tests, checkpointing).
+ *   which  0 codes_m, 1 codes_v, 2 scale_m, 3 scale_v, 4 alpha
+ * The pointers stay owned by the state.
+ */
+int solo_state_raw(const solo_state_t* state, int which, void** dev_ptr, size_t* bytes);
+
+/* Geometry of a state: total elements, total blocks, tensors, bits, block. */
+int solo_state_info(const solo_state_t* state, int64_t* numel, int64_t* num_blocks,
+                    int32_t* num_tensors, int32_t* bits_m, int32_t* bits_v, int32_t* block);
+
+/*
+ * Reads the state's device status word into *status_out (0 = no problem seen;
+ * bit 0 = a solo_multi_step descriptor's numel disagreed with the state and the
+ * affected tensors were skipped).  Synchronizes the device.
+ */
+int solo_state_status(solo_state_t* state, int* status_out);
+
+/*
+ * Signed dynamic-exponent codebook of Appendix A (ascending, 2^bits levels) as the
+ * library uses it, copied to a HOST array of 2^bits floats.
+ */
+int solo_codebook_m(int bits, float* levels_host);
+
+/*
+ * Eq. 7 with the defaults of Sec. 3.4: the recommended beta1 for `bits_m`-bit first
+ * moments, from_scratch = 0 (fine-tuning, b = 5 column of Fig. 4) or 1 (b = 8 column),
+ * floored to one decimal like the paper's own defaults (4 bit: 0.8 / 0.3; 2 bit: 0.5 / 0.1).
+ */
+float solo_default_beta1(int bits_m, int from_scratch);
+
+/* Number of kernel launches issued by this library in the calling process so far. */
+int64_t solo_launch_count(void);
+
+const char* solo_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SOLO_H_ */

@@ -1,0 +1,271 @@
+"""ctypes binding of the C ABI in include/solo.h (argument marshalling only).
+
+Every step of the optimizer runs in the CUDA library; this module passes raw device
+pointers of torch tensors and the current CUDA stream.  If the shared library is not
+there, loading raises: there is no other implementation to fall back to.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from pathlib import Path
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "libsolo_b200.so"
+
+SOLO_OK, SOLO_EINVAL, SOLO_EALIGN, SOLO_ENOMEM, SOLO_ECUDA, SOLO_ESTATE = 0, -1, -2, -3, -4, -5
+
+
+class SoloError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {strerror(status)} ({status})")
+
+
+class Hyper(C.Structure):
+    """solo_hyper_t"""
+
+    _fields_ = [
+        ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+        ("weight_decay", C.c_float), ("p_quantile", C.c_float),
+        ("adamw", C.c_int32), ("bias_correction", C.c_int32), ("round_m", C.c_int32),
+        ("round_v", C.c_int32), ("param_dtype", C.c_int32), ("seed", C.c_uint64),
+    ]
+
+
+class TensorList(C.Structure):
+    """solo_tensor_list_t"""
+
+    _fields_ = [
+        ("num_tensors", C.c_int32), ("param", C.c_void_p), ("grad", C.c_void_p),
+        ("numel", C.c_void_p), ("state", C.c_void_p),
+    ]
+
+
+def hyper(lr=1e-3, beta1=0.8, beta2=0.999, eps=1e-8, weight_decay=0.01, p_quantile=0.1,
+          adamw=1, bias_correction=1, round_m=0, round_v=1, param_dtype=0, seed=0) -> Hyper:
+    return Hyper(lr, beta1, beta2, eps, weight_decay, p_quantile, adamw, bias_correction,
+                 round_m, round_v, param_dtype, seed)
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libsolo_b200.so from the package directory; raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not LIB_PATH.exists():
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2505_00347_b200._build` "
+            "(nvcc, sm_100a).  There is no CPU or PyTorch fallback.")
+    L = C.CDLL(str(LIB_PATH))
+    vp, i64, i32 = C.c_void_p, C.c_int64, C.c_int
+    L.solo_state_create.argtypes = [i64, i32, i32, i32, C.POINTER(vp)]
+    L.solo_state_create_multi.argtypes = [C.POINTER(C.c_int64), i32, i32, i32, i32, C.POINTER(vp)]
+    L.solo_state_destroy.argtypes = [vp]
+    L.solo_state_bytes.argtypes = [i64, i32, i32, i32, C.POINTER(C.c_size_t)]
+    L.solo_step.argtypes = [vp, vp, vp, C.POINTER(Hyper), i64, vp]
+    L.solo_multi_step.argtypes = [C.POINTER(TensorList), C.POINTER(Hyper), i64, vp]
+    L.solo_dequant.argtypes = [vp, i32, vp, vp]
+    L.solo_state_raw.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(C.c_size_t)]
+    L.solo_state_info.argtypes = [vp, C.POINTER(C.c_int64), C.POINTER(C.c_int64),
+                                  C.POINTER(C.c_int32), C.POINTER(C.c_int32),
+                                  C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    L.solo_state_status.argtypes = [vp, C.POINTER(C.c_int)]
+    L.solo_codebook_m.argtypes = [i32, C.POINTER(C.c_float)]
+    L.solo_default_beta1.argtypes = [i32, i32]
+    L.solo_default_beta1.restype = C.c_float
+    L.solo_launch_count.argtypes = []
+    L.solo_launch_count.restype = C.c_int64
+    L.solo_strerror.argtypes = [i32]
+    L.solo_strerror.restype = C.c_char_p
+    for name in ("solo_state_create", "solo_state_create_multi", "solo_state_destroy",
+                 "solo_state_bytes", "solo_step", "solo_multi_step", "solo_dequant",
+                 "solo_state_raw", "solo_state_info", "solo_state_status", "solo_codebook_m"):
+        getattr(L, name).restype = C.c_int
+    _lib = L
+    return L
+
+
+def strerror(status: int) -> str:
+    return lib().solo_strerror(status).decode()
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != SOLO_OK:
+        raise SoloError(rc, what)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+RAW = {"codes_m": 0, "codes_v": 1, "scale_m": 2, "scale_v": 3, "alpha": 4}
+_RAW_DTYPE = {0: torch.uint8, 1: torch.uint8, 2: torch.float32, 3: torch.float32, 4: torch.float32}
+
+
+class State:
+    """Owner of a solo_state_t handle (single tensor or tensor list)."""
+
+    def __init__(self, numel, bits_m: int, bits_v: int, block: int = 128):
+        self.handle = C.c_void_p()
+        self.sizes = [int(numel)] if isinstance(numel, int) else [int(n) for n in numel]
+        if isinstance(numel, int):
+            rc = lib().solo_state_create(numel, bits_m, bits_v, block, C.byref(self.handle))
+        else:
+            arr = (C.c_int64 * len(self.sizes))(*self.sizes)
+            rc = lib().solo_state_create_multi(arr, len(self.sizes), bits_m, bits_v, block,
+                                               C.byref(self.handle))
+        _check(rc, "solo_state_create")
+        self.bits_m, self.bits_v, self.block = bits_m, bits_v, block
+        self.device = torch.device("cuda", torch.cuda.current_device())
+
+    def destroy(self) -> None:
+        if getattr(self, "handle", None) is not None and self.handle:
+            lib().solo_state_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def info(self) -> dict:
+        n, nb = C.c_int64(), C.c_int64()
+        t, bm, bv, blk = C.c_int32(), C.c_int32(), C.c_int32(), C.c_int32()
+        _check(lib().solo_state_info(self.handle, C.byref(n), C.byref(nb), C.byref(t), C.byref(bm),
+                                     C.byref(bv), C.byref(blk)), "solo_state_info")
+        return dict(numel=n.value, num_blocks=nb.value, num_tensors=t.value, bits_m=bm.value,
+                    bits_v=bv.value, block=blk.value)
+
+    def raw_ptr(self, which) -> tuple[int, int]:
+        w = RAW[which] if isinstance(which, str) else which
+        p, b = C.c_void_p(), C.c_size_t()
+        _check(lib().solo_state_raw(self.handle, w, C.byref(p), C.byref(b)), "solo_state_raw")
+        return p.value or 0, b.value
+
+    def raw_get(self, which) -> torch.Tensor:
+        """Copy of one state buffer as a CPU tensor (uint8 codes / float32 scales)."""
+        w = RAW[which] if isinstance(which, str) else which
+        ptr, nbytes = self.raw_ptr(w)
+        out = torch.empty(nbytes, dtype=torch.uint8)
+        torch.cuda.synchronize()
+        _cuda_memcpy(out.data_ptr(), ptr, nbytes, 2)
+        return out if _RAW_DTYPE[w] == torch.uint8 else out.view(torch.float32)
+
+    def raw_set(self, which, value: torch.Tensor) -> None:
+        """Overwrite one state buffer from a CPU tensor of the same byte size."""
+        w = RAW[which] if isinstance(which, str) else which
+        ptr, nbytes = self.raw_ptr(w)
+        v = value.contiguous().view(torch.uint8).cpu()
+        if v.numel() != nbytes:
+            raise ValueError(f"expected {nbytes} bytes, got {v.numel()}")
+        torch.cuda.synchronize()
+        _cuda_memcpy(ptr, v.data_ptr(), nbytes, 1)
+
+    def status(self) -> int:
+        s = C.c_int()
+        _check(lib().solo_state_status(self.handle, C.byref(s)), "solo_state_status")
+        return s.value
+
+
+_cudart = None
+
+
+def _cuda_memcpy(dst: int, src: int, nbytes: int, kind: int) -> None:
+    """cudaMemcpy through the runtime that torch already loaded (kind 1 = H2D, 2 = D2H)."""
+    global _cudart
+    if nbytes == 0:
+        return
+    if _cudart is None:
+        _cudart = C.CDLL(_find_cudart())
+        _cudart.cudaMemcpy.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_int]
+        _cudart.cudaMemcpy.restype = C.c_int
+    rc = _cudart.cudaMemcpy(dst, src, nbytes, kind)
+    if rc:
+        raise RuntimeError(f"cudaMemcpy failed with {rc}")
+
+
+def _find_cudart() -> str:
+    import glob
+    import os
+    cands = []
+    for root in (os.path.join(os.path.dirname(torch.__file__), "lib"),
+                 os.path.join(os.path.dirname(os.path.dirname(torch.__file__)), "nvidia",
+                              "cuda_runtime", "lib"),
+                 "/usr/local/cuda/lib64"):
+        cands += sorted(glob.glob(os.path.join(root, "libcudart.so*")))
+    if not cands:
+        raise ImportError("libcudart.so not found")
+    return cands[0]
+
+
+def state_bytes(numel: int, bits_m: int, bits_v: int, block: int = 128) -> int:
+    out = C.c_size_t()
+    _check(lib().solo_state_bytes(numel, bits_m, bits_v, block, C.byref(out)), "solo_state_bytes")
+    return out.value
+
+
+def solo_step(param: torch.Tensor, grad: torch.Tensor, state: State, h: Hyper, step: int) -> None:
+    """One fused step on a single tensor, on the current stream."""
+    _check_tensor(param, grad, h)
+    _check(lib().solo_step(param.data_ptr(), grad.data_ptr(), state.handle, C.byref(h), step,
+                           _stream()), "solo_step")
+
+
+def _check_tensor(param: torch.Tensor, grad: torch.Tensor, h: Hyper) -> None:
+    want = torch.bfloat16 if h.param_dtype == 1 else torch.float32
+    if not (param.is_cuda and grad.is_cuda and param.is_contiguous() and grad.is_contiguous()):
+        raise ValueError("param and grad must be contiguous CUDA tensors")
+    if param.dtype != want or grad.dtype != torch.bfloat16 or param.numel() != grad.numel():
+        raise ValueError("param must be fp32/bf16 per hyper.param_dtype, grad bf16, same numel")
+
+
+class TensorSet:
+    """Device-side descriptor arrays of a tensor list (built once, reused every step)."""
+
+    def __init__(self, params: list[torch.Tensor], grads: list[torch.Tensor], state: State):
+        if len(params) != len(grads) or len(params) != len(state.sizes):
+            raise ValueError("params, grads and state must have the same number of tensors")
+        for p, g, n in zip(params, grads, state.sizes):
+            if p.numel() != n or g.numel() != n or g.dtype != torch.bfloat16:
+                raise ValueError("tensor sizes / dtypes do not match the state")
+            if not (p.is_cuda and g.is_cuda and p.is_contiguous() and g.is_contiguous()):
+                raise ValueError("tensors must be contiguous CUDA tensors")
+        dev = params[0].device
+        self.params, self.grads, self.state = params, grads, state
+        self.param_ptrs = torch.tensor([p.data_ptr() for p in params], dtype=torch.int64, device=dev)
+        self.grad_ptrs = torch.tensor([g.data_ptr() for g in grads], dtype=torch.int64, device=dev)
+        self.numel = torch.tensor(state.sizes, dtype=torch.int64, device=dev)
+        self.desc = TensorList(len(params), self.param_ptrs.data_ptr(), self.grad_ptrs.data_ptr(),
+                               self.numel.data_ptr(), state.handle)
+
+
+def solo_multi_step(ts: TensorSet, h: Hyper, step: int) -> None:
+    """One fused step over the whole tensor list in one launch, on the current stream."""
+    _check(lib().solo_multi_step(C.byref(ts.desc), C.byref(h), step, _stream()), "solo_multi_step")
+
+
+def solo_dequant(state: State, which: int) -> torch.Tensor:
+    """Dequantized first (0) or second (1) moment of every element, as a float32 CUDA tensor."""
+    out = torch.empty(sum(state.sizes), dtype=torch.float32, device=state.device)
+    _check(lib().solo_dequant(state.handle, which, out.data_ptr(), _stream()), "solo_dequant")
+    return out
+
+
+def codebook_m(bits: int) -> torch.Tensor:
+    buf = (C.c_float * (1 << bits))()
+    _check(lib().solo_codebook_m(bits, buf), "solo_codebook_m")
+    return torch.tensor(list(buf), dtype=torch.float32)
+
+
+def default_beta1(bits_m: int, from_scratch: bool = False) -> float:
+    return float(lib().solo_default_beta1(bits_m, 1 if from_scratch else 0))
+
+
+def launch_count() -> int:
+    return int(lib().solo_launch_count())

@@ -1,0 +1,416 @@
+// Host side of the C ABI declared in include/solo.h: state management, argument
+// validation, hyper-parameter reduction and kernel dispatch.
+#include "solo.h"
+
+#include <algorithm>
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "solo_device.cuh"
+#include "solo_dispatch.h"
+
+using solo::StepArgs;
+
+struct solo_state {
+    int device = 0;
+    int bits_m = 0, bits_v = 0, block = 0, num_tensors = 0;
+    int64_t numel_total = 0, nblk_total = 0, tiles_total = 0;
+    std::vector<int64_t> numel, block_start, tile_start, elem_start;  // host copies
+    // device
+    uint8_t* codes_m = nullptr;
+    uint8_t* codes_v = nullptr;
+    float* scale_m = nullptr;
+    float* scale_v = nullptr;
+    float* alpha = nullptr;
+    int64_t* geom = nullptr;      // numel[T] | block_start[T+1] | tile_start[T+1] | elem_start[T+1]
+    float* tables_m = nullptr;    // first-moment codebook tables for bits_m
+    float* tables_v = nullptr;    // same construction for bits_v (solo_dequant of m only needs bits_m)
+    int* status = nullptr;
+    size_t bytes_codes_m = 0, bytes_codes_v = 0;
+};
+
+namespace {
+
+std::atomic<int64_t> g_launches{0};
+
+bool valid_bits(int b) { return b == 2 || b == 3 || b == 4 || b == 8; }
+bool valid_block(int b) { return b == 64 || b == 128 || b == 256 || b == 2048; }
+
+// Signed dynamic-exponent levels (Appendix A), ascending.  With b bits, one is the
+// sign and the other b-1 are E zeros, a one, and F fraction bits; a magnitude is the
+// midpoint of fraction cell j of [0.1, 1] scaled by 10^-E.  Written here as the exact
+// rational (2^(F+1) + 9(2j+1)) / (10^(E+1) 2^(F+1)), one binary64 division, rounded
+// to binary32.  Zero and +1 complete the 2^b levels.
+void de_signed_levels(int bits, std::vector<float>& y) {
+    std::vector<float> pos;
+    for (int E = bits - 2; E >= 0; --E) {                 // smallest decade first
+        const int F = bits - 2 - E;
+        const double two = (double)(1 << (F + 1));
+        double ten = 10.0;
+        for (int i = 0; i < E; ++i) ten *= 10.0;
+        for (int j = 0; j < (1 << F); ++j)
+            pos.push_back((float)((two + 9.0 * (double)(2 * j + 1)) / (ten * two)));
+    }
+    y.clear();
+    for (size_t i = pos.size(); i-- > 0;) y.push_back(-pos[i]);
+    y.push_back(0.0f);
+    for (float v : pos) y.push_back(v);
+    y.push_back(1.0f);
+}
+
+// y[K] | mid[K-1] = (y[k]+y[k+1])/2 | inv_gap[K-1] = 1/(y[k+1]-y[k]), all binary32.
+void codebook_tables(int bits, std::vector<float>& t) {
+    std::vector<float> y;
+    de_signed_levels(bits, y);
+    const int K = 1 << bits;
+    t.assign(3 * K - 2, 0.0f);
+    for (int k = 0; k < K; ++k) t[k] = y[k];
+    for (int k = 0; k + 1 < K; ++k) {
+        t[K + k] = 0.5f * (y[k] + y[k + 1]);
+        t[2 * K - 1 + k] = 1.0f / (y[k + 1] - y[k]);
+    }
+}
+
+__global__ void fill_f32(float* p, int64_t n, float v) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n;
+         i += (int64_t)gridDim.x * blockDim.x)
+        p[i] = v;
+}
+
+int sm_count(int device) {
+    static std::mutex mu;
+    static int cached[64];
+    static bool have[64];
+    std::lock_guard<std::mutex> lk(mu);
+    if (device < 0 || device >= 64) return 148;
+    if (!have[device]) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || v <= 0)
+            v = 148;
+        cached[device] = v;
+        have[device] = true;
+    }
+    return cached[device];
+}
+
+int check_hyper(const solo_hyper_t* h, int64_t step) {
+    if (!h || step < 1) return SOLO_EINVAL;
+    auto unit = [](float b) { return b >= 0.0f && b < 1.0f; };
+    if (!unit(h->beta1) || !unit(h->beta2) || !unit(h->p_quantile)) return SOLO_EINVAL;
+    if (!(h->eps >= 0.0f) || !std::isfinite(h->lr) || !std::isfinite(h->weight_decay)) return SOLO_EINVAL;
+    if (h->param_dtype != 0 && h->param_dtype != 1) return SOLO_EINVAL;
+    return SOLO_OK;
+}
+
+// Bias corrections in binary64, rounded once; everything else is the caller's binary32.
+void reduce_hyper(const solo_hyper_t* h, int64_t step, int block, StepArgs& a) {
+    const double t = (double)step;
+    const double bc1 = h->bias_correction ? 1.0 - std::pow((double)h->beta1, t) : 1.0;
+    const double bc2 = h->bias_correction ? 1.0 - std::pow((double)h->beta2, t) : 1.0;
+    a.beta1 = h->beta1;
+    a.beta2 = h->beta2;
+    a.omb1 = 1.0f - h->beta1;
+    a.omb2 = 1.0f - h->beta2;
+    a.step_size = (float)((double)h->lr / bc1);
+    a.inv_sqrt_bc2 = (float)(1.0 / std::sqrt(bc2));
+    a.eps = h->eps;
+    a.decay = h->adamw ? (float)(1.0 - (double)h->lr * (double)h->weight_decay) : 1.0f;
+    a.weight_decay = h->weight_decay;
+    a.p_quantile = h->p_quantile;
+    a.l2 = (!h->adamw && h->weight_decay != 0.0f) ? 1 : 0;
+    a.round_m = h->round_m ? 1 : 0;
+    a.round_v = h->round_v ? 1 : 0;
+    a.param_bf16 = h->param_dtype;
+    a.block = block;
+    int64_t k = (int64_t)std::ceil((double)h->p_quantile * (double)block);
+    a.k_full = (int)std::min<int64_t>(std::max<int64_t>(k, 1), block);
+    a.seed_lo = (uint32_t)h->seed;
+    a.seed_hi = (uint32_t)(h->seed >> 32);
+    a.step32 = (uint32_t)step;
+}
+
+int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
+    const bool cta_group = s->block == 2048;
+    solo::StepKernel k = solo::step_kernel(s->bits_m, s->bits_v, cta_group);
+    if (!k) return SOLO_EINVAL;
+    int per_sm = solo::step_kernel_occupancy(s->bits_m, s->bits_v, cta_group);
+    if (per_sm <= 0) return SOLO_ECUDA;
+    int64_t grid = std::min<int64_t>(s->tiles_total, (int64_t)sm_count(s->device) * per_sm);
+    void* params[] = {(void*)&a};
+    cudaError_t e = cudaLaunchKernel((const void*)k, dim3((unsigned)grid), dim3(solo::CTA), params, 0, stream);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return SOLO_ECUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return SOLO_OK;
+}
+
+void fill_state_args(const solo_state* s, StepArgs& a) {
+    const int T = s->num_tensors;
+    a.numel = s->geom;
+    a.block_start = s->geom + T;
+    a.tile_start = s->geom + T + (T + 1);
+    a.num_tensors = T;
+    a.total_tiles = s->tiles_total;
+    a.codes_m = s->codes_m;
+    a.codes_v = s->codes_v;
+    a.scale_m = s->scale_m;
+    a.scale_v = s->scale_v;
+    a.alpha = s->alpha;
+    a.tables = s->tables_m;
+    a.status = s->status;
+}
+
+bool on_state_device(const solo_state* s) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == s->device;
+}
+
+}  // namespace
+
+extern "C" {
+
+int solo_state_bytes(int64_t numel, int bits_m, int bits_v, int block, size_t* out) {
+    if (!out || numel < 0 || !valid_bits(bits_m) || !valid_bits(bits_v) || !valid_block(block))
+        return SOLO_EINVAL;
+    const int64_t nblk = (numel + block - 1) / block;
+    *out = (size_t)nblk * (size_t)(block * bits_m / 8) + (size_t)nblk * (size_t)(block * bits_v / 8) +
+           (size_t)nblk * 12u;
+    return SOLO_OK;
+}
+
+int solo_state_create_multi(const int64_t* numel_host, int num_tensors, int bits_m, int bits_v,
+                            int block, solo_state_t** out) {
+    if (!out) return SOLO_EINVAL;
+    *out = nullptr;
+    if (!numel_host || num_tensors < 1 || !valid_bits(bits_m) || !valid_bits(bits_v) || !valid_block(block))
+        return SOLO_EINVAL;
+    for (int t = 0; t < num_tensors; ++t)
+        if (numel_host[t] < 1) return SOLO_EINVAL;
+    solo_state* s = new (std::nothrow) solo_state();
+    if (!s) return SOLO_ENOMEM;
+    if (cudaGetDevice(&s->device) != cudaSuccess) { delete s; return SOLO_ECUDA; }
+    s->bits_m = bits_m; s->bits_v = bits_v; s->block = block; s->num_tensors = num_tensors;
+    const int T = num_tensors;
+    s->numel.assign(numel_host, numel_host + T);
+    s->block_start.assign(T + 1, 0);
+    s->tile_start.assign(T + 1, 0);
+    s->elem_start.assign(T + 1, 0);
+    for (int t = 0; t < T; ++t) {
+        s->block_start[t + 1] = s->block_start[t] + (numel_host[t] + block - 1) / block;
+        s->tile_start[t + 1] = s->tile_start[t] + (numel_host[t] + solo::TILE - 1) / solo::TILE;
+        s->elem_start[t + 1] = s->elem_start[t] + numel_host[t];
+    }
+    s->numel_total = s->elem_start[T];
+    s->nblk_total = s->block_start[T];
+    s->tiles_total = s->tile_start[T];
+    s->bytes_codes_m = (size_t)s->nblk_total * (size_t)(block * bits_m / 8);
+    s->bytes_codes_v = (size_t)s->nblk_total * (size_t)(block * bits_v / 8);
+
+    std::vector<int64_t> geom;
+    geom.insert(geom.end(), s->numel.begin(), s->numel.end());
+    geom.insert(geom.end(), s->block_start.begin(), s->block_start.end());
+    geom.insert(geom.end(), s->tile_start.begin(), s->tile_start.end());
+    geom.insert(geom.end(), s->elem_start.begin(), s->elem_start.end());
+    std::vector<float> tm, tv;
+    codebook_tables(bits_m, tm);
+    codebook_tables(bits_v, tv);
+
+    bool ok = true;
+    auto alloc = [&](void** p, size_t bytes) {
+        if (ok && cudaMalloc(p, bytes ? bytes : 1) != cudaSuccess) { ok = false; cudaGetLastError(); }
+    };
+    // +8 bytes of slack after the codes so that the widest per-thread access of a
+    // block's last slot never leaves the allocation
+    alloc((void**)&s->codes_m, s->bytes_codes_m + 8);
+    alloc((void**)&s->codes_v, s->bytes_codes_v + 8);
+    alloc((void**)&s->scale_m, (size_t)s->nblk_total * 4);
+    alloc((void**)&s->scale_v, (size_t)s->nblk_total * 4);
+    alloc((void**)&s->alpha, (size_t)s->nblk_total * 4);
+    alloc((void**)&s->geom, geom.size() * 8);
+    alloc((void**)&s->tables_m, tm.size() * 4);
+    alloc((void**)&s->tables_v, tv.size() * 4);
+    alloc((void**)&s->status, 4);
+    if (!ok) { solo_state_destroy(s); return SOLO_ENOMEM; }
+    cudaError_t e = cudaSuccess;
+    auto chk = [&](cudaError_t r) { if (e == cudaSuccess) e = r; };
+    chk(cudaMemset(s->codes_m, 0, s->bytes_codes_m + 8));
+    chk(cudaMemset(s->codes_v, 0, s->bytes_codes_v + 8));
+    chk(cudaMemset(s->scale_m, 0, (size_t)s->nblk_total * 4));
+    chk(cudaMemset(s->scale_v, 0, (size_t)s->nblk_total * 4));
+    chk(cudaMemset(s->status, 0, 4));
+    chk(cudaMemcpy(s->geom, geom.data(), geom.size() * 8, cudaMemcpyHostToDevice));
+    chk(cudaMemcpy(s->tables_m, tm.data(), tm.size() * 4, cudaMemcpyHostToDevice));
+    chk(cudaMemcpy(s->tables_v, tv.data(), tv.size() * 4, cudaMemcpyHostToDevice));
+    if (e == cudaSuccess) {
+        fill_f32<<<1024, 256>>>(s->alpha, s->nblk_total, 0.5f);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        chk(cudaGetLastError());
+        chk(cudaDeviceSynchronize());
+    }
+    if (e != cudaSuccess) { solo_state_destroy(s); return SOLO_ECUDA; }
+    *out = s;
+    return SOLO_OK;
+}
+
+int solo_state_create(int64_t numel, int bits_m, int bits_v, int block, solo_state_t** out) {
+    return solo_state_create_multi(&numel, 1, bits_m, bits_v, block, out);
+}
+
+int solo_state_destroy(solo_state_t* s) {
+    if (!s) return SOLO_OK;
+    cudaDeviceSynchronize();
+    void* ptrs[] = {s->codes_m, s->codes_v, s->scale_m, s->scale_v, s->alpha,
+                    s->geom, s->tables_m, s->tables_v, s->status};
+    for (void* p : ptrs)
+        if (p) cudaFree(p);
+    delete s;
+    return SOLO_OK;
+}
+
+int solo_step(void* param_dev, const void* grad_dev, solo_state_t* s, const solo_hyper_t* hyper,
+              int64_t step, void* stream) {
+    if (!param_dev || !grad_dev || !s) return SOLO_EINVAL;
+    int rc = check_hyper(hyper, step);
+    if (rc) return rc;
+    if (s->num_tensors != 1 || !on_state_device(s)) return SOLO_ESTATE;
+    if ((((uintptr_t)param_dev) | ((uintptr_t)grad_dev)) & 15u) return SOLO_EALIGN;
+    StepArgs a;
+    std::memset(&a, 0, sizeof(a));
+    fill_state_args(s, a);
+    reduce_hyper(hyper, step, s->block, a);
+    a.param_single = param_dev;
+    a.grad_single = grad_dev;
+    return launch_step(s, a, (cudaStream_t)stream);
+}
+
+int solo_multi_step(const solo_tensor_list_t* list, const solo_hyper_t* hyper, int64_t step,
+                    void* stream) {
+    if (!list || !list->state || !list->param || !list->grad) return SOLO_EINVAL;
+    int rc = check_hyper(hyper, step);
+    if (rc) return rc;
+    solo_state* s = list->state;
+    if (list->num_tensors != s->num_tensors || !on_state_device(s)) return SOLO_ESTATE;
+    StepArgs a;
+    std::memset(&a, 0, sizeof(a));
+    fill_state_args(s, a);
+    reduce_hyper(hyper, step, s->block, a);
+    a.param_list = list->param;
+    a.grad_list = list->grad;
+    a.numel_check = list->numel;
+    return launch_step(s, a, (cudaStream_t)stream);
+}
+
+int solo_dequant(const solo_state_t* s, int which, float* out_dev, void* stream) {
+    if (!s || !out_dev || (which != 0 && which != 1)) return SOLO_EINVAL;
+    if (!on_state_device(s)) return SOLO_ESTATE;
+    solo::DequantArgs a;
+    std::memset(&a, 0, sizeof(a));
+    const int T = s->num_tensors;
+    a.numel = s->geom;
+    a.block_start = s->geom + T;
+    a.tile_start = s->geom + T + (T + 1);
+    a.elem_start = s->geom + T + 2 * (T + 1);
+    a.num_tensors = T;
+    a.total_tiles = s->tiles_total;
+    a.codes = which == 0 ? s->codes_m : s->codes_v;
+    a.scale = which == 0 ? s->scale_m : s->scale_v;
+    a.alpha = s->alpha;
+    a.tables = s->tables_m;
+    a.out = out_dev;
+    a.block = s->block;
+    a.which = which;
+    const int bits = which == 0 ? s->bits_m : s->bits_v;
+    int64_t grid = std::min<int64_t>(s->tiles_total, (int64_t)sm_count(s->device) * 8);
+    cudaError_t e = solo::launch_dequant(bits, a, (unsigned)grid, (cudaStream_t)stream);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return SOLO_ECUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return SOLO_OK;
+}
+
+int solo_state_raw(const solo_state_t* s, int which, void** dev_ptr, size_t* bytes) {
+    if (!s || !dev_ptr || !bytes) return SOLO_EINVAL;
+    switch (which) {
+        case 0: *dev_ptr = s->codes_m; *bytes = s->bytes_codes_m; break;
+        case 1: *dev_ptr = s->codes_v; *bytes = s->bytes_codes_v; break;
+        case 2: *dev_ptr = s->scale_m; *bytes = (size_t)s->nblk_total * 4; break;
+        case 3: *dev_ptr = s->scale_v; *bytes = (size_t)s->nblk_total * 4; break;
+        case 4: *dev_ptr = s->alpha; *bytes = (size_t)s->nblk_total * 4; break;
+        default: return SOLO_EINVAL;
+    }
+    return SOLO_OK;
+}
+
+int solo_state_info(const solo_state_t* s, int64_t* numel, int64_t* num_blocks, int32_t* num_tensors,
+                    int32_t* bits_m, int32_t* bits_v, int32_t* block) {
+    if (!s) return SOLO_EINVAL;
+    if (numel) *numel = s->numel_total;
+    if (num_blocks) *num_blocks = s->nblk_total;
+    if (num_tensors) *num_tensors = s->num_tensors;
+    if (bits_m) *bits_m = s->bits_m;
+    if (bits_v) *bits_v = s->bits_v;
+    if (block) *block = s->block;
+    return SOLO_OK;
+}
+
+int solo_state_status(solo_state_t* s, int* status_out) {
+    if (!s || !status_out) return SOLO_EINVAL;
+    if (!on_state_device(s)) return SOLO_ESTATE;
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return SOLO_ECUDA; }
+    if (cudaMemcpy(status_out, s->status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
+        cudaGetLastError();
+        return SOLO_ECUDA;
+    }
+    return SOLO_OK;
+}
+
+int solo_codebook_m(int bits, float* levels_host) {
+    if (!valid_bits(bits) || !levels_host) return SOLO_EINVAL;
+    std::vector<float> y;
+    de_signed_levels(bits, y);
+    std::memcpy(levels_host, y.data(), y.size() * 4);
+    return SOLO_OK;
+}
+
+float solo_default_beta1(int bits_m, int from_scratch) {
+    if (bits_m < 2 || bits_m > 8) return 0.0f;
+    auto r_median = [](int bits) {
+        std::vector<float> y;
+        de_signed_levels(bits, y);
+        std::vector<double> r;
+        for (size_t k = 0; k + 1 < y.size(); ++k) r.push_back(0.5 * ((double)y[k + 1] - (double)y[k]));
+        std::sort(r.begin(), r.end());
+        const size_t n = r.size();
+        return n % 2 ? r[n / 2] : 0.5 * (r[n / 2 - 1] + r[n / 2]);
+    };
+    const int b = from_scratch ? 8 : 5;
+    if (bits_m >= b) return 0.9f;
+    const double c = 0.9 / 0.1 * r_median(b) / r_median(bits_m);
+    const double bound = c / (1.0 + c);
+    return (float)(std::floor(bound * 10.0 + 1e-9) / 10.0);
+}
+
+int64_t solo_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* solo_strerror(int status) {
+    switch (status) {
+        case SOLO_OK: return "ok";
+        case SOLO_EINVAL: return "invalid argument";
+        case SOLO_EALIGN: return "parameter or gradient pointer is not 16-byte aligned";
+        case SOLO_ENOMEM: return "out of memory";
+        case SOLO_ECUDA: return "CUDA call or kernel launch failed";
+        case SOLO_ESTATE: return "state does not match the call";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,49 @@
+// Kernel lookup tables and the dequantization launcher.
+#include "solo_dispatch.h"
+
+#include <mutex>
+
+namespace solo {
+
+StepKernel step_kernel(int bits_m, int bits_v, bool cta_group) {
+    const int bv = bits_index(bits_v);
+    switch (bits_m) {
+        case 2: return step_kernel_bm2(bv, cta_group);
+        case 3: return step_kernel_bm3(bv, cta_group);
+        case 4: return step_kernel_bm4(bv, cta_group);
+        case 8: return step_kernel_bm8(bv, cta_group);
+        default: return nullptr;
+    }
+}
+
+int step_kernel_occupancy(int bits_m, int bits_v, bool cta_group) {
+    static std::mutex mu;
+    static int cache[4][4][2];
+    const int bm = bits_index(bits_m), bv = bits_index(bits_v);
+    if (bm < 0 || bv < 0) return 0;
+    std::lock_guard<std::mutex> lk(mu);
+    int& c = cache[bm][bv][cta_group ? 1 : 0];
+    if (c == 0) {
+        StepKernel k = step_kernel(bits_m, bits_v, cta_group);
+        int n = 0;
+        if (!k || cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k, CTA, 0) != cudaSuccess || n <= 0) {
+            cudaGetLastError();
+            return 0;
+        }
+        c = n;
+    }
+    return c;
+}
+
+cudaError_t launch_dequant(int bits, const DequantArgs& a, unsigned grid, cudaStream_t stream) {
+    switch (bits) {
+        case 2: solo_dequant_kernel<2><<<grid, CTA, 0, stream>>>(a); break;
+        case 3: solo_dequant_kernel<3><<<grid, CTA, 0, stream>>>(a); break;
+        case 4: solo_dequant_kernel<4><<<grid, CTA, 0, stream>>>(a); break;
+        case 8: solo_dequant_kernel<8><<<grid, CTA, 0, stream>>>(a); break;
+        default: return cudaErrorInvalidValue;
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace solo

@@ -1,0 +1,35 @@
+// Kernel lookup by (bits_m, bits_v, block kind).  The step kernel is instantiated
+// once per first-moment width in its own translation unit (solo_step_inst.cu compiled
+// with -DSOLO_BM=2,3,4,8) so that the instantiations build in parallel.
+#pragma once
+#include <cuda_runtime.h>
+
+#include "solo_device.cuh"
+
+namespace solo {
+
+using StepKernel = void (*)(const StepArgs);
+
+// Per-translation-unit tables: index [bv_index][cta_group], bv_index 0..3 for 2,3,4,8 bits.
+StepKernel step_kernel_bm2(int bv_index, bool cta_group);
+StepKernel step_kernel_bm3(int bv_index, bool cta_group);
+StepKernel step_kernel_bm4(int bv_index, bool cta_group);
+StepKernel step_kernel_bm8(int bv_index, bool cta_group);
+
+inline int bits_index(int bits) {
+    switch (bits) {
+        case 2: return 0;
+        case 3: return 1;
+        case 4: return 2;
+        case 8: return 3;
+        default: return -1;
+    }
+}
+
+StepKernel step_kernel(int bits_m, int bits_v, bool cta_group);
+// Resident CTAs per SM of that kernel (cached), 0 on error.
+int step_kernel_occupancy(int bits_m, int bits_v, bool cta_group);
+
+cudaError_t launch_dequant(int bits, const DequantArgs& a, unsigned grid, cudaStream_t stream);
+
+}  // namespace solo

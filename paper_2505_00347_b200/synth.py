@@ -165,3 +165,46 @@ def bf16_bits(t: torch.Tensor) -> np.ndarray:
 def bits_to_bf16(a: np.ndarray, device="cpu") -> torch.Tensor:
     """numpy uint16 bit patterns -> bf16 tensor."""
     return torch.from_numpy(a.view(np.int16).copy()).view(torch.bfloat16).to(device)
+
+
+def make_state(sizes, bits_m: int, bits_v: int, block: int, seed: int, device="cpu") -> dict:
+    """A random packed optimizer state for a tensor list, as torch tensors on `device` in the
+    library's layout (tensors one after the other, each starting on a new block).  Code bytes
+    are uniform random (every bit pattern is a valid code string; the padding codes of a short
+    last block are random too and must be ignored by a reader), scales are log-uniform, bases
+    uniform in (0.2, 0.98); about 3 % of the blocks are the zero state."""
+    g = _gen(device, seed, 77)
+    nb = sum(-(-int(n) // block) for n in sizes)
+    out = {}
+    zero = torch.rand(nb, device=device, generator=g) < 0.03
+    for key, b in (("m", bits_m), ("v", bits_v)):
+        slot = block * b // 8
+        codes = torch.randint(0, 256, (nb, slot), device=device, dtype=torch.uint8, generator=g)
+        codes[zero] = 0
+        out["codes_" + key] = codes.reshape(-1)
+
+    def loguniform(lo, hi):
+        u = torch.rand(nb, device=device, generator=g)
+        return torch.exp(u * (math.log(hi) - math.log(lo)) + math.log(lo)).float()
+
+    out["scale_m"] = loguniform(1e-8, 1e-1).masked_fill_(zero, 0.0)
+    out["scale_v"] = loguniform(1e-14, 1e-2).masked_fill_(zero, 0.0)
+    out["alpha"] = (torch.rand(nb, device=device, generator=g) * 0.78 + 0.2).float().masked_fill_(zero, 0.5)
+    return out
+
+
+def pack_codes(codes: np.ndarray, b: int) -> np.ndarray:
+    """[n_blocks, block] integer codes -> bytes; element e takes bits [e*b, e*b+b) of its
+    block's little-endian bit string."""
+    nb, block = codes.shape
+    bitsarr = ((codes[:, :, None].astype(np.uint16) >> np.arange(b, dtype=np.uint16)) & 1)
+    return np.packbits(bitsarr.reshape(nb, block * b).astype(np.uint8), axis=1,
+                       bitorder="little").reshape(-1)
+
+
+def unpack_codes(packed: np.ndarray, b: int, block: int) -> np.ndarray:
+    """Inverse of pack_codes: bytes -> [n_blocks, block] codes."""
+    nb = packed.size // (block * b // 8)
+    bitsarr = np.unpackbits(packed.reshape(nb, -1), axis=1, bitorder="little")
+    bitsarr = bitsarr.reshape(nb, block, b).astype(np.uint16)
+    return (bitsarr << np.arange(b, dtype=np.uint16)).sum(axis=2).astype(np.uint8)

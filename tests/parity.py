@@ -1,0 +1,200 @@
+"""Helpers shared by the GPU parity tests: run the CUDA library and the CPU oracle on the
+same seeded inputs and compare them element by element.
+
+Tolerances (north-star of the build): packed codes, scales and bases bit-exact, except codes
+of elements whose pre-quantization value the oracle flags as lying within 1e-6 relative of a
+rounding boundary (counted); parameters and dequantized states within 1e-6 relative /
+1e-9 absolute.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2505_00347_b200 import synth
+
+RTOL, ATOL = 1e-6, 1e-9
+KEYS = ("codes_m", "codes_v", "scale_m", "scale_v", "alpha")
+
+
+def hyper_pair(**kw):
+    """The same hyper-parameters for the oracle and for the library."""
+    from paper_2505_00347_b200 import binding as B
+    return oracle.hyper(**kw), B.hyper(**kw)
+
+
+def split_state(sd: dict, sizes, bits_m, bits_v, block) -> list:
+    """Library-layout host arrays -> one oracle.State per tensor (copies)."""
+    out, j = [], 0
+    sm, sv = block * bits_m // 8, block * bits_v // 8
+    for n in sizes:
+        st = oracle.State(int(n), bits_m, bits_v, block)
+        k = st.nblk
+        st.codes_m[:] = sd["codes_m"][j * sm:(j + k) * sm]
+        st.codes_v[:] = sd["codes_v"][j * sv:(j + k) * sv]
+        st.scale_m[:] = sd["scale_m"][j:j + k]
+        st.scale_v[:] = sd["scale_v"][j:j + k]
+        st.alpha[:] = sd["alpha"][j:j + k]
+        out.append(st)
+        j += k
+    return out
+
+
+def join_state(states: list) -> dict:
+    return {k: np.concatenate([getattr(s, k) for s in states]) for k in KEYS}
+
+
+def to_numpy_state(sd: dict) -> dict:
+    return {k: (v.detach().cpu().numpy().copy() if isinstance(v, torch.Tensor) else np.array(v))
+            for k, v in sd.items()}
+
+
+def upload_state(gstate, sd: dict) -> None:
+    for k in KEYS:
+        v = sd[k]
+        gstate.raw_set(k, v if isinstance(v, torch.Tensor) else torch.from_numpy(np.ascontiguousarray(v)))
+
+
+def download_state(gstate) -> dict:
+    return {k: gstate.raw_get(k).numpy().copy() for k in KEYS}
+
+
+def zero_state(sizes, bits_m, bits_v, block) -> dict:
+    return join_state([oracle.State(int(n), bits_m, bits_v, block) for n in sizes])
+
+
+class Report:
+    def __init__(self):
+        self.elements = 0
+        self.exempt_m = 0
+        self.exempt_v = 0
+        self.max_param_rel = 0.0
+
+    def __repr__(self):
+        return (f"elements={self.elements} exempt_m={self.exempt_m} exempt_v={self.exempt_v} "
+                f"max_param_err={self.max_param_rel:.3g}")
+
+
+def close(a: np.ndarray, b: np.ndarray) -> np.ndarray:
+    """|a - b| <= 1e-6 |b| + 1e-9, NaN equal to NaN."""
+    a64, b64 = a.astype(np.float64), b.astype(np.float64)
+    with np.errstate(invalid="ignore"):
+        ok = np.abs(a64 - b64) <= RTOL * np.abs(b64) + ATOL
+    return ok | (np.isnan(a64) & np.isnan(b64)) | (a64 == b64)
+
+
+def compare_states(got: dict, want: dict, flags_per_block, bits_m, bits_v, block, rep: Report, where=""):
+    """got / want: library-layout host arrays.  flags_per_block: uint8 [n_blocks, block]
+    (bit 0: m within 1e-6 of a boundary, bit 1: v) or None."""
+    for k in ("scale_m", "scale_v", "alpha"):
+        g, w = got[k].view(np.uint32), want[k].view(np.uint32)
+        both_nan = np.isnan(got[k]) & np.isnan(want[k])
+        bad = (g != w) & ~both_nan
+        assert not bad.any(), (where, k, int(bad.sum()), np.nonzero(bad)[0][:5], got[k][bad][:5], want[k][bad][:5])
+    for key, b, bit in (("codes_m", bits_m, 1), ("codes_v", bits_v, 2)):
+        if np.array_equal(got[key], want[key]):
+            continue
+        g = synth.unpack_codes(got[key], b, block)
+        w = synth.unpack_codes(want[key], b, block)
+        diff = g != w
+        if flags_per_block is None:
+            assert not diff.any(), (where, key, int(diff.sum()))
+        exempt = diff & ((flags_per_block & bit) != 0)
+        hard = diff & ~exempt
+        assert not hard.any(), (where, key, int(hard.sum()), np.argwhere(hard)[:5], g[hard][:5], w[hard][:5])
+        if bit == 1:
+            rep.exempt_m += int(exempt.sum())
+        else:
+            rep.exempt_v += int(exempt.sum())
+
+
+def flags_to_blocks(flags_list, sizes, block) -> np.ndarray:
+    rows = []
+    for f, n in zip(flags_list, sizes):
+        nb = -(-int(n) // block)
+        pad = np.zeros(nb * block, np.uint8)
+        pad[:int(n)] = f
+        rows.append(pad.reshape(nb, block))
+    return np.concatenate(rows)
+
+
+def run_lockstep(sizes, bits_m, bits_v, block, hyper_kw, steps, grads_fn, params0, state0=None,
+                 multi=None, free_run=False, nthreads=8):
+    """Runs `steps` steps on both sides.
+
+    lock-step (free_run=False): before every step the library's state and parameters are set to
+    the oracle's, so each step is compared on identical inputs.  free_run=True: the library runs
+    on its own state for all steps and the final result is compared.
+    grads_fn(step) -> list of CPU bf16 tensors; params0: list of CPU tensors (fp32 or bf16).
+    """
+    from paper_2505_00347_b200 import binding as B
+    sizes = [int(n) for n in sizes]
+    multi = len(sizes) > 1 if multi is None else multi
+    ho, hg = hyper_pair(**hyper_kw)
+    bf16p = hyper_kw.get("param_dtype", 0) == 1
+    rep = Report()
+    sd = zero_state(sizes, bits_m, bits_v, block) if state0 is None else to_numpy_state(state0)
+    ostates = split_state(sd, sizes, bits_m, bits_v, block)
+    if bf16p:
+        oparams = [synth.bf16_bits(p) for p in params0]
+    else:
+        oparams = [p.numpy().copy() for p in params0]
+    gstate = B.State(sizes if multi else sizes[0], bits_m, bits_v, block)
+    upload_state(gstate, sd)
+    gparams = [p.clone().cuda() for p in params0]
+    ts = None
+
+    def gpu_step(t, ggrads):
+        nonlocal ts
+        if multi:
+            ts = B.TensorSet(gparams, ggrads, gstate)
+            B.solo_multi_step(ts, hg, t)
+        else:
+            B.solo_step(gparams[0], ggrads[0], gstate, hg, t)
+        torch.cuda.synchronize()
+        assert gstate.status() == 0
+
+    def compare(t, flags):
+        got = download_state(gstate)
+        want = join_state(ostates)
+        fl = flags_to_blocks(flags, sizes, block)
+        compare_states(got, want, fl, bits_m, bits_v, block, rep, where=f"step {t}")
+        exempt_elem = fl.reshape(-1) != 0
+        off = 0
+        boff = 0
+        dm, dv = B.solo_dequant(gstate, 0).cpu().numpy(), B.solo_dequant(gstate, 1).cpu().numpy()
+        for i, n in enumerate(sizes):
+            gp = gparams[i].float().cpu().numpy() if bf16p else gparams[i].cpu().numpy()
+            wp = (synth.bits_to_bf16(oparams[i]).float().numpy() if bf16p else oparams[i])
+            ok = close(gp, wp)
+            assert ok.all(), (f"step {t} tensor {i} params", int((~ok).sum()), gp[~ok][:4], wp[~ok][:4])
+            with np.errstate(invalid="ignore", divide="ignore"):
+                rel = np.nanmax(np.abs(gp.astype(np.float64) - wp) / (np.abs(wp) + 1e-3)) if n else 0.0
+            rep.max_param_rel = max(rep.max_param_rel, float(rel))
+            nb = -(-n // block)
+            ex = exempt_elem[boff * block: boff * block + n]
+            for which, d in ((0, dm), (1, dv)):
+                ok = close(d[off:off + n], oracle.dequant(ostates[i], which)) | ex
+                assert ok.all(), (f"step {t} tensor {i} dequant {which}", int((~ok).sum()))
+            off += n
+            boff += nb
+        rep.elements += sum(sizes)
+
+    for t in range(1, steps + 1):
+        grads = grads_fn(t)
+        ggrads = [g.cuda() for g in grads]
+        if not free_run and t > 1:
+            upload_state(gstate, join_state(ostates))
+            for gp, op in zip(gparams, oparams):
+                gp.copy_(synth.bits_to_bf16(op) if bf16p else torch.from_numpy(op))
+        gpu_step(t, ggrads)
+        flags = []
+        for i, n in enumerate(sizes):
+            _, _, fl = oracle.step(oparams[i], synth.bf16_bits(grads[i]), ostates[i], ho, t, tensor=i,
+                                   nthreads=nthreads, want_flags=True)
+            flags.append(fl)
+        if not free_run or t == steps:
+            compare(t, flags)
+    gstate.destroy()
+    return rep
