@@ -146,7 +146,11 @@ __device__ __forceinline__ uint32_t group_select(uint32_t (&key)[EPT], int k, ui
         cswap(key[1], key[4]); cswap(key[3], key[6]);
         cswap(key[2], key[4]); cswap(key[3], key[5]);
         cswap(key[3], key[4]);
+        // Row j of the lane's column holds its (j+1)-th smallest key; row 0 holds the
+        // "exhausted" sentinel, so that popping is one unconditional load and two selects
+        // (no divergent branch between the warp-synchronous operations of the loop).
         uint32_t* mine = s_sort + threadIdx.x;
+        mine[0] = 0xFFFFFFFFu;
 #pragma unroll
         for (int j = 1; j < EPT; ++j) mine[j * CTA] = key[j];
         uint32_t head = key[0];
@@ -154,13 +158,13 @@ __device__ __forceinline__ uint32_t group_select(uint32_t (&key)[EPT], int k, ui
         uint32_t gmin;
         while (true) {
             gmin = __reduce_min_sync(mask, head);
-            bool eq = head == gmin;
+            const bool eq = head == gmin;
             cnt += __popc(__ballot_sync(mask, eq));
             if (cnt >= k) break;
-            if (eq) {
-                ++ptr;
-                head = ptr < EPT ? mine[ptr * CTA] : 0xFFFFFFFFu;
-            }
+            const int np = ptr + 1;
+            const uint32_t nxt = mine[(np & (EPT - 1)) * CTA];
+            head = eq ? nxt : head;
+            ptr = eq ? np : ptr;
         }
         return gmin;
     } else {
