@@ -85,8 +85,8 @@ def lib() -> C.CDLL:
         getattr(L, name).restype = C.c_float
     L.so_philox4x32_10.argtypes = [u32p, u32p, u32p]
     L.so_philox4x32_10.restype = None
-    L.so_philox_word.argtypes = [C.c_uint64, C.c_int64, C.c_int32, C.c_int64, C.c_int]
-    L.so_philox_word.restype = C.c_uint32
+    L.so_philox_draw16.argtypes = [C.c_uint64, C.c_int64, C.c_int32, C.c_int64, C.c_int]
+    L.so_philox_draw16.restype = C.c_uint32
     for name in ("so_xi", "so_u"):
         getattr(L, name).argtypes = [C.c_uint32]
         getattr(L, name).restype = C.c_float
@@ -151,16 +151,17 @@ def philox4x32_10(ctr, key) -> np.ndarray:
     return out
 
 
-def philox_word(seed: int, step: int, tensor: int, idx: int, purpose: int) -> int:
-    return int(lib().so_philox_word(seed, step, tensor, idx, purpose))
+def philox_draw16(seed: int, step: int, tensor: int, idx: int, purpose: int) -> int:
+    """The 16-bit draw of element ``idx`` (purpose 0: second moment, 1: first moment)."""
+    return int(lib().so_philox_draw16(seed, step, tensor, idx, purpose))
 
 
-def xi(word: int) -> float:
-    return lib().so_xi(word)
+def xi(draw16: int) -> float:
+    return lib().so_xi(draw16)
 
 
-def u01(word: int) -> float:
-    return lib().so_u(word)
+def u01(draw16: int) -> float:
+    return lib().so_u(draw16)
 
 
 def quant_nearest(levels: np.ndarray, r: float) -> int:

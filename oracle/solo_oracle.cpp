@@ -166,26 +166,30 @@ void philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]
 
 enum Purpose { PURPOSE_V = 0, PURPOSE_M = 1 };
 
-// The 32-bit word that belongs to element `idx` of tensor `tensor` at `step`:
-// key = seed, counter = (idx/4 low, idx/4 high, step, 4*tensor + purpose),
-// word idx mod 4.
-uint32_t philox_word(uint64_t seed, int64_t step, int32_t tensor, int64_t idx, int purpose) {
-    uint64_t q = (uint64_t)idx >> 2;
+// The 16-bit draw that belongs to element `idx` of tensor `tensor` at `step`.
+// One Philox call serves eight consecutive elements:
+// key = seed, counter = (idx/8 low, idx/8 high, step, 4*tensor + purpose);
+// element idx takes halfword idx mod 8 of the 128 output bits, i.e. the low
+// (even idx) or high (odd idx) half of output word (idx mod 8) / 2.
+uint32_t philox_draw16(uint64_t seed, int64_t step, int32_t tensor, int64_t idx, int purpose) {
+    uint64_t q = (uint64_t)idx >> 3;
     uint32_t ctr[4] = {(uint32_t)q, (uint32_t)(q >> 32), (uint32_t)step,
                        (uint32_t)tensor * 4u + (uint32_t)purpose};
     uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
     uint32_t out[4];
     philox4x32_10(ctr, key, out);
-    return out[idx & 3];
+    uint32_t w = out[(idx & 7) >> 1];
+    return (idx & 1) ? (w >> 16) : (w & 0xFFFFu);
 }
 
-// xi ~ U(-1/2, 1/2) of Eq. 6: 23 random bits on a symmetric grid that never
-// touches +-1/2.
-inline float xi_from_word(uint32_t w) {
-    return (float)(w >> 9) * 0x1p-23f - 0.5f + 0x1p-24f;
+// xi ~ U(-1/2, 1/2) of Eq. 6 from a 16-bit draw d: the midpoints of 2^16 equal
+// cells of [-1/2, 1/2], a symmetric grid that never touches +-1/2.  Every value
+// is exact in binary32.
+inline float xi_from_draw(uint32_t d) {
+    return (float)(d & 0xFFFFu) * 0x1p-16f - 0.5f + 0x1p-17f;
 }
-// u ~ U[0, 1) for Eq. 5: 24 random bits.
-inline float u_from_word(uint32_t w) { return (float)(w >> 8) * 0x1p-24f; }
+// u ~ U[0, 1) for Eq. 5 from a 16-bit draw.
+inline float u_from_draw(uint32_t d) { return (float)(d & 0xFFFFu) * 0x1p-16f; }
 
 // ---------------------------------------------------------------------------
 // Quantizers.
@@ -302,11 +306,11 @@ float so_exp2_sp(float x) { return exp2_sp(x); }
 void so_philox4x32_10(const uint32_t* ctr, const uint32_t* key, uint32_t* out) {
     philox4x32_10(ctr, key, out);
 }
-uint32_t so_philox_word(uint64_t seed, int64_t step, int32_t tensor, int64_t idx, int purpose) {
-    return philox_word(seed, step, tensor, idx, purpose);
+uint32_t so_philox_draw16(uint64_t seed, int64_t step, int32_t tensor, int64_t idx, int purpose) {
+    return philox_draw16(seed, step, tensor, idx, purpose);
 }
-float so_xi(uint32_t w) { return xi_from_word(w); }
-float so_u(uint32_t w) { return u_from_word(w); }
+float so_xi(uint32_t d) { return xi_from_draw(d); }
+float so_u(uint32_t d) { return u_from_draw(d); }
 int so_quant_nearest(const float* y, int K, float r) { return quant_nearest(y, K, r); }
 int so_quant_stochastic(const float* y, int K, float r, float u) {
     return quant_stochastic(y, K, r, u);
@@ -438,8 +442,8 @@ static void step_blocks(void* param, const uint16_t* grad, int64_t n, int64_t el
                 float r = mh[e] * inv;
                 int q;
                 if (h->round_m) {
-                    uint32_t w = philox_word(h->seed, step, tensor, elem_offset + e0 + e, PURPOSE_M);
-                    q = quant_stochastic(ym, Km, r, u_from_word(w));
+                    uint32_t d = philox_draw16(h->seed, step, tensor, elem_offset + e0 + e, PURPOSE_M);
+                    q = quant_stochastic(ym, Km, r, u_from_draw(d));
                 } else {
                     q = quant_nearest(ym, Km, r);
                     if (flags) {
@@ -475,8 +479,8 @@ static void step_blocks(void* param, const uint16_t* grad, int64_t n, int64_t el
                 float r = vh[e] * inv;
                 float xi = 0.0f;
                 if (h->round_v) {
-                    uint32_t w = philox_word(h->seed, step, tensor, elem_offset + e0 + e, PURPOSE_V);
-                    xi = xi_from_word(w);
+                    uint32_t d = philox_draw16(h->seed, step, tensor, elem_offset + e0 + e, PURPOSE_V);
+                    xi = xi_from_draw(d);
                 }
                 int q = quant_log(r, inv_lambda, xi, Kv);
                 set_code(cv, e, bits_v, q);
@@ -542,8 +546,9 @@ int so_hardware_threads(void) { return (int)std::thread::hardware_concurrency();
 // signal swamping (Thm 3.1, Cor. 3.2, Example 3.3), exact decay (Prop. 3.5) and
 // stochastic rounding (Thm 3.6).
 //   mode 0: nearest rounding (Eq. 1) on codebook `kind`
-//   mode 1: stochastic rounding (Eq. 5) on codebook `kind`, u from `rnd` (n words)
-//   mode 2: SOLO logarithmic quantizer (Eq. 6), xi from `rnd` (null: xi = 0);
+//   mode 1: stochastic rounding (Eq. 5) on codebook `kind`, u from the upper
+//           halves of `rnd` (n words, one 16-bit draw each)
+//   mode 2: SOLO logarithmic quantizer (Eq. 6), xi from `rnd` likewise (null: xi = 0);
 //           fixed_alpha > 0 keeps that base, otherwise the base comes from the
 //           p-quantile of the new values.
 // codes: one int per element (unpacked).  delta/alpha: in/out scalars.
@@ -587,11 +592,11 @@ int so_qema(int mode, int kind, int bits, int64_t n, int32_t* codes, float* delt
             *alpha = log_base(s[k - 1], inv, K0, &inv_lambda);
         }
         for (int64_t i = 0; i < n; ++i)
-            codes[i] = quant_log(xh[i] * inv, inv_lambda, rnd ? xi_from_word(rnd[i]) : 0.0f, K0);
+            codes[i] = quant_log(xh[i] * inv, inv_lambda, rnd ? xi_from_draw(rnd[i] >> 16) : 0.0f, K0);
     } else {
         for (int64_t i = 0; i < n; ++i) {
             float r = xh[i] * inv;
-            codes[i] = mode == 1 ? quant_stochastic(y, K, r, u_from_word(rnd[i]))
+            codes[i] = mode == 1 ? quant_stochastic(y, K, r, u_from_draw(rnd[i] >> 16))
                                  : quant_nearest(y, K, r);
         }
     }

@@ -157,20 +157,26 @@ def test_philox_known_answers():
         assert tuple(int(x) for x in oracle.philox4x32_10(ctr, key)) == out
 
 
-def test_philox_word_addressing_and_uniforms():
+def test_philox_draw_addressing_and_uniforms():
+    """One Philox call serves eight elements; element idx takes halfword idx mod 8."""
     seed, step, tensor = 0x1234_5678_9ABC_DEF0, 7, 3
-    for idx in (0, 1, 2, 3, 4, 5, (1 << 34) + 6):
-        blockwords = oracle.philox4x32_10(
-            ((idx >> 2) & 0xffffffff, (idx >> 2) >> 32, step, tensor * 4 + 1),
+    for idx in (0, 1, 2, 3, 4, 5, 6, 7, 8, 13, (1 << 36) + 6, (1 << 36) + 7):
+        words = oracle.philox4x32_10(
+            ((idx >> 3) & 0xffffffff, (idx >> 3) >> 32, step, tensor * 4 + 1),
             (seed & 0xffffffff, seed >> 32))
-        assert oracle.philox_word(seed, step, tensor, idx, 1) == int(blockwords[idx & 3])
-    # xi lies strictly inside (-1/2, 1/2), is symmetric and uses 23 bits; u in [0, 1)
-    assert oracle.xi(0) == -0.5 + 2.0 ** -24 and oracle.xi(0xffffffff) == 0.5 - 2.0 ** -24
-    assert oracle.xi(0x80000000) == 2.0 ** -24 and oracle.xi(0x7fffffff) == -(2.0 ** -24)
-    assert oracle.u01(0) == 0.0 and oracle.u01(0xffffffff) == 1.0 - 2.0 ** -24
-    words = [oracle.philox_word(1, 1, 0, i, 0) for i in range(4000)]
-    xs = np.array([oracle.xi(w) for w in words])
+        halves = [int(w) >> s & 0xffff for w in words for s in (0, 16)]
+        assert oracle.philox_draw16(seed, step, tensor, idx, 1) == halves[idx & 7]
+    # xi: midpoints of 2^16 cells of [-1/2, 1/2]: strictly inside, symmetric; u in [0, 1)
+    assert oracle.xi(0) == -0.5 + 2.0 ** -17 and oracle.xi(0xffff) == 0.5 - 2.0 ** -17
+    assert oracle.xi(0x8000) == 2.0 ** -17 and oracle.xi(0x7fff) == -(2.0 ** -17)
+    for d in (0, 1, 0x1234, 0x7fff, 0xffff):
+        assert oracle.xi(d) == -oracle.xi(0xffff - d)
+        assert oracle.xi(d) == (d + 0.5) / 65536 - 0.5          # exact in binary32
+    assert oracle.u01(0) == 0.0 and oracle.u01(0xffff) == 1.0 - 2.0 ** -16
+    draws = [oracle.philox_draw16(1, 1, 0, i, 0) for i in range(4000)]
+    xs = np.array([oracle.xi(d) for d in draws])
     assert abs(xs.mean()) < 0.02 and abs(xs.var() - 1 / 12) < 0.01
+    assert len(set(draws)) > 3800                              # halves of a word are not copies
 
 
 def test_log2_exp2_accuracy():

@@ -100,7 +100,7 @@ def test_block_quantities_rederived(bits_m, bits_v, block):
             rv = vh[sl].astype(np.float64) / float(st.scale_v[j])
             qv = np.array([oracle.get_code(st.codes_v[j * (block * bits_v // 8):], e, bits_v) for e in range(nb)])
             for e in range(nb):
-                w = oracle.philox_word(99, t, 2, sl.start + e, 0)
+                w = oracle.philox_draw16(99, t, 2, sl.start + e, 0)
                 tt = math.log(rv[e]) / math.log(a) + oracle.xi(w) if rv[e] > 0 else Kv
                 q_ref_v = int(min(max(round(tt), 0), Kv - 1))
                 assert qv[e] == q_ref_v or abs(tt - math.floor(tt) - 0.5) < 2e-4, (j, e, tt, qv[e])
