@@ -128,6 +128,7 @@ def run_ours(args, rank, world):
     torch.cuda.set_device(local)
     device = torch.device("cuda", local)
     w, params, grads = build_workload(args.workload, device, args)
+    B.set_kernel_policy(args.policy)
     state = B.State(list(w.sizes), w.bits_m, w.bits_v, w.block)
     ts = B.TensorSet(params, grads, state)
     h = B.hyper(lr=w.lr, beta1=w.beta1, beta2=w.beta2, weight_decay=w.weight_decay, seed=1234)
@@ -273,6 +274,7 @@ def main():
     ap.add_argument("--max-tensors", type=int, default=0, help="use only the first tensors (small captures)")
     ap.add_argument("--cpu-sample", type=int, default=1 << 27)
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--policy", type=int, default=0, help="kernel policy: 0 streamlined where it applies, 1 general")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -174,6 +174,26 @@ int solo_codebook_m(int bits, float* levels_host);
  */
 float solo_default_beta1(int bits_m, int from_scratch);
 
+/*
+ * Kernel selection.  0 (default): configurations with 2/3/4-bit states, block 128 or 256,
+ * fp32 parameters, nearest rounding of the first moment and eps >= 1e-12 run the
+ * streamlined kernel, everything else the general one.  1: always the general kernel.  Both produce the same
+ * packed state; the streamlined kernel's parameters differ from the IEEE sequence of
+ * divisions and square roots by at most a few 1e-7 of the update term.  Process-wide.
+ */
+int solo_set_kernel_policy(int policy);
+
+/*
+ * Test hook for the streamlined kernel's rounding guard in Eq. 6: compares the hardware
+ * base-2 logarithm approximation with the exact operation sequence for every binary32
+ * whose bit pattern lies in [lo_bits, hi_bits] (positive normal numbers).  Writes to
+ * HOST *max_excess_host the largest |approx - exact| - rel/2 * |exact| seen (or -1) and to
+ * *abs_bound_host the absolute bound the kernel assumes; the guard is sound while the
+ * former stays below half of the latter.  Synchronous; allocates 4 bytes of device memory.
+ */
+int solo_debug_check_fast_log(uint32_t lo_bits, uint32_t hi_bits, float* max_excess_host,
+                              float* abs_bound_host);
+
 /* Number of kernel launches issued by this library in the calling process so far. */
 int64_t solo_launch_count(void);
 

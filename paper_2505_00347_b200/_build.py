@@ -28,6 +28,9 @@ UNITS = [
     ("solo_step_inst.cu", "solo_step_bm3.o", ["-DSOLO_BM=3"]),
     ("solo_step_inst.cu", "solo_step_bm4.o", ["-DSOLO_BM=4"]),
     ("solo_step_inst.cu", "solo_step_bm8.o", ["-DSOLO_BM=8"]),
+    ("solo_fast_inst.cu", "solo_fast_bm2.o", ["-DSOLO_BM=2"]),
+    ("solo_fast_inst.cu", "solo_fast_bm3.o", ["-DSOLO_BM=3"]),
+    ("solo_fast_inst.cu", "solo_fast_bm4.o", ["-DSOLO_BM=4"]),
 ]
 
 

@@ -78,13 +78,17 @@ def lib() -> C.CDLL:
     L.solo_codebook_m.argtypes = [i32, C.POINTER(C.c_float)]
     L.solo_default_beta1.argtypes = [i32, i32]
     L.solo_default_beta1.restype = C.c_float
+    L.solo_set_kernel_policy.argtypes = [i32]
+    L.solo_debug_check_fast_log.argtypes = [C.c_uint32, C.c_uint32, C.POINTER(C.c_float),
+                                            C.POINTER(C.c_float)]
     L.solo_launch_count.argtypes = []
     L.solo_launch_count.restype = C.c_int64
     L.solo_strerror.argtypes = [i32]
     L.solo_strerror.restype = C.c_char_p
     for name in ("solo_state_create", "solo_state_create_multi", "solo_state_destroy",
                  "solo_state_bytes", "solo_step", "solo_multi_step", "solo_dequant",
-                 "solo_state_raw", "solo_state_info", "solo_state_status", "solo_codebook_m"):
+                 "solo_state_raw", "solo_state_info", "solo_state_status", "solo_codebook_m",
+                 "solo_set_kernel_policy", "solo_debug_check_fast_log"):
         getattr(L, name).restype = C.c_int
     _lib = L
     return L
@@ -265,6 +269,19 @@ def codebook_m(bits: int) -> torch.Tensor:
 
 def default_beta1(bits_m: int, from_scratch: bool = False) -> float:
     return float(lib().solo_default_beta1(bits_m, 1 if from_scratch else 0))
+
+
+def set_kernel_policy(policy: int) -> None:
+    """0: streamlined kernel where it applies (default); 1: always the general kernel."""
+    _check(lib().solo_set_kernel_policy(policy), "solo_set_kernel_policy")
+
+
+def debug_check_fast_log(lo_bits: int, hi_bits: int) -> tuple[float, float]:
+    """(largest excess of the lg2 approximation over the relative bound, assumed absolute bound)."""
+    ex, ab = C.c_float(), C.c_float()
+    _check(lib().solo_debug_check_fast_log(lo_bits, hi_bits, C.byref(ex), C.byref(ab)),
+           "solo_debug_check_fast_log")
+    return ex.value, ab.value
 
 
 def launch_count() -> int:

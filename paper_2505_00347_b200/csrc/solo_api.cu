@@ -37,6 +37,7 @@ struct solo_state {
 namespace {
 
 std::atomic<int64_t> g_launches{0};
+std::atomic<int> g_policy{0};          // 0: pick the streamlined kernel where it applies; 1: general kernel only
 
 bool valid_bits(int b) { return b == 2 || b == 3 || b == 4 || b == 8; }
 bool valid_block(int b) { return b == 64 || b == 128 || b == 256 || b == 2048; }
@@ -132,13 +133,20 @@ void reduce_hyper(const solo_hyper_t* h, int64_t step, int block, StepArgs& a) {
     a.seed_lo = (uint32_t)h->seed;
     a.seed_hi = (uint32_t)(h->seed >> 32);
     a.step32 = (uint32_t)step;
+    for (int r = 0; r < 10; ++r) {
+        a.rk[2 * r] = a.seed_lo + (uint32_t)r * 0x9E3779B9u;
+        a.rk[2 * r + 1] = a.seed_hi + (uint32_t)r * 0xBB67AE85u;
+    }
 }
 
 int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
     const bool cta_group = s->block == 2048;
-    solo::StepKernel k = solo::step_kernel(s->bits_m, s->bits_v, cta_group);
+    solo::StepKernel k = nullptr;
+    if (g_policy.load(std::memory_order_relaxed) == 0 && !a.round_m && !a.param_bf16 && a.eps >= 1e-12f)
+        k = solo::fast_kernel(s->bits_m, s->bits_v, s->block);
+    if (!k) k = solo::step_kernel(s->bits_m, s->bits_v, cta_group);
     if (!k) return SOLO_EINVAL;
-    int per_sm = solo::step_kernel_occupancy(s->bits_m, s->bits_v, cta_group);
+    int per_sm = solo::kernel_occupancy(k);
     if (per_sm <= 0) return SOLO_ECUDA;
     int64_t grid = std::min<int64_t>(s->tiles_total, (int64_t)sm_count(s->device) * per_sm);
     void* params[] = {(void*)&a};
@@ -397,6 +405,30 @@ float solo_default_beta1(int bits_m, int from_scratch) {
     const double c = 0.9 / 0.1 * r_median(b) / r_median(bits_m);
     const double bound = c / (1.0 + c);
     return (float)(std::floor(bound * 10.0 + 1e-9) / 10.0);
+}
+
+int solo_set_kernel_policy(int policy) {
+    if (policy != 0 && policy != 1) return SOLO_EINVAL;
+    g_policy.store(policy, std::memory_order_relaxed);
+    return SOLO_OK;
+}
+
+int solo_debug_check_fast_log(uint32_t lo_bits, uint32_t hi_bits, float* max_excess_host,
+                              float* abs_bound_host) {
+    if (!max_excess_host || !abs_bound_host || lo_bits > hi_bits || lo_bits < 0x00800000u ||
+        hi_bits >= 0x7F800000u)
+        return SOLO_EINVAL;
+    float* d = nullptr;
+    if (cudaMalloc((void**)&d, 4) != cudaSuccess) { cudaGetLastError(); return SOLO_ENOMEM; }
+    const float init = -1.0f;
+    cudaError_t e = cudaMemcpy(d, &init, 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = solo::launch_fast_log_check(lo_bits, hi_bits, d, nullptr);
+    if (e == cudaSuccess) g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (e == cudaSuccess) e = cudaMemcpy(max_excess_host, d, 4, cudaMemcpyDeviceToHost);
+    cudaFree(d);
+    if (e != cudaSuccess) { cudaGetLastError(); return SOLO_ECUDA; }
+    *abs_bound_host = solo::fast_log_abs_bound();
+    return SOLO_OK;
 }
 
 int64_t solo_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

@@ -51,6 +51,8 @@ struct StepArgs {
     float beta1, beta2, omb1, omb2, step_size, inv_sqrt_bc2, eps, decay, weight_decay, p_quantile;
     int32_t l2, round_m, round_v, param_bf16, block, k_full;
     uint32_t seed_lo, seed_hi, step32;
+    // Philox round keys (seed + r * Weyl constant), r = 0..9: [2r] low word, [2r+1] high word
+    uint32_t rk[20];
 };
 
 // ---------------------------------------------------------------------------
@@ -107,6 +109,11 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
         k1 += 0xBB67AE85u;
     }
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// 16-bit draw of element i (0..7) of a thread's eight: halfword i of the Philox block.
+__device__ __forceinline__ uint32_t draw16(const uint32_t (&w)[4], int i) {
+    return (i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xFFFFu);
 }
 
 // ---------------------------------------------------------------------------
@@ -400,13 +407,11 @@ __global__ void __launch_bounds__(CTA) solo_step_kernel(const StepArgs a) {
         uint64_t om = 0;
         if (!zero_m) {
             const float inv = 1.0f / dm_new;
-            uint32_t wm[EPT];
+            uint32_t wm[4];
             if (a.round_m) {
-                const uint64_t c = (uint64_t)e0 >> 2;
+                const uint64_t c = (uint64_t)e0 >> 3;             // one Philox block per 8 elements
                 philox4x32_10((uint32_t)c, (uint32_t)(c >> 32), a.step32, (uint32_t)tensor * 4u + 1u,
                               a.seed_lo, a.seed_hi, wm);
-                philox4x32_10((uint32_t)(c + 1), (uint32_t)((c + 1) >> 32), a.step32,
-                              (uint32_t)tensor * 4u + 1u, a.seed_lo, a.seed_hi, wm + 4);
             }
 #pragma unroll
             for (int i = 0; i < EPT; ++i) {
@@ -419,7 +424,7 @@ __global__ void __launch_bounds__(CTA) solo_step_kernel(const StepArgs a) {
                         if (c <= KM - 2 && r >= s_y[c]) q = c;
                     }
                     const float frac = (r - s_y[q]) * s_gap[q];
-                    const float u = (float)(wm[i] >> 8) * 0x1p-24f;
+                    const float u = (float)draw16(wm, i) * 0x1p-16f;
                     q += u < frac ? 1u : 0u;
                 } else {
 #pragma unroll
@@ -445,18 +450,16 @@ __global__ void __launch_bounds__(CTA) solo_step_kernel(const StepArgs a) {
             const float lam = log2_sp(rho) * (1.0f / (float)(KV - 1));
             al_new = exp2_sp(lam);
             const float inv_lambda = 1.0f / log2_sp(al_new);
-            uint32_t wv[EPT];
+            uint32_t wv[4];
             if (a.round_v) {
-                const uint64_t c = (uint64_t)e0 >> 2;
+                const uint64_t c = (uint64_t)e0 >> 3;
                 philox4x32_10((uint32_t)c, (uint32_t)(c >> 32), a.step32, (uint32_t)tensor * 4u,
                               a.seed_lo, a.seed_hi, wv);
-                philox4x32_10((uint32_t)(c + 1), (uint32_t)((c + 1) >> 32), a.step32,
-                              (uint32_t)tensor * 4u, a.seed_lo, a.seed_hi, wv + 4);
             }
 #pragma unroll
             for (int i = 0; i < EPT; ++i) {
                 const float r = vh[i] * inv;
-                const float xi = a.round_v ? (float)(wv[i] >> 9) * 0x1p-23f - 0.5f + 0x1p-24f : 0.0f;
+                const float xi = a.round_v ? (float)draw16(wv, i) * 0x1p-16f - 0.5f + 0x1p-17f : 0.0f;
                 uint32_t q = KV - 1;
                 if (!(r < TINY)) {
                     float t = __fmaf_rn(log2_sp(r), inv_lambda, xi);

@@ -1,6 +1,7 @@
 // Kernel lookup tables and the dequantization launcher.
 #include "solo_dispatch.h"
 
+#include <map>
 #include <mutex>
 
 namespace solo {
@@ -14,6 +15,33 @@ StepKernel step_kernel(int bits_m, int bits_v, bool cta_group) {
         case 8: return step_kernel_bm8(bv, cta_group);
         default: return nullptr;
     }
+}
+
+StepKernel fast_kernel(int bits_m, int bits_v, int block) {
+    const int bv = bits_index(bits_v);
+    if (bv < 0 || bv > 2) return nullptr;
+    switch (bits_m) {
+        case 2: return fast_kernel_bm2(bv, block);
+        case 3: return fast_kernel_bm3(bv, block);
+        case 4: return fast_kernel_bm4(bv, block);
+        default: return nullptr;
+    }
+}
+
+int kernel_occupancy(StepKernel k) {
+    static std::mutex mu;
+    static std::map<const void*, int> cache;
+    if (!k) return 0;
+    std::lock_guard<std::mutex> lk(mu);
+    auto it = cache.find((const void*)k);
+    if (it != cache.end()) return it->second;
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k, CTA, 0) != cudaSuccess || n <= 0) {
+        cudaGetLastError();
+        return 0;
+    }
+    cache[(const void*)k] = n;
+    return n;
 }
 
 int step_kernel_occupancy(int bits_m, int bits_v, bool cta_group) {

@@ -27,6 +27,20 @@ inline int bits_index(int bits) {
 }
 
 StepKernel step_kernel(int bits_m, int bits_v, bool cta_group);
+
+// Streamlined kernel (2/3/4-bit states, block 128 or 256); null outside that domain.  The
+// caller additionally requires fp32 parameters, nearest rounding of the first moment and
+// eps >= 1e-12.
+StepKernel fast_kernel_bm2(int bv_index, int block);
+StepKernel fast_kernel_bm3(int bv_index, int block);
+StepKernel fast_kernel_bm4(int bv_index, int block);
+StepKernel fast_kernel(int bits_m, int bits_v, int block);
+// Resident CTAs per SM of a step kernel (cached per kernel), 0 on error.
+int kernel_occupancy(StepKernel k);
+
+// Exhaustive comparison of the hardware lg2 approximation with log2_sp (tests).
+cudaError_t launch_fast_log_check(uint32_t lo, uint32_t hi, float* out_max_excess, cudaStream_t stream);
+float fast_log_abs_bound();
 // Resident CTAs per SM of that kernel (cached), 0 on error.
 int step_kernel_occupancy(int bits_m, int bits_v, bool cta_group);
 

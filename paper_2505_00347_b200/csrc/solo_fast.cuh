@@ -1,0 +1,560 @@
+// Streamlined fused step for the common configurations: 2/3/4-bit states, blocks of
+// 128 or 256 elements, fp32 parameters, nearest rounding of the first moment, eps >= 1e-12.
+//
+// Same packed state as the general kernel (solo_device.cuh): every quantity that decides
+// a stored code (EMA values, block scales, p-quantile, base, rounded logarithm) is computed
+// with the same IEEE operation sequence or is proven equal to it:
+//   * log_alpha(r) + xi is first evaluated with the hardware lg2 approximation; only when
+//     the result lies within a proven error bound of a rounding boundary is the exact
+//     polynomial log2_sp evaluated (rare), so the rounded code is always the one the exact
+//     sequence gives;
+//   * the k-th smallest v^ of a block is found by popping one minimum per round from
+//     per-thread sorted lists; if ties made a round pop several elements the exact
+//     tie-counting loop is used instead.
+// The parameter update uses an approximate square root and a reciprocal refined by one
+// Newton step (quotient error below 1.5 ulp); parameters therefore agree with the IEEE
+// sequence to a few 1e-7 of the update term, not bit for bit.
+//
+// Work split: a CTA of 256 threads owns a tile of 2048 consecutive elements, a thread
+// eight of them, a block of B elements G = B/8 consecutive lanes (half a warp or a warp).
+// The per-block scalar work (reciprocals of the scales, base of the logarithmic codebook
+// and its logarithm) is done once per block by the first warp for the whole tile and
+// passed through shared memory.
+//
+// Warp collectives are always issued with the full mask (one REDUX each).  For G = 16 the
+// two halves of a warp are reduced by one minimum and one maximum over a transformed
+// value: all quantities reduced here are non-negative binary32 bit patterns (bit 31
+// clear), so complementing the upper half's values moves them above every lower-half
+// value and reverses their order.
+#pragma once
+
+#include "solo_device.cuh"
+
+namespace solo {
+
+// Error model of lg2.approx.ftz.f32 against log2_sp, |diff| <= LG2_ABS + LG2_REL * |log2 x|
+// (checked exhaustively over all binary32 in [2^-100, 2) by solo_debug_check_fast_log with
+// half of these constants); LG2_REL also covers the two roundings of t.
+constexpr float LG2_ABS = 0x1p-20f;
+constexpr float LG2_REL = 0x1p-21f;
+
+constexpr uint32_t KEY_MAX = 0x7FFFFFFFu;    // sentinel key: above or equal to every valid key
+
+struct FastShared {
+    uint32_t sort[16][CTA];                  // rows 0..6: 2nd..8th smallest key of a thread; rows 7..15: sentinel
+    float tab[CTA / 16][32];                 // per group: K_v second-moment levels, then K_m first-moment levels
+    uint4 xin[2][CTA / 16];                  // per group: bits of Delta_m', Delta_v', x_p
+    float4 xout[2][CTA / 16];                // per group: 1/Delta_m', 1/Delta_v', 1/log2(alpha'), rounding limit
+    uint32_t xflag[2][CTA / 16];             // bit 0: vanishing first moment, bit 1: vanishing second moment
+};
+
+__device__ __forceinline__ float lg2_approx(float x) {
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float sqrt_approx(float x) {
+    float y;
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Philox4x32-10 with the round keys taken from the kernel arguments.
+__device__ __forceinline__ void philox_rk(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                          const uint32_t (&rk)[20], uint32_t (&out)[4]) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ rk[2 * r];
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ rk[2 * r + 1];
+        c1 = (uint32_t)p1;
+        c3 = (uint32_t)p0;
+        c0 = n0;
+        c2 = n2;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// ---------------------------------------------------------------------------
+// Group collectives on 31-bit values, full-mask instructions only.
+// `hi`: the lane belongs to the upper half of its warp (G = 16 only).
+// ---------------------------------------------------------------------------
+template <int G>
+__device__ __forceinline__ uint32_t seg_max31(uint32_t x, bool hi) {
+    if constexpr (G == 32) {
+        return __reduce_max_sync(0xffffffffu, x);
+    } else {
+        // lower half: complement of the low 31 bits (order reversed, bit 31 clear);
+        // upper half: bit 31 set.  min = lower half's maximum, max = upper half's maximum.
+        const uint32_t c = hi ? 0x80000000u : 0x7FFFFFFFu;
+        const uint32_t u = x ^ c;
+        const uint32_t lo = __reduce_min_sync(0xffffffffu, u);
+        const uint32_t up = __reduce_max_sync(0xffffffffu, u);
+        return (hi ? up : lo) ^ c;
+    }
+}
+template <int G>
+__device__ __forceinline__ int seg_sum16(int x, bool hi) {
+    if constexpr (G == 32) {
+        return __reduce_add_sync(0xffffffffu, x);
+    } else {
+        const int s = __reduce_add_sync(0xffffffffu, hi ? x << 16 : x);
+        return hi ? (int)((uint32_t)s >> 16) : s & 0xFFFF;
+    }
+}
+// Minimum of the group's keys in the "v domain": lower half keeps x, upper half holds ~x.
+// Returns the value a lane compares its own v with (equal <=> the lane holds the minimum).
+template <int G>
+__device__ __forceinline__ uint32_t seg_min_v(uint32_t v, bool hi) {
+    if constexpr (G == 32) {
+        return __reduce_min_sync(0xffffffffu, v);
+    } else {
+        const uint32_t lo = __reduce_min_sync(0xffffffffu, v);
+        const uint32_t up = __reduce_max_sync(0xffffffffu, v);
+        return hi ? up : lo;
+    }
+}
+
+// Codes of the thread's eight elements.  2 and 4 bit: one aligned 16/32-bit access.
+// 3 bit: the warp's 256 codes are 24 consecutive words; lanes 0..23 access one word
+// each and the 24-bit pieces travel by shuffle.
+template <int BITS>
+__device__ __forceinline__ uint32_t warp_load_codes(const uint8_t* warp_base, int lane) {
+    if constexpr (BITS == 2) {
+        return __ldcs(reinterpret_cast<const unsigned short*>(warp_base) + lane);
+    } else if constexpr (BITS == 4) {
+        return __ldcs(reinterpret_cast<const unsigned int*>(warp_base) + lane);
+    } else {
+        uint32_t w = 0;
+        if (lane < 24) w = __ldcs(reinterpret_cast<const unsigned int*>(warp_base) + lane);
+        const int a = (3 * lane) >> 2, o = ((3 * lane) & 3) * 8;
+        const uint32_t lo = __shfl_sync(0xffffffffu, w, a);
+        const uint32_t hi = __shfl_sync(0xffffffffu, w, (a + 1) & 31);
+        return __funnelshift_r(lo, hi, o) & 0xFFFFFFu;
+    }
+}
+template <int BITS>
+__device__ __forceinline__ void warp_store_codes(uint8_t* warp_base, int lane, uint32_t c) {
+    if constexpr (BITS == 2) {
+        __stcs(reinterpret_cast<unsigned short*>(warp_base) + lane, (unsigned short)c);
+    } else if constexpr (BITS == 4) {
+        __stcs(reinterpret_cast<unsigned int*>(warp_base) + lane, c);
+    } else {
+        const int a = (4 * lane) / 3, o = 32 * lane - 24 * a;        // o in {0, 8, 16} for lane < 24
+        const uint32_t lo = __shfl_sync(0xffffffffu, c, a & 31);
+        const uint32_t hi = __shfl_sync(0xffffffffu, c, (a + 1) & 31);
+        if (lane < 24)
+            __stcs(reinterpret_cast<unsigned int*>(warp_base) + lane, (lo >> (o & 31)) | (hi << ((24 - o) & 31)));
+    }
+}
+
+__device__ __forceinline__ void sort8(uint32_t (&key)[EPT]) {
+    cswap(key[0], key[1]); cswap(key[2], key[3]); cswap(key[4], key[5]); cswap(key[6], key[7]);
+    cswap(key[0], key[2]); cswap(key[1], key[3]); cswap(key[4], key[6]); cswap(key[5], key[7]);
+    cswap(key[1], key[2]); cswap(key[5], key[6]); cswap(key[0], key[4]); cswap(key[3], key[7]);
+    cswap(key[1], key[5]); cswap(key[2], key[6]);
+    cswap(key[1], key[4]); cswap(key[3], key[6]);
+    cswap(key[2], key[4]); cswap(key[3], key[5]);
+    cswap(key[3], key[4]);
+}
+
+// k-th smallest key of the group with ties counted, in the v domain.  k is uniform over the
+// group and may differ between the two halves of a warp; k <= 0 marks a group without a
+// block.  `col` is the thread's column of sorted keys (rows 0..6, sentinel in row 7).
+// Every round pops each group's current minimum (all its copies), so a group with k keys
+// or more terminates after at most k rounds; the loop ends when both halves are done.
+template <int G>
+__device__ __forceinline__ uint32_t select_counting(uint32_t head, const uint32_t* col, int k, bool hi) {
+    int ptr = 0, cnt = 0;
+    bool done = k <= 0;
+    uint32_t ans = 0;
+    while (true) {
+        const uint32_t tgt = seg_min_v<G>(head, hi);
+        const bool eq = head == tgt;
+        const uint32_t bal = __ballot_sync(0xffffffffu, eq);
+        cnt += __popc(G == 32 ? bal : (hi ? bal >> 16 : bal & 0xFFFFu));
+        if (!done && cnt >= k) {
+            ans = tgt;
+            done = true;
+        }
+        if (__all_sync(0xffffffffu, done)) break;
+        const uint32_t nxt = col[min(ptr, 7) * CTA];
+        head = eq ? nxt : head;
+        ptr += eq ? 1 : 0;
+    }
+    return ans;
+}
+
+// One round: pops the group's minimum from the thread that holds it and returns that minimum
+// (v domain).  `addr` is the shared-memory byte address of the thread's next row.
+// Unclamped form: `addr` advances by one row per pop, so it may be used for at most 16 rounds
+// (rows 7..15 of the column hold the sentinel).  Clamped form: any number of rounds; the
+// address stops at the first sentinel row.
+template <int G, bool CLAMP>
+__device__ __forceinline__ uint32_t pop_round(uint32_t& head, uint32_t& addr, uint32_t last, bool hi) {
+    const uint32_t tgt = seg_min_v<G>(head, hi);
+    if constexpr (CLAMP) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.eq.u32 p, %0, %2;\n\t@p ld.shared.u32 %0, [%1];\n\t"
+            "@p add.u32 %1, %1, %3;\n\t@p min.u32 %1, %1, %4;\n\t}"
+            : "+r"(head), "+r"(addr) : "r"(tgt), "n"(CTA * 4), "r"(last) : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.eq.u32 p, %0, %2;\n\t@p ld.shared.u32 %0, [%1];\n\t"
+            "@p add.u32 %1, %1, %3;\n\t}"
+            : "+r"(head), "+r"(addr) : "r"(tgt), "n"(CTA * 4) : "memory");
+    }
+    return tgt;
+}
+// k rounds.  Returns the last minimum and, in `popped`, the number of keys this thread popped
+// (at least 7 means "7 or more": beyond that only sentinels were read).
+template <int G>
+__device__ __forceinline__ uint32_t pop_rounds(uint32_t head, const uint32_t* col, int k, bool hi,
+                                               int& popped) {
+    const uint32_t addr0 = (uint32_t)__cvta_generic_to_shared(col);
+    const uint32_t last = addr0 + 7 * CTA * 4;
+    uint32_t addr = addr0, tgt = 0;
+    if (k == 13) {
+#pragma unroll
+        for (int r = 0; r < 13; ++r) tgt = pop_round<G, false>(head, addr, last, hi);
+    } else if (k <= 16) {
+#pragma unroll 1
+        for (int r = 0; r < k; ++r) tgt = pop_round<G, false>(head, addr, last, hi);
+    } else {
+#pragma unroll 2
+        for (int r = 0; r < k; ++r) tgt = pop_round<G, true>(head, addr, last, hi);
+    }
+    popped = (int)(addr - addr0) / (CTA * 4);
+    return tgt;
+}
+
+__device__ __forceinline__ void bar_sync(int id) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(CTA) : "memory");
+}
+
+// One tile.  FULL: all 2048 elements exist and both tensor pointers are 16-byte aligned.
+template <int BM, int BV, int G, bool FULL>
+__device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, const float* s_y,
+                                          const float* s_mid, char* pbase, const char* gbase,
+                                          const int64_t n, const int64_t tin, const int64_t jb_tile,
+                                          const int tensor, const int par) {
+    constexpr int KM = 1 << BM, KV = 1 << BV;
+    constexpr int NG = CTA / G, B = G * EPT;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int gl = tid & (G - 1), grp = tid / G;
+    const bool hi = G == 16 && (lane & 16) != 0;
+    const uint32_t vflip = hi ? 0xFFFFFFFFu : 0u;               // x domain <-> v domain
+
+    // validity (all true in a full tile)
+    const int64_t tile_elem0 = tin * TILE;
+    const int64_t rem_tile = n - tile_elem0;                    // elements of the tensor from the tile's first on, > 0
+    const bool have_block = FULL || (int64_t)grp * B < rem_tile;
+    const int nb = FULL ? B : (int)max((int64_t)0, min((int64_t)B, rem_tile - (int64_t)grp * B));
+    const int nv = FULL ? EPT : (int)max((int64_t)0, min((int64_t)EPT, rem_tile - (int64_t)tid * EPT));
+
+    char* const pt = pbase + tile_elem0 * 4;                    // the tile's parameters and gradients
+    const char* const gt = gbase + tile_elem0 * 2;
+    const int64_t tile_slot0 = jb_tile * G;                     // slot = 8 elements = one thread's codes
+    const int64_t jb = jb_tile + grp;
+
+    // ---- load ----
+    float p[EPT], g[EPT];
+    if (FULL) {
+        const uint4 gw = __ldcs(reinterpret_cast<const uint4*>(gt) + tid);
+        const float4 p0 = __ldcs(reinterpret_cast<const float4*>(pt) + 2 * tid);
+        const float4 p1 = __ldcs(reinterpret_cast<const float4*>(pt) + 2 * tid + 1);
+        const uint32_t gg[4] = {gw.x, gw.y, gw.z, gw.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            g[2 * i] = __uint_as_float(gg[i] << 16);
+            g[2 * i + 1] = __uint_as_float(gg[i] & 0xffff0000u);
+        }
+        p[0] = p0.x; p[1] = p0.y; p[2] = p0.z; p[3] = p0.w;
+        p[4] = p1.x; p[5] = p1.y; p[6] = p1.z; p[7] = p1.w;
+    } else {
+#pragma unroll
+        for (int i = 0; i < EPT; ++i) {
+            p[i] = 0.0f; g[i] = 0.0f;
+            if (i < nv) {
+                g[i] = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(gt)[tid * EPT + i] << 16);
+                p[i] = reinterpret_cast<const float*>(pt)[tid * EPT + i];
+            }
+        }
+    }
+    uint32_t cm = 0, cv = 0;
+    float dm = 0.0f, dv = 0.0f, al = 0.5f;
+    uint8_t* const wcm = a.codes_m + (tile_slot0 + warp * 32) * BM;   // the warp's 32 slots
+    uint8_t* const wcv = a.codes_v + (tile_slot0 + warp * 32) * BV;
+    if (FULL) {
+        cm = warp_load_codes<BM>(wcm, lane);
+        cv = warp_load_codes<BV>(wcv, lane);
+    } else if (have_block) {
+        cm = (uint32_t)load_codes<BM>(wcm + lane * BM);
+        cv = (uint32_t)load_codes<BV>(wcv + lane * BV);
+    }
+    if (have_block) {
+        dm = __ldg(a.scale_m + jb);
+        dv = __ldg(a.scale_v + jb);
+        al = __ldg(a.alpha + jb);
+    }
+
+    // ---- per-block level tables: alpha^k Delta_v and y_k Delta_m (Eq. 2) ----
+    float* const tab = s.tab[grp];
+    {
+        float a2[BV];
+        a2[0] = al;
+#pragma unroll
+        for (int i = 1; i < BV; ++i) a2[i] = a2[i - 1] * a2[i - 1];
+        if (gl < KV) tab[gl] = pow_sm<BV>(a2, (uint32_t)gl) * dv;
+        if (gl < KM) tab[KV + gl] = s_y[gl] * dm;
+    }
+    __syncwarp();
+
+    if (a.l2) {
+#pragma unroll
+        for (int i = 0; i < EPT; ++i) g[i] = __fmaf_rn(a.weight_decay, p[i], g[i]);
+    }
+
+    // ---- Eq. 2, Eq. 3, Adam(W) ----
+    float mh[EPT], vh[EPT];
+    uint32_t mx_m = 0, mx_v = 0;
+    const char* const tab_v = reinterpret_cast<const char*>(tab);
+    const char* const tab_m = reinterpret_cast<const char*>(tab + KV);
+    const uint32_t cm4 = cm << 2, cv4 = cv << 2;
+#pragma unroll
+    for (int i = 0; i < EPT; ++i) {
+        const uint32_t im = i * BM >= 2 ? (cm >> (i * BM - 2)) & ((KM - 1) << 2) : (cm4 >> (i * BM)) & ((KM - 1) << 2);
+        const uint32_t iv = i * BV >= 2 ? (cv >> (i * BV - 2)) & ((KV - 1) << 2) : (cv4 >> (i * BV)) & ((KV - 1) << 2);
+        const float mt = *reinterpret_cast<const float*>(tab_m + im);
+        const float vt = *reinterpret_cast<const float*>(tab_v + iv);
+        const float gi = g[i];
+        mh[i] = __fmaf_rn(a.beta1, mt, a.omb1 * gi);
+        vh[i] = __fmaf_rn(a.beta2, vt, a.omb2 * (gi * gi));
+        const float den = __fmaf_rn(sqrt_approx(vh[i]), a.inv_sqrt_bc2, a.eps);
+        const float rc = rcp_approx(den);
+        const float q0 = mh[i] * rc;
+        const float q1 = __fmaf_rn(__fmaf_rn(-den, q0, mh[i]), rc, q0);
+        p[i] = __fmaf_rn(-a.step_size, q1, p[i] * a.decay);
+        const bool valid = FULL || i < nv;
+        mx_m = max(mx_m, valid ? __float_as_uint(mh[i]) & 0x7fffffffu : 0u);
+        mx_v = max(mx_v, valid ? __float_as_uint(vh[i]) : 0u);
+    }
+
+    // ---- store parameters ----
+    if (FULL) {
+        __stcs(reinterpret_cast<float4*>(pt) + 2 * tid, make_float4(p[0], p[1], p[2], p[3]));
+        __stcs(reinterpret_cast<float4*>(pt) + 2 * tid + 1, make_float4(p[4], p[5], p[6], p[7]));
+    } else {
+#pragma unroll
+        for (int i = 0; i < EPT; ++i)
+            if (i < nv) reinterpret_cast<float*>(pt)[tid * EPT + i] = p[i];
+    }
+
+    // ---- block scales and the p-quantile of v^ (Sec. 3.2.2) ----
+    mx_m = seg_max31<G>(mx_m, hi);
+    mx_v = seg_max31<G>(mx_v, hi);
+    uint32_t x_p;
+    {
+        uint32_t key[EPT];
+#pragma unroll
+        for (int i = 0; i < EPT; ++i) key[i] = (FULL || i < nv) ? __float_as_uint(vh[i]) : KEY_MAX;
+        sort8(key);
+        uint32_t* const col = &s.sort[0][tid];
+#pragma unroll
+        for (int j = 1; j < EPT; ++j) col[(j - 1) * CTA] = key[j] ^ vflip;
+        const uint32_t head = key[0] ^ vflip;
+        uint32_t xv;
+        if (FULL) {
+            // one pop per round; exact when no round popped more than one key.  A thread that
+            // reached the sentinel row has popped 7 or 8 keys, which cannot be told apart: it
+            // sends its group to the counting loop as well.
+            const int k = a.k_full;
+            int popped;
+            xv = pop_rounds<G>(head, col, k, hi, popped);
+            const bool redo = seg_sum16<G>(popped >= 7 ? 256 : popped, hi) != k;
+            if (__any_sync(0xffffffffu, redo)) {
+                const uint32_t xc = select_counting<G>(head, col, redo ? k : 0, hi);
+                if (redo) xv = xc;
+            }
+        } else {
+            int k = (int)ceil((double)a.p_quantile * (double)nb);
+            k = min(max(k, 1), nb);                              // 0 for a group without a block
+            xv = select_counting<G>(head, col, k, hi);
+        }
+        x_p = xv ^ vflip;
+    }
+
+    // ---- per-block scalars, once per block, by the first warp; the others draw xi meanwhile ----
+    if (gl == 0) s.xin[par][grp] = make_uint4(mx_m, mx_v, x_p, 0u);
+    bar_sync(1);
+    uint32_t w[4] = {0u, 0u, 0u, 0u};
+    const uint64_t ctr = (uint64_t)tin * (TILE / EPT) + (uint32_t)tid;     // element index / 8
+    if (warp != 0) {
+        if (a.round_v) philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, (uint32_t)tensor * 4u, a.rk, w);
+    } else if (tid < NG) {
+        const uint4 in = s.xin[par][tid];
+        const float dm_new = __uint_as_float(in.x), dv_new = __uint_as_float(in.y);
+        const bool zero_m = dm_new < TINY, zero_v = dv_new < TINY;
+        const float inv_dm = 1.0f / dm_new;
+        const float inv_dv = 1.0f / dv_new;
+        const float rho = fminf(fmaxf(__uint_as_float(in.z) * inv_dv, RHO_MIN), RHO_MAX);
+        const float lam = log2_sp(rho) * (1.0f / (float)(KV - 1));
+        const float al_new = exp2_sp(lam);
+        const float inv_lambda = 1.0f / log2_sp(al_new);
+        const float guard = __fmaf_rn(fabsf(inv_lambda), LG2_ABS, LG2_REL * (float)(KV + 1));
+        s.xout[par][tid] = make_float4(inv_dm, inv_dv, inv_lambda, 0.5f - guard);
+        s.xflag[par][tid] = (zero_m ? 1u : 0u) | (zero_v ? 2u : 0u);
+        const bool blk_exists = FULL || (int64_t)tid * B < rem_tile;
+        if (blk_exists) {
+            const int64_t j = jb_tile + tid;
+            a.scale_m[j] = zero_m ? 0.0f : dm_new;
+            a.scale_v[j] = zero_v ? 0.0f : dv_new;
+            a.alpha[j] = zero_v ? 0.5f : al_new;
+        }
+    }
+    bar_sync(2);
+    if (warp == 0 && a.round_v)
+        philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, (uint32_t)tensor * 4u, a.rk, w);
+    float xi[EPT];
+    {
+#pragma unroll
+        for (int i = 0; i < EPT; ++i) {
+            // (d + 1/2) / 2^16 - 1/2 for the 16-bit draw d, via the binary32 1 + d 2^-16
+            const uint32_t h7 = (i & 1) ? (w[i >> 1] >> 9) & 0x007FFF80u : (w[i >> 1] << 7) & 0x007FFF80u;
+            xi[i] = a.round_v ? __uint_as_float(0x3F800000u | h7) + (-1.5f + 0x1p-17f) : 0.0f;
+        }
+    }
+    const float4 sc = s.xout[par][grp];
+    const uint32_t zf = s.xflag[par][grp];
+
+    // ---- first moment: nearest level (Eq. 1) ----
+    uint32_t om = 0;
+    {
+        const float inv = sc.x;
+        if constexpr (BM == 2) {
+            const float mid0 = s_mid[0], mid1 = s_mid[1], mid2 = s_mid[2];
+#pragma unroll
+            for (int i = EPT - 1; i >= 0; --i) {
+                const float r = mh[i] * inv;
+                const bool c1 = r > mid1;
+                const bool c0 = r > (c1 ? mid2 : mid0);
+                const uint32_t q = (c1 ? 2u : 0u) + (c0 ? 1u : 0u);
+                om = (om << BM) + ((FULL || i < nv) ? q : 0u);
+            }
+        } else {
+#pragma unroll
+            for (int i = EPT - 1; i >= 0; --i) {
+                const float r = mh[i] * inv;
+                uint32_t q = 0;
+#pragma unroll
+                for (int st = KM / 2; st >= 1; st >>= 1)
+                    if (r > s_mid[q + st - 1]) q += st;
+                om = (om << BM) + ((FULL || i < nv) ? q : 0u);
+            }
+        }
+    }
+
+    // ---- second moment: Eq. 6 ----
+    uint32_t ov = 0;
+    {
+        const float inv = sc.y, il = sc.z, lim = sc.w;
+        constexpr float MAGIC = 12582912.0f;                     // 1.5 * 2^23: adding it rounds to an integer
+        constexpr uint32_t MAGIC_BITS = 0x4B400000u;
+        float worst = 0.0f;
+        uint32_t acc = 0;
+#pragma unroll
+        for (int i = EPT - 1; i >= 0; --i) {
+            const float r = vh[i] * inv;
+            float t = __fmaf_rn(lg2_approx(r), il, xi[i]);
+            t = fminf(fmaxf(t, 0.0f), (float)(KV - 1));
+            const float u = t + MAGIC;
+            worst = fmaxf(worst, fabsf(t - (u - MAGIC)));
+            acc = (acc << BV) + ((FULL || i < nv) ? __float_as_uint(u) : MAGIC_BITS);
+        }
+        uint32_t magic_sum = 0;
+#pragma unroll
+        for (int i = 0; i < EPT; ++i) magic_sum = (magic_sum << BV) + MAGIC_BITS;
+        ov = acc - magic_sum;
+        if (__any_sync(0xffffffffu, worst > lim)) {
+            // some element of the warp is too close to a rounding boundary for the
+            // approximate logarithm: evaluate the exact sequence for all eight
+            ov = 0;
+#pragma unroll
+            for (int i = EPT - 1; i >= 0; --i) {
+                const float r = vh[i] * inv;
+                uint32_t q = KV - 1;
+                if (!(r < TINY)) {
+                    float t = __fmaf_rn(log2_sp(r), il, xi[i]);
+                    t = fminf(fmaxf(t, 0.0f), (float)(KV - 1));
+                    q = (uint32_t)__float2int_rn(t);
+                }
+                ov = (ov << BV) + ((FULL || i < nv) ? q : 0u);
+            }
+        }
+    }
+    if (zf & 1u) om = 0;
+    if (zf & 2u) ov = 0;
+
+    // ---- store the codes ----
+    if (FULL) {
+        warp_store_codes<BM>(wcm, lane, om);
+        warp_store_codes<BV>(wcv, lane, ov);
+    } else if (have_block) {
+        store_codes<BM>(wcm + lane * BM, om);
+        store_codes<BV>(wcv + lane * BV, ov);
+    }
+}
+
+template <int BM, int BV, int G>
+__global__ void __launch_bounds__(CTA, 3) solo_step_fast_kernel(const StepArgs a) {
+    constexpr int KM = 1 << BM;
+    __shared__ FastShared s;
+    __shared__ float s_y[KM];
+    __shared__ float s_mid[KM];
+    const int tid = threadIdx.x;
+    for (int i = tid; i < KM; i += CTA) {
+        s_y[i] = a.tables[i];
+        if (i < KM - 1) s_mid[i] = a.tables[KM + i];
+    }
+    for (int r = 7; r < 16; ++r) s.sort[r][tid] = (G == 16 && (tid & 16)) ? ~KEY_MAX : KEY_MAX;   // sentinels, v domain
+    __syncthreads();
+
+    int tensor = -1;
+    int64_t t_lo = 0, t_hi = 0, n = 0, jb0 = 0;
+    char* pbase = nullptr;
+    const char* gbase = nullptr;
+    bool aligned = false, skip = false;
+    int par = 0;
+    for (int64_t tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x) {
+        if (tile >= t_hi) {
+            do {
+                ++tensor;
+                t_hi = __ldg(a.tile_start + tensor + 1);
+            } while (tile >= t_hi);
+            t_lo = __ldg(a.tile_start + tensor);
+            n = __ldg(a.numel + tensor);
+            jb0 = __ldg(a.block_start + tensor);
+            pbase = (char*)(a.param_list ? a.param_list[tensor] : a.param_single);
+            gbase = (const char*)(a.grad_list ? a.grad_list[tensor] : a.grad_single);
+            aligned = ((((uintptr_t)pbase) | ((uintptr_t)gbase)) & 15u) == 0;
+            skip = a.numel_check != nullptr && __ldg(a.numel_check + tensor) != n;
+            if (skip && tid == 0) atomicOr(a.status, 1);
+        }
+        if (skip) continue;
+        const int64_t tin = tile - t_lo;
+        const int64_t jb_tile = jb0 + tin * (CTA / G);
+        if (aligned && (tin + 1) * TILE <= n)
+            fast_tile<BM, BV, G, true>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par);
+        else
+            fast_tile<BM, BV, G, false>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par);
+        par ^= 1;
+    }
+}
+
+}  // namespace solo

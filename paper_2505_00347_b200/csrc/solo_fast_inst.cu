@@ -1,0 +1,54 @@
+// Instantiations of the streamlined step kernel for one first-moment width (SOLO_BM = 2, 3, 4).
+#include "solo_dispatch.h"
+#include "solo_fast.cuh"
+
+#ifndef SOLO_BM
+#error "compile with -DSOLO_BM=2|3|4"
+#endif
+
+#define SOLO_CAT_(a, b) a##b
+#define SOLO_CAT(a, b) SOLO_CAT_(a, b)
+
+namespace solo {
+
+StepKernel SOLO_CAT(fast_kernel_bm, SOLO_BM)(int bv_index, int block) {
+    static const StepKernel table[3][2] = {
+        {solo_step_fast_kernel<SOLO_BM, 2, 16>, solo_step_fast_kernel<SOLO_BM, 2, 32>},
+        {solo_step_fast_kernel<SOLO_BM, 3, 16>, solo_step_fast_kernel<SOLO_BM, 3, 32>},
+        {solo_step_fast_kernel<SOLO_BM, 4, 16>, solo_step_fast_kernel<SOLO_BM, 4, 32>},
+    };
+    if (bv_index < 0 || bv_index > 2 || (block != 128 && block != 256)) return nullptr;
+    return table[bv_index][block == 256 ? 1 : 0];
+}
+
+#if SOLO_BM == 2
+// Exhaustive check of the error model used above: for every binary32 x with bit pattern
+// in [lo, hi] (positive, finite) the largest value of
+//   |lg2.approx(x) - log2_sp(x)| - (LG2_REL / 2) |log2_sp(x)|
+// is written (as a maximum over the launch) to *out_max_excess, which starts at -1.
+__global__ void fast_log_check_kernel(uint32_t lo, uint32_t hi, float* out_max_excess) {
+    float worst = -1.0f;
+    for (uint64_t b = (uint64_t)lo + blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; b <= hi;
+         b += (uint64_t)gridDim.x * blockDim.x) {
+        const float x = __uint_as_float((uint32_t)b);
+        const float exact = log2_sp(x);
+        const float ex = fabsf(lg2_approx(x) - exact) - (0.5f * LG2_REL) * fabsf(exact);
+        worst = fmaxf(worst, ex);
+    }
+    worst = fmaxf(worst, __shfl_xor_sync(0xffffffffu, worst, 16));
+    worst = fmaxf(worst, __shfl_xor_sync(0xffffffffu, worst, 8));
+    worst = fmaxf(worst, __shfl_xor_sync(0xffffffffu, worst, 4));
+    worst = fmaxf(worst, __shfl_xor_sync(0xffffffffu, worst, 2));
+    worst = fmaxf(worst, __shfl_xor_sync(0xffffffffu, worst, 1));
+    if ((threadIdx.x & 31) == 0 && worst > 0.0f)
+        atomicMax(reinterpret_cast<int*>(out_max_excess), __float_as_int(worst));
+}
+
+cudaError_t launch_fast_log_check(uint32_t lo, uint32_t hi, float* out_max_excess, cudaStream_t stream) {
+    fast_log_check_kernel<<<148 * 8, 256, 0, stream>>>(lo, hi, out_max_excess);
+    return cudaGetLastError();
+}
+float fast_log_abs_bound() { return LG2_ABS; }
+#endif
+
+}  // namespace solo
