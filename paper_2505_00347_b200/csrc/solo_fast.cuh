@@ -8,9 +8,8 @@
 //     the result lies within a proven error bound of a rounding boundary is the exact
 //     polynomial log2_sp evaluated (rare), so the rounded code is always the one the exact
 //     sequence gives;
-//   * the k-th smallest v^ of a block is found by popping one minimum per round from
-//     per-thread sorted lists; if ties made a round pop several elements the exact
-//     tie-counting loop is used instead.
+//   * the k-th smallest v^ of a block is found exactly, duplicates included, by popping one
+//     minimum per round from per-thread sorted lists.
 // The parameter update uses an approximate square root and a reciprocal refined by one
 // Newton step (quotient error below 1.5 ulp); parameters therefore agree with the IEEE
 // sequence to a few 1e-7 of the update term, not bit for bit.
@@ -164,74 +163,67 @@ __device__ __forceinline__ void sort8(uint32_t (&key)[EPT]) {
     cswap(key[3], key[4]);
 }
 
-// k-th smallest key of the group with ties counted, in the v domain.  k is uniform over the
-// group and may differ between the two halves of a warp; k <= 0 marks a group without a
-// block.  `col` is the thread's column of sorted keys (rows 0..6, sentinel in row 7).
-// Every round pops each group's current minimum (all its copies), so a group with k keys
-// or more terminates after at most k rounds; the loop ends when both halves are done.
-template <int G>
-__device__ __forceinline__ uint32_t select_counting(uint32_t head, const uint32_t* col, int k, bool hi) {
-    int ptr = 0, cnt = 0;
-    bool done = k <= 0;
-    uint32_t ans = 0;
-    while (true) {
-        const uint32_t tgt = seg_min_v<G>(head, hi);
-        const bool eq = head == tgt;
-        const uint32_t bal = __ballot_sync(0xffffffffu, eq);
-        cnt += __popc(G == 32 ? bal : (hi ? bal >> 16 : bal & 0xFFFFu));
-        if (!done && cnt >= k) {
-            ans = tgt;
-            done = true;
-        }
-        if (__all_sync(0xffffffffu, done)) break;
-        const uint32_t nxt = col[min(ptr, 7) * CTA];
-        head = eq ? nxt : head;
-        ptr += eq ? 1 : 0;
-    }
-    return ans;
-}
-
-// One round: pops the group's minimum from the thread that holds it and returns that minimum
-// (v domain).  `addr` is the shared-memory byte address of the thread's next row.
-// Unclamped form: `addr` advances by one row per pop, so it may be used for at most 16 rounds
-// (rows 7..15 of the column hold the sentinel).  Clamped form: any number of rounds; the
-// address stops at the first sentinel row.
+// One selection round: finds the group's smallest unpopped key and pops it from exactly one
+// thread (the lowest lane among those whose head equals it), so that after r rounds the r
+// smallest keys, duplicates included, have been popped.  Returns that key (v domain).
+// `addr` is the shared-memory byte address of the thread's next row, `lt` the mask of the
+// lanes of the thread's group below it.  Unclamped form: `addr` advances one row per pop and
+// may be used for at most 16 rounds (rows 7..15 of a column hold the sentinel).  Clamped form:
+// any number of rounds; the address stops at the first sentinel row.
 template <int G, bool CLAMP>
-__device__ __forceinline__ uint32_t pop_round(uint32_t& head, uint32_t& addr, uint32_t last, bool hi) {
+__device__ __forceinline__ uint32_t pop_round(uint32_t& head, uint32_t& addr, uint32_t last, uint32_t lt,
+                                              bool hi) {
     const uint32_t tgt = seg_min_v<G>(head, hi);
+    const bool eq = head == tgt;
+    const uint32_t lower = __ballot_sync(0xffffffffu, eq) & lt;
     if constexpr (CLAMP) {
         asm volatile(
-            "{\n\t.reg .pred p;\n\tsetp.eq.u32 p, %0, %2;\n\t@p ld.shared.u32 %0, [%1];\n\t"
-            "@p add.u32 %1, %1, %3;\n\t@p min.u32 %1, %1, %4;\n\t}"
-            : "+r"(head), "+r"(addr) : "r"(tgt), "n"(CTA * 4), "r"(last) : "memory");
+            "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %3, 0;\n\tsetp.eq.and.u32 p, %2, 0, q;\n\t"
+            "@p ld.shared.u32 %0, [%1];\n\t"
+            "@p add.u32 %1, %1, %4;\n\t@p min.u32 %1, %1, %5;\n\t}"
+            : "+r"(head), "+r"(addr) : "r"(lower), "r"((int)eq), "n"(CTA * 4), "r"(last) : "memory");
     } else {
         asm volatile(
-            "{\n\t.reg .pred p;\n\tsetp.eq.u32 p, %0, %2;\n\t@p ld.shared.u32 %0, [%1];\n\t"
-            "@p add.u32 %1, %1, %3;\n\t}"
-            : "+r"(head), "+r"(addr) : "r"(tgt), "n"(CTA * 4) : "memory");
+            "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %3, 0;\n\tsetp.eq.and.u32 p, %2, 0, q;\n\t"
+            "@p ld.shared.u32 %0, [%1];\n\t"
+            "@p add.u32 %1, %1, %4;\n\t}"
+            : "+r"(head), "+r"(addr) : "r"(lower), "r"((int)eq), "n"(CTA * 4) : "memory");
     }
     return tgt;
 }
-// k rounds.  Returns the last minimum and, in `popped`, the number of keys this thread popped
-// (at least 7 means "7 or more": beyond that only sentinels were read).
-template <int G>
-__device__ __forceinline__ uint32_t pop_rounds(uint32_t head, const uint32_t* col, int k, bool hi,
-                                               int& popped) {
+
+// k-th smallest key of the group (duplicates counted), v domain.  k is uniform over the group
+// and may differ between the two halves of a warp (k <= 0: a group without a block, result
+// unused).  `col` is the thread's column of sorted keys (rows 0..6, sentinels from row 7 on),
+// `head` its smallest key.  UNIFORM_K: every group of the warp has the same k.
+template <int G, bool UNIFORM_K>
+__device__ __forceinline__ uint32_t select_kth(uint32_t head, const uint32_t* col, int k, bool hi) {
+    const int lane = threadIdx.x & 31;
+    const uint32_t below = (1u << lane) - 1u;
+    const uint32_t lt = (G == 16 && hi) ? below & 0xFFFF0000u : below;
     const uint32_t addr0 = (uint32_t)__cvta_generic_to_shared(col);
     const uint32_t last = addr0 + 7 * CTA * 4;
-    uint32_t addr = addr0, tgt = 0;
-    if (k == 13) {
+    uint32_t addr = addr0, ans = 0;
+    if (UNIFORM_K && k == 13) {
 #pragma unroll
-        for (int r = 0; r < 13; ++r) tgt = pop_round<G, false>(head, addr, last, hi);
-    } else if (k <= 16) {
-#pragma unroll 1
-        for (int r = 0; r < k; ++r) tgt = pop_round<G, false>(head, addr, last, hi);
+        for (int r = 0; r < 13; ++r) ans = pop_round<G, false>(head, addr, last, lt, hi);
     } else {
-#pragma unroll 2
-        for (int r = 0; r < k; ++r) tgt = pop_round<G, true>(head, addr, last, hi);
+        const int rounds = UNIFORM_K ? k : __reduce_max_sync(0xffffffffu, k);
+        if (rounds <= 16) {
+#pragma unroll 1
+            for (int r = 1; r <= rounds; ++r) {
+                const uint32_t t = pop_round<G, false>(head, addr, last, lt, hi);
+                if (r == k) ans = t;
+            }
+        } else {
+#pragma unroll 1
+            for (int r = 1; r <= rounds; ++r) {
+                const uint32_t t = pop_round<G, true>(head, addr, last, lt, hi);
+                if (r == k) ans = t;
+            }
+        }
     }
-    popped = (int)(addr - addr0) / (CTA * 4);
-    return tgt;
+    return ans;
 }
 
 __device__ __forceinline__ void bar_sync(int id) {
@@ -371,21 +363,11 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
         const uint32_t head = key[0] ^ vflip;
         uint32_t xv;
         if (FULL) {
-            // one pop per round; exact when no round popped more than one key.  A thread that
-            // reached the sentinel row has popped 7 or 8 keys, which cannot be told apart: it
-            // sends its group to the counting loop as well.
-            const int k = a.k_full;
-            int popped;
-            xv = pop_rounds<G>(head, col, k, hi, popped);
-            const bool redo = seg_sum16<G>(popped >= 7 ? 256 : popped, hi) != k;
-            if (__any_sync(0xffffffffu, redo)) {
-                const uint32_t xc = select_counting<G>(head, col, redo ? k : 0, hi);
-                if (redo) xv = xc;
-            }
+            xv = select_kth<G, true>(head, col, a.k_full, hi);
         } else {
             int k = (int)ceil((double)a.p_quantile * (double)nb);
             k = min(max(k, 1), nb);                              // 0 for a group without a block
-            xv = select_counting<G>(head, col, k, hi);
+            xv = select_kth<G, false>(head, col, k, hi);
         }
         x_p = xv ^ vflip;
     }
