@@ -48,7 +48,8 @@ typedef enum {
     SOLO_EALIGN = -2,   /* a parameter / gradient pointer is not 16-byte aligned */
     SOLO_ENOMEM = -3,   /* device or host allocation failed */
     SOLO_ECUDA = -4,    /* a CUDA runtime call or the kernel launch failed */
-    SOLO_ESTATE = -5    /* the state does not match the call (sizes, tensor count) */
+    SOLO_ESTATE = -5,   /* the state does not match the call (sizes, tensor count) */
+    SOLO_ELIMIT = -6    /* more tensors than solo_multi_step_static has room for */
 } solo_status_t;
 
 /* Constants of the quantizers that the paper leaves open. */
@@ -193,6 +194,57 @@ int solo_set_kernel_policy(int policy);
  */
 int solo_debug_check_fast_log(uint32_t lo_bits, uint32_t hi_bits, float* max_excess_host,
                               float* abs_bound_host);
+
+/*
+ * Optimizer state in buffers that the CALLER allocated (device memory), for
+ * solo_multi_step_static.  Same layout as the library's own state (see the top of this
+ * file): with n_blk = sum over tensors of ceil(numel / block),
+ *   codes_m  n_blk * block * bits_m / 8 bytes     codes_v  n_blk * block * bits_v / 8 bytes
+ *   scale_m, scale_v, alpha  n_blk floats each
+ * every buffer 16-byte aligned.  A fresh state is all-zero codes and scales and alpha = 0.5.
+ */
+typedef struct {
+    void* codes_m;
+    void* codes_v;
+    float* scale_m;
+    float* scale_v;
+    float* alpha;
+    int32_t bits_m, bits_v, block;
+} solo_raw_state_t;
+
+#define SOLO_STATIC_MAX_TENSORS 1024
+
+/*
+ * solo_multi_step for callers that must not allocate device memory.  (The paper has no
+ * counterpart; this is a convenience of the library.)
+ *
+ * Some hosts of this step cannot call cudaMalloc at the moment they need it: code running
+ * under a framework's caching allocator that wants every byte accounted for, a process whose
+ * whole GPU memory was handed to a pool up front, or a step issued from a place (a stream
+ * callback's consumer, a tight real-time loop) where the implicit device synchronisation of
+ * cudaMalloc / cudaFree is not acceptable.  solo_state_create allocates; this entry point
+ * never does.  The caller brings the state buffers (solo_raw_state_t); the small tables the
+ * kernel needs besides them -- the tile and block offsets of every tensor, the first-moment
+ * codebook and a status word, 32 KiB in all -- live in one fixed array inside the library
+ * that every GPU loading the library holds until the process exits.
+ *
+ *   num_tensors        1 .. SOLO_STATIC_MAX_TENSORS; more is refused with SOLO_ELIMIT
+ *   param_dev, grad_dev  DEVICE arrays of num_tensors device pointers (as in solo_tensor_list_t)
+ *   numel_host         HOST array of the tensors' element counts, each > 0
+ *   st                 the caller's state buffers and their geometry
+ * Parameters fp32 or bf16, gradients bf16, hyper-parameters and `step` as for solo_multi_step;
+ * the result is the same as solo_multi_step's on a library-owned state with equal contents.
+ *
+ * The fixed array is shared by every call on a device and is rewritten by each call, in
+ * stream order: calls whose GPU work can overlap (different streams without ordering between
+ * them) race on it and must be serialised by the caller.  Its address is looked up on the
+ * first call on each device; make that first call outside any stream capture.  No
+ * cudaMalloc, cudaFree or other allocating routine is called.  Asynchronous on `stream`
+ * except for the copy of the offsets from host memory, which is staged before the call returns.
+ */
+int solo_multi_step_static(int32_t num_tensors, void* const* param_dev, const void* const* grad_dev,
+                           const int64_t* numel_host, const solo_raw_state_t* st,
+                           const solo_hyper_t* hyper, int64_t step, void* stream);
 
 /* Number of kernel launches issued by this library in the calling process so far. */
 int64_t solo_launch_count(void);

@@ -15,6 +15,8 @@ _PKG = Path(__file__).resolve().parent
 LIB_PATH = _PKG / "libsolo_b200.so"
 
 SOLO_OK, SOLO_EINVAL, SOLO_EALIGN, SOLO_ENOMEM, SOLO_ECUDA, SOLO_ESTATE = 0, -1, -2, -3, -4, -5
+SOLO_ELIMIT = -6
+STATIC_MAX_TENSORS = 1024
 
 
 class SoloError(RuntimeError):
@@ -40,6 +42,16 @@ class TensorList(C.Structure):
     _fields_ = [
         ("num_tensors", C.c_int32), ("param", C.c_void_p), ("grad", C.c_void_p),
         ("numel", C.c_void_p), ("state", C.c_void_p),
+    ]
+
+
+class RawState(C.Structure):
+    """solo_raw_state_t: caller-owned state buffers for solo_multi_step_static"""
+
+    _fields_ = [
+        ("codes_m", C.c_void_p), ("codes_v", C.c_void_p), ("scale_m", C.c_void_p),
+        ("scale_v", C.c_void_p), ("alpha", C.c_void_p),
+        ("bits_m", C.c_int32), ("bits_v", C.c_int32), ("block", C.c_int32),
     ]
 
 
@@ -81,6 +93,9 @@ def lib() -> C.CDLL:
     L.solo_set_kernel_policy.argtypes = [i32]
     L.solo_debug_check_fast_log.argtypes = [C.c_uint32, C.c_uint32, C.POINTER(C.c_float),
                                             C.POINTER(C.c_float)]
+    L.solo_multi_step_static.argtypes = [C.c_int32, vp, vp, C.POINTER(C.c_int64), C.POINTER(RawState),
+                                         C.POINTER(Hyper), i64, vp]
+    L.solo_multi_step_static.restype = C.c_int
     L.solo_launch_count.argtypes = []
     L.solo_launch_count.restype = C.c_int64
     L.solo_strerror.argtypes = [i32]
@@ -259,6 +274,26 @@ def solo_dequant(state: State, which: int) -> torch.Tensor:
     out = torch.empty(sum(state.sizes), dtype=torch.float32, device=state.device)
     _check(lib().solo_dequant(state.handle, which, out.data_ptr(), _stream()), "solo_dequant")
     return out
+
+
+def solo_multi_step_static(params: list[torch.Tensor], grads: list[torch.Tensor], sizes: list[int],
+                           buffers: dict, bits_m: int, bits_v: int, block: int, h: Hyper, step: int,
+                           param_ptrs: torch.Tensor = None, grad_ptrs: torch.Tensor = None) -> None:
+    """The allocation-free step: `buffers` maps codes_m / codes_v (uint8) and scale_m / scale_v /
+    alpha (float32) to CUDA tensors that the caller allocated in the library's state layout.
+    `param_ptrs` / `grad_ptrs` are int64 CUDA tensors of the tensors' data pointers (built here,
+    with torch, when not given; the library call itself allocates nothing)."""
+    if param_ptrs is None:
+        param_ptrs = torch.tensor([p.data_ptr() for p in params], dtype=torch.int64, device=params[0].device)
+    if grad_ptrs is None:
+        grad_ptrs = torch.tensor([g.data_ptr() for g in grads], dtype=torch.int64, device=params[0].device)
+    raw = RawState(buffers["codes_m"].data_ptr(), buffers["codes_v"].data_ptr(),
+                   buffers["scale_m"].data_ptr(), buffers["scale_v"].data_ptr(),
+                   buffers["alpha"].data_ptr(), bits_m, bits_v, block)
+    numel = (C.c_int64 * len(sizes))(*[int(n) for n in sizes])
+    _check(lib().solo_multi_step_static(len(sizes), param_ptrs.data_ptr(), grad_ptrs.data_ptr(), numel,
+                                        C.byref(raw), C.byref(h), step, _stream()),
+           "solo_multi_step_static")
 
 
 def codebook_m(bits: int) -> torch.Tensor:

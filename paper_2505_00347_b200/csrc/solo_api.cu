@@ -180,6 +180,39 @@ bool on_state_device(const solo_state* s) {
     return cudaGetDevice(&dev) == cudaSuccess && dev == s->device;
 }
 
+// ---------------------------------------------------------------------------
+// Fixed scratch of the allocation-free entry point: per device, held until exit.
+//   int64 numel[MAX] | block_start[MAX+1] | tile_start[MAX+1]   then
+//   float tables[3*256-2] (y | mid | 1/gap of the first-moment codebook)   then   int status
+// ---------------------------------------------------------------------------
+constexpr int STATIC_MAX_T = SOLO_STATIC_MAX_TENSORS;
+constexpr size_t STATIC_GEOM_BYTES = (size_t)(3 * STATIC_MAX_T + 2) * sizeof(int64_t);
+constexpr size_t STATIC_TABLE_BYTES = (size_t)(3 * 256 - 2) * sizeof(float);
+constexpr size_t STATIC_STATUS_OFF = (STATIC_GEOM_BYTES + STATIC_TABLE_BYTES + 15) / 16 * 16;
+constexpr size_t STATIC_BYTES = STATIC_STATUS_OFF + 16;
+static_assert(STATIC_BYTES <= 32 * 1024, "documented size of the fixed scratch");
+
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_BYTES];
+
+// Device address of g_static_scratch on the current device (the symbol's name is only a
+// host-side handle).  Looked up once per device, with that device current.
+int static_scratch(int device, unsigned char** out) {
+    static std::mutex mu;
+    static unsigned char* ptr[64];
+    if (device < 0 || device >= 64) return SOLO_EINVAL;
+    std::lock_guard<std::mutex> lk(mu);
+    if (!ptr[device]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return SOLO_ECUDA;
+        }
+        ptr[device] = (unsigned char*)p;
+    }
+    *out = ptr[device];
+    return SOLO_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -315,6 +348,84 @@ int solo_multi_step(const solo_tensor_list_t* list, const solo_hyper_t* hyper, i
     return launch_step(s, a, (cudaStream_t)stream);
 }
 
+int solo_multi_step_static(int32_t num_tensors, void* const* param_dev, const void* const* grad_dev,
+                           const int64_t* numel_host, const solo_raw_state_t* st,
+                           const solo_hyper_t* hyper, int64_t step, void* stream_) {
+    if (!param_dev || !grad_dev || !numel_host || !st || num_tensors < 1) return SOLO_EINVAL;
+    if (num_tensors > STATIC_MAX_T) return SOLO_ELIMIT;
+    if (!valid_bits(st->bits_m) || !valid_bits(st->bits_v) || !valid_block(st->block)) return SOLO_EINVAL;
+    if (!st->codes_m || !st->codes_v || !st->scale_m || !st->scale_v || !st->alpha) return SOLO_EINVAL;
+    if ((((uintptr_t)st->codes_m) | ((uintptr_t)st->codes_v) | ((uintptr_t)st->scale_m) |
+         ((uintptr_t)st->scale_v) | ((uintptr_t)st->alpha)) & 15u)
+        return SOLO_EALIGN;
+    int rc = check_hyper(hyper, step);
+    if (rc) return rc;
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) { cudaGetLastError(); return SOLO_ECUDA; }
+    unsigned char* scratch = nullptr;
+    rc = static_scratch(device, &scratch);
+    if (rc) return rc;
+    cudaStream_t stream = (cudaStream_t)stream_;
+
+    // geometry and codebook tables, built in fixed-size host arrays (no heap, no device allocation)
+    const int T = num_tensors, block = st->block;
+    int64_t geom[3 * STATIC_MAX_T + 2];
+    int64_t* numel = geom;
+    int64_t* block_start = geom + T;
+    int64_t* tile_start = geom + T + (T + 1);
+    block_start[0] = 0;
+    tile_start[0] = 0;
+    for (int t = 0; t < T; ++t) {
+        if (numel_host[t] < 1) return SOLO_EINVAL;
+        numel[t] = numel_host[t];
+        block_start[t + 1] = block_start[t] + (numel_host[t] + block - 1) / block;
+        tile_start[t + 1] = tile_start[t] + (numel_host[t] + solo::TILE - 1) / solo::TILE;
+    }
+    float tables[3 * 256 - 2];
+    {
+        std::vector<float> tm;                       // host memory only
+        codebook_tables(st->bits_m, tm);
+        std::memcpy(tables, tm.data(), tm.size() * sizeof(float));
+    }
+    const size_t geom_bytes = (size_t)(3 * T + 2) * sizeof(int64_t);
+    const size_t table_bytes = (size_t)(3 * (1 << st->bits_m) - 2) * sizeof(float);
+    int64_t* d_geom = (int64_t*)scratch;
+    float* d_tables = (float*)(scratch + STATIC_GEOM_BYTES);
+    int* d_status = (int*)(scratch + STATIC_STATUS_OFF);
+    // pageable sources: both copies are staged before cudaMemcpyAsync returns
+    if (cudaMemcpyAsync(d_geom, geom, geom_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(d_tables, tables, table_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaMemsetAsync(d_status, 0, 16, stream) != cudaSuccess) {
+        cudaGetLastError();
+        return SOLO_ECUDA;
+    }
+
+    solo_state tmp;                                   // host-side description only; owns nothing
+    tmp.device = device;
+    tmp.bits_m = st->bits_m; tmp.bits_v = st->bits_v; tmp.block = block; tmp.num_tensors = T;
+    tmp.tiles_total = tile_start[T];
+    tmp.nblk_total = block_start[T];
+    StepArgs a;
+    std::memset(&a, 0, sizeof(a));
+    a.numel = d_geom;
+    a.block_start = d_geom + T;
+    a.tile_start = d_geom + T + (T + 1);
+    a.num_tensors = T;
+    a.total_tiles = tmp.tiles_total;
+    a.codes_m = (uint8_t*)st->codes_m;
+    a.codes_v = (uint8_t*)st->codes_v;
+    a.scale_m = st->scale_m;
+    a.scale_v = st->scale_v;
+    a.alpha = st->alpha;
+    a.tables = d_tables;
+    a.status = d_status;
+    reduce_hyper(hyper, step, block, a);
+    a.param_list = param_dev;
+    a.grad_list = grad_dev;
+    a.numel_check = nullptr;
+    return launch_step(&tmp, a, stream);
+}
+
 int solo_dequant(const solo_state_t* s, int which, float* out_dev, void* stream) {
     if (!s || !out_dev || (which != 0 && which != 1)) return SOLO_EINVAL;
     if (!on_state_device(s)) return SOLO_ESTATE;
@@ -441,6 +552,7 @@ const char* solo_strerror(int status) {
         case SOLO_ENOMEM: return "out of memory";
         case SOLO_ECUDA: return "CUDA call or kernel launch failed";
         case SOLO_ESTATE: return "state does not match the call";
+        case SOLO_ELIMIT: return "too many tensors for solo_multi_step_static (limit SOLO_STATIC_MAX_TENSORS)";
         default: return "unknown status";
     }
 }

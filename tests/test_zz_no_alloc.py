@@ -1,0 +1,81 @@
+"""The allocation-free entry point solo_multi_step_static against solo_multi_step.
+
+Callers that run under a memory pool which owns all of the GPU's memory, or that must not
+trigger the device-wide synchronisation of cudaMalloc / cudaFree in the middle of a training
+step, bring their own state buffers; the library keeps the few tables it needs besides them in a
+fixed array of its own.  Both entry points launch the same kernels, so on equal inputs the packed
+state and the parameters must come out identical; this is checked on two consecutive calls (the
+fixed array is rewritten by every call, the second one with a different tensor list).
+
+Collected last on purpose: a failure here leaves every other test already run.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2505_00347_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _fresh_buffers(sizes, bits_m, bits_v, block, state0=None):
+    nb = sum(-(-int(n) // block) for n in sizes)
+    if state0 is not None:
+        return {k: v.clone().cuda() for k, v in state0.items()}
+    return {
+        "codes_m": torch.zeros(nb * block * bits_m // 8, dtype=torch.uint8, device="cuda"),
+        "codes_v": torch.zeros(nb * block * bits_v // 8, dtype=torch.uint8, device="cuda"),
+        "scale_m": torch.zeros(nb, dtype=torch.float32, device="cuda"),
+        "scale_v": torch.zeros(nb, dtype=torch.float32, device="cuda"),
+        "alpha": torch.full((nb,), 0.5, dtype=torch.float32, device="cuda"),
+    }
+
+
+def _run_pair(B, sizes, bits_m, bits_v, block, steps, seed, state0=None):
+    w = synth.workload(2, sizes=tuple(sizes))
+    h = B.hyper(lr=1e-3, beta1=0.6, beta2=0.999, weight_decay=0.01, seed=seed)
+    params = [synth.make_param(w, i) for i in range(len(sizes))]
+    p_lib = [p.clone().cuda() for p in params]
+    p_sta = [p.clone().cuda() for p in params]
+    lib_state = B.State(list(sizes), bits_m, bits_v, block)
+    bufs = _fresh_buffers(sizes, bits_m, bits_v, block, state0)
+    if state0 is not None:
+        for k, v in state0.items():
+            lib_state.raw_set(k, v)
+    for t in range(1, steps + 1):
+        grads = [synth.make_grad(w, i, t).cuda() for i in range(len(sizes))]
+        B.solo_multi_step(B.TensorSet(p_lib, grads, lib_state), h, t)
+        B.solo_multi_step_static(p_sta, grads, list(sizes), bufs, bits_m, bits_v, block, h, t)
+        torch.cuda.synchronize()
+        for key in ("codes_m", "codes_v", "scale_m", "scale_v", "alpha"):
+            got = bufs[key].cpu().numpy().view(np.uint8)
+            want = lib_state.raw_get(key).numpy().view(np.uint8)
+            assert np.array_equal(got, want), (key, t)
+        for a, b in zip(p_sta, p_lib):
+            assert torch.equal(a, b), t          # same kernel, same inputs: bit-identical parameters
+    lib_state.destroy()
+
+
+def test_static_entry_point_matches_library_state_twice():
+    from paper_2505_00347_b200 import binding as B
+    # first call sequence: streamlined kernel (2/3 bit, block 128), ragged multi-tensor list
+    _run_pair(B, (2048 * 3 + 77, 1, 128, 5000), 2, 3, 128, steps=2, seed=7)
+    # second, with another list and widths (general kernel: 8-bit, block 2048), from a random state
+    sizes = (2048 * 2 + 5, 300, 4097)
+    st0 = synth.make_state(sizes, 8, 4, 2048, seed=99)
+    _run_pair(B, sizes, 8, 4, 2048, steps=2, seed=8, state0=st0)
+
+
+def test_static_entry_point_rejects_what_it_cannot_hold():
+    from paper_2505_00347_b200 import binding as B
+    n = B.STATIC_MAX_TENSORS + 1
+    sizes = [8] * n
+    ps = [torch.zeros(8, device="cuda") for _ in range(2)]
+    gs = [torch.zeros(8, device="cuda", dtype=torch.bfloat16) for _ in range(2)]
+    bufs = _fresh_buffers(sizes, 4, 4, 128)
+    ptrs = torch.zeros(n, dtype=torch.int64, device="cuda")
+    with pytest.raises(B.SoloError) as e:
+        B.solo_multi_step_static(ps, gs, sizes, bufs, 4, 4, 128, B.hyper(), 1, param_ptrs=ptrs, grad_ptrs=ptrs)
+    assert e.value.status == B.SOLO_ELIMIT and "SOLO_STATIC_MAX_TENSORS" in str(e.value)
+    with pytest.raises(B.SoloError):
+        B.solo_multi_step_static(ps, gs, [8, 0], bufs, 4, 4, 128, B.hyper(), 1)
