@@ -33,9 +33,10 @@ namespace solo {
 
 // Error model of lg2.approx.ftz.f32 against log2_sp, |diff| <= LG2_ABS + LG2_REL * |log2 x|
 // (checked exhaustively over all binary32 in [2^-100, 2) by solo_debug_check_fast_log with
-// half of these constants); LG2_REL also covers the two roundings of t.
+// half of these constants); the other half of LG2_REL covers the roundings of t, which the
+// kernel evaluates scaled to [0, 1] (a few 2^-24 relative each).
 constexpr float LG2_ABS = 0x1p-20f;
-constexpr float LG2_REL = 0x1p-21f;
+constexpr float LG2_REL = 0x1p-20f;
 
 constexpr uint32_t KEY_MAX = 0x7FFFFFFFu;    // sentinel key: above or equal to every valid key
 
@@ -45,6 +46,14 @@ struct FastShared {
     uint4 xin[2][CTA / 16];                  // per group: bits of Delta_m', Delta_v', x_p
     float4 xout[2][CTA / 16];                // per group: 1/Delta_m', 1/Delta_v', 1/log2(alpha'), rounding limit
     uint32_t xflag[2][CTA / 16];             // bit 0: vanishing first moment, bit 1: vanishing second moment
+    // Inputs of a full tile, copied asynchronously (cp.async) one tile ahead of their use.  Every
+    // thread copies the parameters and gradients it reads itself; codes and scales are shared by
+    // a warp.
+    float4 st_p0[CTA], st_p1[CTA];           // a thread's eight parameters
+    uint4 st_g[CTA];                         // its eight bf16 gradients
+    uint32_t st_cm[CTA / 32][32];            // a warp's packed codes (8 * bits words)
+    uint32_t st_cv[CTA / 32][32];
+    float st_sc[CTA / 16][4];                // a group's Delta_m, Delta_v, alpha
 };
 
 __device__ __forceinline__ float lg2_approx(float x) {
@@ -62,6 +71,32 @@ __device__ __forceinline__ float rcp_approx(float x) {
     asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+
+// The two 16-bit halves of a word as binary32 (one conversion each, no shift or mask).
+__device__ __forceinline__ void halves_to_float(uint32_t w, float& lo, float& hi) {
+    asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\tcvt.rn.f32.u16 %0, l;\n\tcvt.rn.f32.u16 %1, h;\n\t}"
+        : "=f"(lo), "=f"(hi) : "r"(w));
+}
+
+// Byte offsets (4 * code) of the eight W-bit codes packed in `c`, for a table of floats.  The
+// codes at even and at odd positions are kept in two words with the other positions zeroed, so
+// that a left shift that brings a code to the top of the word followed by a right shift leaves
+// 4 * code without a mask.
+template <int W>
+struct CodeOffsets {
+    uint32_t even, odd;
+    __device__ __forceinline__ explicit CodeOffsets(uint32_t c) {
+        uint32_t me = 0;
+#pragma unroll
+        for (int i = 0; i < 8; i += 2) me |= ((1u << W) - 1u) << (i * W);
+        even = c & me;
+        odd = c & (me << W);
+    }
+    __device__ __forceinline__ uint32_t operator()(int i) const {
+        const uint32_t w = (i & 1) ? odd : even;
+        return (w * (1u << (32 - (i + 1) * W))) >> (30 - W);
+    }
+};
 
 // Philox4x32-10 with the round keys taken from the kernel arguments.
 __device__ __forceinline__ void philox_rk(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
@@ -121,17 +156,17 @@ __device__ __forceinline__ uint32_t seg_min_v(uint32_t v, bool hi) {
 }
 
 // Codes of the thread's eight elements.  2 and 4 bit: one aligned 16/32-bit access.
-// 3 bit: the warp's 256 codes are 24 consecutive words; lanes 0..23 access one word
+// 3 bit: the warp's 256 codes are 24 consecutive words; lanes 0..23 hold one word
 // each and the 24-bit pieces travel by shuffle.
 template <int BITS>
-__device__ __forceinline__ uint32_t warp_load_codes(const uint8_t* warp_base, int lane) {
+__device__ __forceinline__ uint32_t warp_codes_from_words(const uint32_t* words, int lane) {
+    // `words`: the warp's 8 * BITS packed words in shared memory
     if constexpr (BITS == 2) {
-        return __ldcs(reinterpret_cast<const unsigned short*>(warp_base) + lane);
+        return reinterpret_cast<const uint16_t*>(words)[lane];
     } else if constexpr (BITS == 4) {
-        return __ldcs(reinterpret_cast<const unsigned int*>(warp_base) + lane);
+        return words[lane];
     } else {
-        uint32_t w = 0;
-        if (lane < 24) w = __ldcs(reinterpret_cast<const unsigned int*>(warp_base) + lane);
+        const uint32_t w = words[lane];                           // lanes 24..31 read stale words, never used
         const int a = (3 * lane) >> 2, o = ((3 * lane) & 3) * 8;
         const uint32_t lo = __shfl_sync(0xffffffffu, w, a);
         const uint32_t hi = __shfl_sync(0xffffffffu, w, (a + 1) & 31);
@@ -166,29 +201,22 @@ __device__ __forceinline__ void sort8(uint32_t (&key)[EPT]) {
 // One selection round: finds the group's smallest unpopped key and pops it from exactly one
 // thread (the lowest lane among those whose head equals it), so that after r rounds the r
 // smallest keys, duplicates included, have been popped.  Returns that key (v domain).
-// `addr` is the shared-memory byte address of the thread's next row, `lt` the mask of the
-// lanes of the thread's group below it.  Unclamped form: `addr` advances one row per pop and
-// may be used for at most 16 rounds (rows 7..15 of a column hold the sentinel).  Clamped form:
-// any number of rounds; the address stops at the first sentinel row.
+// `off` is the word offset of the thread's next row in its column `col`, `le` the mask of the
+// lanes of the thread's group up to and including it, `self` the thread's own lane bit.
+// Unclamped form: `off` advances one row per pop and may be used for at most 16 rounds (rows
+// 7..15 of a column hold the sentinel).  Clamped form: any number of rounds; the offset stops at
+// the first sentinel row.
 template <int G, bool CLAMP>
-__device__ __forceinline__ uint32_t pop_round(uint32_t& head, uint32_t& addr, uint32_t last, uint32_t lt,
-                                              bool hi) {
+__device__ __forceinline__ uint32_t pop_round(uint32_t& head, int& off, const uint32_t* col, uint32_t le,
+                                              uint32_t self, bool hi) {
+    const uint32_t nxt = col[off];                               // the key that follows, should this thread pop
     const uint32_t tgt = seg_min_v<G>(head, hi);
-    const bool eq = head == tgt;
-    const uint32_t lower = __ballot_sync(0xffffffffu, eq) & lt;
-    if constexpr (CLAMP) {
-        asm volatile(
-            "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %3, 0;\n\tsetp.eq.and.u32 p, %2, 0, q;\n\t"
-            "@p ld.shared.u32 %0, [%1];\n\t"
-            "@p add.u32 %1, %1, %4;\n\t@p min.u32 %1, %1, %5;\n\t}"
-            : "+r"(head), "+r"(addr) : "r"(lower), "r"((int)eq), "n"(CTA * 4), "r"(last) : "memory");
-    } else {
-        asm volatile(
-            "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %3, 0;\n\tsetp.eq.and.u32 p, %2, 0, q;\n\t"
-            "@p ld.shared.u32 %0, [%1];\n\t"
-            "@p add.u32 %1, %1, %4;\n\t}"
-            : "+r"(head), "+r"(addr) : "r"(lower), "r"((int)eq), "n"(CTA * 4) : "memory");
-    }
+    // the lowest lane of the group whose head equals the minimum pops: its own bit is the lowest
+    // set bit of the ballot within the lanes of its group up to itself
+    const bool pop = (__ballot_sync(0xffffffffu, head == tgt) & le) == self;
+    head = pop ? nxt : head;
+    off += pop ? CTA : 0;
+    if constexpr (CLAMP) off = min(off, 7 * CTA);
     return tgt;
 }
 
@@ -196,29 +224,36 @@ __device__ __forceinline__ uint32_t pop_round(uint32_t& head, uint32_t& addr, ui
 // and may differ between the two halves of a warp (k <= 0: a group without a block, result
 // unused).  `col` is the thread's column of sorted keys (rows 0..6, sentinels from row 7 on),
 // `head` its smallest key.  UNIFORM_K: every group of the warp has the same k.
-template <int G, bool UNIFORM_K>
-__device__ __forceinline__ uint32_t select_kth(uint32_t head, const uint32_t* col, int k, bool hi) {
+// `side(i)`, i = 0..7, is independent work of the caller (the parameter update of element i)
+// that is issued between the rounds, where the warp would otherwise wait for the collectives.
+template <int G, bool UNIFORM_K, class Side>
+__device__ __forceinline__ uint32_t select_kth(uint32_t head, const uint32_t* col, int k, bool hi, Side&& side) {
     const int lane = threadIdx.x & 31;
-    const uint32_t below = (1u << lane) - 1u;
-    const uint32_t lt = (G == 16 && hi) ? below & 0xFFFF0000u : below;
-    const uint32_t addr0 = (uint32_t)__cvta_generic_to_shared(col);
-    const uint32_t last = addr0 + 7 * CTA * 4;
-    uint32_t addr = addr0, ans = 0;
+    const uint32_t self = 1u << lane;
+    const uint32_t upto = self | (self - 1u);
+    const uint32_t le = (G == 16 && hi) ? upto & 0xFFFF0000u : upto;
+    int off = 0;
+    uint32_t ans = 0;
     if (UNIFORM_K && k == 13) {
 #pragma unroll
-        for (int r = 0; r < 13; ++r) ans = pop_round<G, false>(head, addr, last, lt, hi);
+        for (int r = 0; r < 13; ++r) {
+            ans = pop_round<G, false>(head, off, col, le, self, hi);
+            if (r < EPT) side(r);
+        }
     } else {
+#pragma unroll
+        for (int i = 0; i < EPT; ++i) side(i);
         const int rounds = UNIFORM_K ? k : __reduce_max_sync(0xffffffffu, k);
         if (rounds <= 16) {
 #pragma unroll 1
             for (int r = 1; r <= rounds; ++r) {
-                const uint32_t t = pop_round<G, false>(head, addr, last, lt, hi);
+                const uint32_t t = pop_round<G, false>(head, off, col, le, self, hi);
                 if (r == k) ans = t;
             }
         } else {
 #pragma unroll 1
             for (int r = 1; r <= rounds; ++r) {
-                const uint32_t t = pop_round<G, true>(head, addr, last, lt, hi);
+                const uint32_t t = pop_round<G, true>(head, off, col, le, self, hi);
                 if (r == k) ans = t;
             }
         }
@@ -230,12 +265,50 @@ __device__ __forceinline__ void bar_sync(int id) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(CTA) : "memory");
 }
 
-// One tile.  FULL: all 2048 elements exist and both tensor pointers are 16-byte aligned.
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
+                 "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async4(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
+                 "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
+// Starts the asynchronous copy of a full tile's inputs into the staging area: `pt` / `gt` the
+// tile's parameters / gradients, `jb_tile` its first state block.  The caller has made sure (by
+// __syncwarp after its own reads) that the warp no longer reads the area.
+template <int BM, int BV, int G>
+__device__ __forceinline__ void stage_full(const StepArgs& a, FastShared& s, const char* pt, const char* gt,
+                                           int64_t jb_tile) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    cp_async16(&s.st_g[tid], gt + tid * 16);
+    cp_async16(&s.st_p0[tid], pt + tid * 32);
+    cp_async16(&s.st_p1[tid], pt + tid * 32 + 16);
+    const int64_t warp_slot0 = jb_tile * G + warp * 32;        // slot = 8 elements; 32 slots per warp
+    if (lane < 8 * BM) cp_async4(&s.st_cm[warp][lane], a.codes_m + warp_slot0 * BM + lane * 4);
+    if (lane < 8 * BV) cp_async4(&s.st_cv[warp][lane], a.codes_v + warp_slot0 * BV + lane * 4);
+    const int gl = tid & (G - 1), grp = tid / G;
+    if (gl < 3) {
+        const float* const src = gl == 0 ? a.scale_m : gl == 1 ? a.scale_v : a.alpha;
+        cp_async4(&s.st_sc[grp][gl], src + jb_tile + grp);
+    }
+    cp_async_commit();
+}
+
+// One tile.  FULL: all 2048 elements exist and both tensor pointers are 16-byte aligned.  A full
+// tile reads its inputs from the staging area; `staged` says whether the tile before it already
+// started that copy.  `next_full`: the tile this CTA visits next (`next_dtin` tiles further in
+// the same tensor) is full too, so its copy is started here and runs during this tile's
+// arithmetic.
+
 template <int BM, int BV, int G, bool FULL>
 __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, const float* s_y,
                                           const float* s_mid, char* pbase, const char* gbase,
                                           const int64_t n, const int64_t tin, const int64_t jb_tile,
-                                          const int tensor, const int par) {
+                                          const int tensor, const int par, bool& staged,
+                                          const bool next_full, const int64_t next_dtin) {
     constexpr int KM = 1 << BM, KV = 1 << BV;
     constexpr int NG = CTA / G, B = G * EPT;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -255,12 +328,19 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     const int64_t tile_slot0 = jb_tile * G;                     // slot = 8 elements = one thread's codes
     const int64_t jb = jb_tile + grp;
 
-    // ---- load ----
+    uint8_t* const wcm = a.codes_m + (tile_slot0 + warp * 32) * BM;   // the warp's 32 slots
+    uint8_t* const wcv = a.codes_v + (tile_slot0 + warp * 32) * BV;
+
+    // ---- inputs ----
     float p[EPT], g[EPT];
+    uint32_t cm = 0, cv = 0;
+    float dm = 0.0f, dv = 0.0f, al = 0.5f;
     if (FULL) {
-        const uint4 gw = __ldcs(reinterpret_cast<const uint4*>(gt) + tid);
-        const float4 p0 = __ldcs(reinterpret_cast<const float4*>(pt) + 2 * tid);
-        const float4 p1 = __ldcs(reinterpret_cast<const float4*>(pt) + 2 * tid + 1);
+        if (!staged) stage_full<BM, BV, G>(a, s, pt, gt, jb_tile);
+        cp_async_wait_all();                                     // this thread's copies have landed
+        __syncwarp();                                            // ... and those of the warp's other lanes
+        const uint4 gw = s.st_g[tid];
+        const float4 p0 = s.st_p0[tid], p1 = s.st_p1[tid];
         const uint32_t gg[4] = {gw.x, gw.y, gw.z, gw.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -269,6 +349,14 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
         }
         p[0] = p0.x; p[1] = p0.y; p[2] = p0.z; p[3] = p0.w;
         p[4] = p1.x; p[5] = p1.y; p[6] = p1.z; p[7] = p1.w;
+        cm = warp_codes_from_words<BM>(s.st_cm[warp], lane);
+        cv = warp_codes_from_words<BV>(s.st_cv[warp], lane);
+        dm = s.st_sc[grp][0]; dv = s.st_sc[grp][1]; al = s.st_sc[grp][2];
+        __syncwarp();                                            // all reads done before the area is refilled
+        staged = next_full;
+        if (next_full)
+            stage_full<BM, BV, G>(a, s, pt + next_dtin * (TILE * 4), gt + next_dtin * (TILE * 2),
+                                  jb_tile + next_dtin * NG);
     } else {
 #pragma unroll
         for (int i = 0; i < EPT; ++i) {
@@ -278,22 +366,13 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
                 p[i] = reinterpret_cast<const float*>(pt)[tid * EPT + i];
             }
         }
-    }
-    uint32_t cm = 0, cv = 0;
-    float dm = 0.0f, dv = 0.0f, al = 0.5f;
-    uint8_t* const wcm = a.codes_m + (tile_slot0 + warp * 32) * BM;   // the warp's 32 slots
-    uint8_t* const wcv = a.codes_v + (tile_slot0 + warp * 32) * BV;
-    if (FULL) {
-        cm = warp_load_codes<BM>(wcm, lane);
-        cv = warp_load_codes<BV>(wcv, lane);
-    } else if (have_block) {
-        cm = (uint32_t)load_codes<BM>(wcm + lane * BM);
-        cv = (uint32_t)load_codes<BV>(wcv + lane * BV);
-    }
-    if (have_block) {
-        dm = __ldg(a.scale_m + jb);
-        dv = __ldg(a.scale_v + jb);
-        al = __ldg(a.alpha + jb);
+        if (have_block) {
+            cm = (uint32_t)load_codes<BM>(wcm + lane * BM);
+            cv = (uint32_t)load_codes<BV>(wcv + lane * BV);
+            dm = __ldg(a.scale_m + jb);
+            dv = __ldg(a.scale_v + jb);
+            al = __ldg(a.alpha + jb);
+        }
     }
 
     // ---- per-block level tables: alpha^k Delta_v and y_k Delta_m (Eq. 2) ----
@@ -315,38 +394,40 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
 
     // ---- Eq. 2, Eq. 3, Adam(W) ----
     float mh[EPT], vh[EPT];
-    uint32_t mx_m = 0, mx_v = 0;
+    uint32_t mx_v = 0;
+    float mx_m_f = 0.0f;                                         // max |m^| (a NaN element is passed over)
     const char* const tab_v = reinterpret_cast<const char*>(tab);
     const char* const tab_m = reinterpret_cast<const char*>(tab + KV);
-    const uint32_t cm4 = cm << 2, cv4 = cv << 2;
+    const CodeOffsets<BM> om4(cm);
+    const CodeOffsets<BV> ov4(cv);
 #pragma unroll
     for (int i = 0; i < EPT; ++i) {
-        const uint32_t im = i * BM >= 2 ? (cm >> (i * BM - 2)) & ((KM - 1) << 2) : (cm4 >> (i * BM)) & ((KM - 1) << 2);
-        const uint32_t iv = i * BV >= 2 ? (cv >> (i * BV - 2)) & ((KV - 1) << 2) : (cv4 >> (i * BV)) & ((KV - 1) << 2);
-        const float mt = *reinterpret_cast<const float*>(tab_m + im);
-        const float vt = *reinterpret_cast<const float*>(tab_v + iv);
+        const float mt = *reinterpret_cast<const float*>(tab_m + om4(i));
+        const float vt = *reinterpret_cast<const float*>(tab_v + ov4(i));
         const float gi = g[i];
         mh[i] = __fmaf_rn(a.beta1, mt, a.omb1 * gi);
         vh[i] = __fmaf_rn(a.beta2, vt, a.omb2 * (gi * gi));
+        const bool valid = FULL || i < nv;
+        mx_m_f = fmaxf(mx_m_f, valid ? fabsf(mh[i]) : 0.0f);
+        mx_v = max(mx_v, valid ? __float_as_uint(vh[i]) : 0u);
+    }
+    uint32_t mx_m = __float_as_uint(mx_m_f);
+
+    // Adam(W) update of element i and, after every fourth, the store; issued between the
+    // rounds of the selection below, which it does not depend on
+    auto update = [&](int i) {
         const float den = __fmaf_rn(sqrt_approx(vh[i]), a.inv_sqrt_bc2, a.eps);
         const float rc = rcp_approx(den);
         const float q0 = mh[i] * rc;
         const float q1 = __fmaf_rn(__fmaf_rn(-den, q0, mh[i]), rc, q0);
         p[i] = __fmaf_rn(-a.step_size, q1, p[i] * a.decay);
-        const bool valid = FULL || i < nv;
-        mx_m = max(mx_m, valid ? __float_as_uint(mh[i]) & 0x7fffffffu : 0u);
-        mx_v = max(mx_v, valid ? __float_as_uint(vh[i]) : 0u);
-    }
-
-    // ---- store parameters ----
-    if (FULL) {
-        __stcs(reinterpret_cast<float4*>(pt) + 2 * tid, make_float4(p[0], p[1], p[2], p[3]));
-        __stcs(reinterpret_cast<float4*>(pt) + 2 * tid + 1, make_float4(p[4], p[5], p[6], p[7]));
-    } else {
-#pragma unroll
-        for (int i = 0; i < EPT; ++i)
+        if (FULL) {
+            if (i == 3) __stcs(reinterpret_cast<float4*>(pt) + 2 * tid, make_float4(p[0], p[1], p[2], p[3]));
+            if (i == 7) __stcs(reinterpret_cast<float4*>(pt) + 2 * tid + 1, make_float4(p[4], p[5], p[6], p[7]));
+        } else {
             if (i < nv) reinterpret_cast<float*>(pt)[tid * EPT + i] = p[i];
-    }
+        }
+    };
 
     // ---- block scales and the p-quantile of v^ (Sec. 3.2.2) ----
     mx_m = seg_max31<G>(mx_m, hi);
@@ -363,11 +444,11 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
         const uint32_t head = key[0] ^ vflip;
         uint32_t xv;
         if (FULL) {
-            xv = select_kth<G, true>(head, col, a.k_full, hi);
+            xv = select_kth<G, true>(head, col, a.k_full, hi, update);
         } else {
             int k = (int)ceil((double)a.p_quantile * (double)nb);
             k = min(max(k, 1), nb);                              // 0 for a group without a block
-            xv = select_kth<G, false>(head, col, k, hi);
+            xv = select_kth<G, false>(head, col, k, hi, update);
         }
         x_p = xv ^ vflip;
     }
@@ -403,15 +484,9 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     bar_sync(2);
     if (warp == 0 && a.round_v)
         philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, (uint32_t)tensor * 4u, a.rk, w);
-    float xi[EPT];
-    {
+    float dr[EPT];                                               // the 16-bit draws d as binary32
 #pragma unroll
-        for (int i = 0; i < EPT; ++i) {
-            // (d + 1/2) / 2^16 - 1/2 for the 16-bit draw d, via the binary32 1 + d 2^-16
-            const uint32_t h7 = (i & 1) ? (w[i >> 1] >> 9) & 0x007FFF80u : (w[i >> 1] << 7) & 0x007FFF80u;
-            xi[i] = a.round_v ? __uint_as_float(0x3F800000u | h7) + (-1.5f + 0x1p-17f) : 0.0f;
-        }
-    }
+    for (int i = 0; i < 4; ++i) halves_to_float(w[i], dr[2 * i], dr[2 * i + 1]);
     const float4 sc = s.xout[par][grp];
     const uint32_t zf = s.xflag[par][grp];
 
@@ -443,21 +518,27 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     }
 
     // ---- second moment: Eq. 6 ----
+    // t = log_alpha(r) + xi is evaluated divided by K - 1, so that the clamp to [0, K-1] is the
+    // saturation of the fused multiply-add; adding 1.5 * 2^23 to (K-1) * t rounds it to an integer.
     uint32_t ov = 0;
     {
         const float inv = sc.y, il = sc.z, lim = sc.w;
-        constexpr float MAGIC = 12582912.0f;                     // 1.5 * 2^23: adding it rounds to an integer
+        constexpr float KM1 = (float)(KV - 1);
+        constexpr float MAGIC = 12582912.0f;
         constexpr uint32_t MAGIC_BITS = 0x4B400000u;
+        const float ils = il * (1.0f / KM1);
+        // xi = (d + 1/2) / 2^16 - 1/2 (exact); scaled copy for the approximate path
+        const float xs1 = a.round_v ? (float)(0x1p-16 / (KV - 1)) : 0.0f;
+        const float xs0 = a.round_v ? (float)((-0.5 + 0x1p-17) / (KV - 1)) : 0.0f;
         float worst = 0.0f;
         uint32_t acc = 0;
 #pragma unroll
         for (int i = EPT - 1; i >= 0; --i) {
             const float r = vh[i] * inv;
-            float t = __fmaf_rn(lg2_approx(r), il, xi[i]);
-            t = fminf(fmaxf(t, 0.0f), (float)(KV - 1));
-            const float u = t + MAGIC;
-            worst = fmaxf(worst, fabsf(t - (u - MAGIC)));
-            acc = (acc << BV) + ((FULL || i < nv) ? __float_as_uint(u) : MAGIC_BITS);
+            const float ts = __saturatef(__fmaf_rn(lg2_approx(r), ils, __fmaf_rn(dr[i], xs1, xs0)));
+            const float u = __fmaf_rn(ts, KM1, MAGIC);
+            worst = fmaxf(worst, fabsf(__fmaf_rn(ts, KM1, MAGIC - u)));
+            acc = acc * (1u << BV) + ((FULL || i < nv) ? __float_as_uint(u) : MAGIC_BITS);
         }
         uint32_t magic_sum = 0;
 #pragma unroll
@@ -466,14 +547,15 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
         if (__any_sync(0xffffffffu, worst > lim)) {
             // some element of the warp is too close to a rounding boundary for the
             // approximate logarithm: evaluate the exact sequence for all eight
+            const float x1 = a.round_v ? 0x1p-16f : 0.0f, x0 = a.round_v ? -0.5f + 0x1p-17f : 0.0f;
             ov = 0;
 #pragma unroll
             for (int i = EPT - 1; i >= 0; --i) {
                 const float r = vh[i] * inv;
                 uint32_t q = KV - 1;
                 if (!(r < TINY)) {
-                    float t = __fmaf_rn(log2_sp(r), il, xi[i]);
-                    t = fminf(fmaxf(t, 0.0f), (float)(KV - 1));
+                    float t = __fmaf_rn(log2_sp(r), il, __fmaf_rn(dr[i], x1, x0));
+                    t = fminf(fmaxf(t, 0.0f), KM1);
                     q = (uint32_t)__float2int_rn(t);
                 }
                 ov = (ov << BV) + ((FULL || i < nv) ? q : 0u);
@@ -511,7 +593,7 @@ __global__ void __launch_bounds__(CTA, 3) solo_step_fast_kernel(const StepArgs a
     int64_t t_lo = 0, t_hi = 0, n = 0, jb0 = 0;
     char* pbase = nullptr;
     const char* gbase = nullptr;
-    bool aligned = false, skip = false;
+    bool aligned = false, skip = false, staged = false;
     int par = 0;
     for (int64_t tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x) {
         if (tile >= t_hi) {
@@ -531,10 +613,15 @@ __global__ void __launch_bounds__(CTA, 3) solo_step_fast_kernel(const StepArgs a
         if (skip) continue;
         const int64_t tin = tile - t_lo;
         const int64_t jb_tile = jb0 + tin * (CTA / G);
+        // the tile this CTA visits next: full and in the same tensor?
+        const int64_t ntin = tin + gridDim.x;
+        const bool next_full = aligned && tile + gridDim.x < t_hi && (ntin + 1) * TILE <= n;
         if (aligned && (tin + 1) * TILE <= n)
-            fast_tile<BM, BV, G, true>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par);
+            fast_tile<BM, BV, G, true>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, staged,
+                                       next_full, (int64_t)gridDim.x);
         else
-            fast_tile<BM, BV, G, false>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par);
+            fast_tile<BM, BV, G, false>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, staged,
+                                        false, 0);
         par ^= 1;
     }
 }
