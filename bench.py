@@ -34,9 +34,10 @@ UNIT = "Gparams/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per parameter of the step kernel from an ncu capture
-# (dram__bytes_read.sum + dram__bytes_write.sum over the parameters of the captured launch);
-# filled in from profiles/ once a capture exists, else None.
-NCU_TRAFFIC_BYTES_PER_PARAM = None
+# (dram__bytes_read.sum + dram__bytes_write.sum over the parameters of the captured launch, taken on
+# the first three tensors of the 7B-shaped set and scaled by the element count; see profiles/).
+# Valid for the 2-bit / 3-bit, block 128 streamlined kernel only; None for anything else.
+NCU_TRAFFIC_BYTES_PER_PARAM = 11.12
 
 
 def algorithmic_bytes_per_param(bits_m: int, bits_v: int, block: int, param_bytes: int = 4) -> float:
@@ -109,8 +110,17 @@ class ClockSampler:
 
 def build_workload(cfg: int, device, args):
     w = synth.workload(cfg)
+    over = {}
     if args.max_tensors:
-        w = synth.workload(cfg, sizes=w.sizes[: args.max_tensors])
+        over["sizes"] = w.sizes[: args.max_tensors]
+    if args.bits_m:
+        over["bits_m"] = args.bits_m
+    if args.bits_v:
+        over["bits_v"] = args.bits_v
+    if args.block:
+        over["block"] = args.block
+    if over:
+        w = synth.workload(cfg, **over)
     params = [synth.make_param(w, i, device=device) for i in range(len(w.sizes))]
     grads = [synth.make_grad(w, i, 1, device=device) for i in range(len(w.sizes))]
     return w, params, grads
@@ -210,8 +220,9 @@ def run_ours(args, rank, world):
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
                      "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind} copy bandwidth",
                      "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
-                     "traffic": (None if NCU_TRAFFIC_BYTES_PER_PARAM is None
-                                 else round(NCU_TRAFFIC_BYTES_PER_PARAM * n))},
+                     "traffic": (round(NCU_TRAFFIC_BYTES_PER_PARAM * n)
+                                 if (NCU_TRAFFIC_BYTES_PER_PARAM is not None and args.policy == 0 and
+                                     (w.bits_m, w.bits_v, w.block) == (2, 3, 128)) else None)},
         "gpu_launches": int(launches),
         "clocks": clk,
     }
@@ -272,6 +283,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=3)
     ap.add_argument("--max-tensors", type=int, default=0, help="use only the first tensors (small captures)")
+    ap.add_argument("--bits-m", type=int, default=0, help="override the workload's first-moment width")
+    ap.add_argument("--bits-v", type=int, default=0, help="override the workload's second-moment width")
+    ap.add_argument("--block", type=int, default=0, help="override the workload's block size")
     ap.add_argument("--cpu-sample", type=int, default=1 << 27)
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--policy", type=int, default=0, help="kernel policy: 0 streamlined where it applies, 1 general")

@@ -576,7 +576,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
 }
 
 template <int BM, int BV, int G>
-__global__ void __launch_bounds__(CTA, 3) solo_step_fast_kernel(const StepArgs a) {
+__global__ void __launch_bounds__(CTA, 4) solo_step_fast_kernel(const StepArgs a) {
     constexpr int KM = 1 << BM;
     __shared__ FastShared s;
     __shared__ float s_y[KM];
