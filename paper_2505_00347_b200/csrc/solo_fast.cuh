@@ -206,9 +206,10 @@ __device__ __forceinline__ void sort8(uint32_t (&key)[EPT]) {
 // Unclamped form: `off` advances one row per pop and may be used for at most 16 rounds (rows
 // 7..15 of a column hold the sentinel).  Clamped form: any number of rounds; the offset stops at
 // the first sentinel row.
-template <int G, bool CLAMP>
+template <int G, bool CLAMP, bool LAST = false>
 __device__ __forceinline__ uint32_t pop_round(uint32_t& head, int& off, const uint32_t* col, uint32_t le,
                                               uint32_t self, bool hi) {
+    if constexpr (LAST) return seg_min_v<G>(head, hi);          // the answer; nothing left to pop
     const uint32_t nxt = col[off];                               // the key that follows, should this thread pop
     const uint32_t tgt = seg_min_v<G>(head, hi);
     // the lowest lane of the group whose head equals the minimum pops: its own bit is the lowest
@@ -236,10 +237,11 @@ __device__ __forceinline__ uint32_t select_kth(uint32_t head, const uint32_t* co
     uint32_t ans = 0;
     if (UNIFORM_K && k == 13) {
 #pragma unroll
-        for (int r = 0; r < 13; ++r) {
-            ans = pop_round<G, false>(head, off, col, le, self, hi);
+        for (int r = 0; r < 12; ++r) {
+            pop_round<G, false>(head, off, col, le, self, hi);
             if (r < EPT) side(r);
         }
+        ans = pop_round<G, false, true>(head, off, col, le, self, hi);
     } else {
 #pragma unroll
         for (int i = 0; i < EPT; ++i) side(i);
@@ -306,9 +308,9 @@ __device__ __forceinline__ void stage_full(const StepArgs& a, FastShared& s, con
 template <int BM, int BV, int G, bool FULL>
 __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, const float* s_y,
                                           const float* s_mid, char* pbase, const char* gbase,
-                                          const int64_t n, const int64_t tin, const int64_t jb_tile,
+                                          const int64_t n, const int tin, const int64_t jb_tile,
                                           const int tensor, const int par, bool& staged,
-                                          const bool next_full, const int64_t next_dtin) {
+                                          const bool next_full, const int next_dtin) {
     constexpr int KM = 1 << BM, KV = 1 << BV;
     constexpr int NG = CTA / G, B = G * EPT;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -317,7 +319,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     const uint32_t vflip = hi ? 0xFFFFFFFFu : 0u;               // x domain <-> v domain
 
     // validity (all true in a full tile)
-    const int64_t tile_elem0 = tin * TILE;
+    const int64_t tile_elem0 = (int64_t)tin * TILE;
     const int64_t rem_tile = n - tile_elem0;                    // elements of the tensor from the tile's first on, > 0
     const bool have_block = FULL || (int64_t)grp * B < rem_tile;
     const int nb = FULL ? B : (int)max((int64_t)0, min((int64_t)B, rem_tile - (int64_t)grp * B));
@@ -355,8 +357,8 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
         __syncwarp();                                            // all reads done before the area is refilled
         staged = next_full;
         if (next_full)
-            stage_full<BM, BV, G>(a, s, pt + next_dtin * (TILE * 4), gt + next_dtin * (TILE * 2),
-                                  jb_tile + next_dtin * NG);
+            stage_full<BM, BV, G>(a, s, pt + (int64_t)next_dtin * (TILE * 4), gt + (int64_t)next_dtin * (TILE * 2),
+                                  jb_tile + (int64_t)next_dtin * NG);
     } else {
 #pragma unroll
         for (int i = 0; i < EPT; ++i) {
@@ -457,7 +459,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     if (gl == 0) s.xin[par][grp] = make_uint4(mx_m, mx_v, x_p, 0u);
     bar_sync(1);
     uint32_t w[4] = {0u, 0u, 0u, 0u};
-    const uint64_t ctr = (uint64_t)tin * (TILE / EPT) + (uint32_t)tid;     // element index / 8
+    const uint64_t ctr = (uint64_t)(uint32_t)tin * (TILE / EPT) + (uint32_t)tid;   // element index / 8
     if (warp != 0) {
         if (a.round_v) philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, (uint32_t)tensor * 4u, a.rk, w);
     } else if (tid < NG) {
@@ -494,7 +496,24 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     uint32_t om = 0;
     {
         const float inv = sc.x;
-        if constexpr (BM == 2) {
+        if constexpr (BM == 2 && FULL) {
+            // code = number of midpoints below r.  Each "r > mid" is evaluated on the FMA pipe as
+            // the saturation of (r - mid) * 2^100: the fused multiply-add rounds the exact
+            // difference, which is zero or at least 2^-30 in magnitude, so the result is exactly
+            // 0 or 1 (a NaN saturates to 0, as the comparison would give).  The eight 2-bit codes
+            // are accumulated in binary32 (16 bits: exact).
+            constexpr float BIG = 0x1p100f;
+            const float n0 = -s_mid[0] * BIG, n1 = -s_mid[1] * BIG, n2 = -s_mid[2] * BIG;
+            float omf = 0.0f;
+#pragma unroll
+            for (int i = EPT - 1; i >= 0; --i) {
+                const float r = mh[i] * inv;
+                omf = __fmaf_rn(omf, 4.0f, __saturatef(__fmaf_rn(r, BIG, n0)));
+                omf += __saturatef(__fmaf_rn(r, BIG, n1));
+                omf += __saturatef(__fmaf_rn(r, BIG, n2));
+            }
+            om = (uint32_t)omf;
+        } else if constexpr (BM == 2) {
             const float mid0 = s_mid[0], mid1 = s_mid[1], mid2 = s_mid[2];
 #pragma unroll
             for (int i = EPT - 1; i >= 0; --i) {
@@ -589,36 +608,38 @@ __global__ void __launch_bounds__(CTA, 4) solo_step_fast_kernel(const StepArgs a
     for (int r = 7; r < 16; ++r) s.sort[r][tid] = (G == 16 && (tid & 16)) ? ~KEY_MAX : KEY_MAX;   // sentinels, v domain
     __syncthreads();
 
+    // Tile indices fit 32 bits (the host selects this kernel only below 2^31 tiles).  Tiles are
+    // visited in increasing order, so the tensor of a tile is found by walking forward.
+    const int total_tiles = (int)a.total_tiles, stride = (int)gridDim.x;
     int tensor = -1;
-    int64_t t_lo = 0, t_hi = 0, n = 0, jb0 = 0;
+    int t_lo = 0, t_hi = 0, full_tiles = 0;      // the tensor's tiles [t_lo, t_hi); its first full_tiles are full
+    int64_t n = 0, jb0 = 0;
     char* pbase = nullptr;
     const char* gbase = nullptr;
-    bool aligned = false, skip = false, staged = false;
+    bool skip = false, staged = false;
     int par = 0;
-    for (int64_t tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x) {
+    for (int tile = blockIdx.x; tile < total_tiles; tile += stride) {
         if (tile >= t_hi) {
             do {
                 ++tensor;
-                t_hi = __ldg(a.tile_start + tensor + 1);
+                t_hi = (int)__ldg(a.tile_start + tensor + 1);
             } while (tile >= t_hi);
-            t_lo = __ldg(a.tile_start + tensor);
+            t_lo = (int)__ldg(a.tile_start + tensor);
             n = __ldg(a.numel + tensor);
             jb0 = __ldg(a.block_start + tensor);
             pbase = (char*)(a.param_list ? a.param_list[tensor] : a.param_single);
             gbase = (const char*)(a.grad_list ? a.grad_list[tensor] : a.grad_single);
-            aligned = ((((uintptr_t)pbase) | ((uintptr_t)gbase)) & 15u) == 0;
+            const bool aligned = ((((uintptr_t)pbase) | ((uintptr_t)gbase)) & 15u) == 0;
+            full_tiles = aligned ? (int)(n / TILE) : 0;
             skip = a.numel_check != nullptr && __ldg(a.numel_check + tensor) != n;
             if (skip && tid == 0) atomicOr(a.status, 1);
         }
         if (skip) continue;
-        const int64_t tin = tile - t_lo;
-        const int64_t jb_tile = jb0 + tin * (CTA / G);
-        // the tile this CTA visits next: full and in the same tensor?
-        const int64_t ntin = tin + gridDim.x;
-        const bool next_full = aligned && tile + gridDim.x < t_hi && (ntin + 1) * TILE <= n;
-        if (aligned && (tin + 1) * TILE <= n)
+        const int tin = tile - t_lo;
+        const int64_t jb_tile = jb0 + (int64_t)tin * (CTA / G);
+        if (tin < full_tiles)
             fast_tile<BM, BV, G, true>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, staged,
-                                       next_full, (int64_t)gridDim.x);
+                                       tin + stride < full_tiles, stride);
         else
             fast_tile<BM, BV, G, false>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, staged,
                                         false, 0);
