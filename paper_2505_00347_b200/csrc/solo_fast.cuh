@@ -94,7 +94,9 @@ struct CodeOffsets {
     }
     __device__ __forceinline__ uint32_t operator()(int i) const {
         const uint32_t w = (i & 1) ? odd : even;
-        return (w * (1u << (32 - (i + 1) * W))) >> (30 - W);
+        uint32_t top;       // the code moved to the top of the word (a multiply: kept apart from the shift)
+        asm("mul.lo.u32 %0, %1, %2;" : "=r"(top) : "r"(w), "r"(1u << (32 - (i + 1) * W)));
+        return top >> (30 - W);
     }
 };
 
