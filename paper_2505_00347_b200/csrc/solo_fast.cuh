@@ -46,14 +46,6 @@ struct FastShared {
     uint4 xin[2][CTA / 16];                  // per group: bits of Delta_m', Delta_v', x_p
     float4 xout[2][CTA / 16];                // per group: 1/Delta_m', 1/Delta_v', 1/log2(alpha'), rounding limit
     uint32_t xflag[2][CTA / 16];             // bit 0: vanishing first moment, bit 1: vanishing second moment
-    // Inputs of a full tile, copied asynchronously (cp.async) one tile ahead of their use.  Every
-    // thread copies the parameters and gradients it reads itself; codes and scales are shared by
-    // a warp.
-    float4 st_p0[CTA], st_p1[CTA];           // a thread's eight parameters
-    uint4 st_g[CTA];                         // its eight bf16 gradients
-    uint32_t st_cm[CTA / 32][32];            // a warp's packed codes (8 * bits words)
-    uint32_t st_cv[CTA / 32][32];
-    float st_sc[CTA / 16][4];                // a group's Delta_m, Delta_v, alpha
 };
 
 __device__ __forceinline__ float lg2_approx(float x) {
@@ -158,17 +150,17 @@ __device__ __forceinline__ uint32_t seg_min_v(uint32_t v, bool hi) {
 }
 
 // Codes of the thread's eight elements.  2 and 4 bit: one aligned 16/32-bit access.
-// 3 bit: the warp's 256 codes are 24 consecutive words; lanes 0..23 hold one word
+// 3 bit: the warp's 256 codes are 24 consecutive words; lanes 0..23 access one word
 // each and the 24-bit pieces travel by shuffle.
 template <int BITS>
-__device__ __forceinline__ uint32_t warp_codes_from_words(const uint32_t* words, int lane) {
-    // `words`: the warp's 8 * BITS packed words in shared memory
+__device__ __forceinline__ uint32_t warp_load_codes(const uint8_t* warp_base, int lane) {
     if constexpr (BITS == 2) {
-        return reinterpret_cast<const uint16_t*>(words)[lane];
+        return __ldcs(reinterpret_cast<const unsigned short*>(warp_base) + lane);
     } else if constexpr (BITS == 4) {
-        return words[lane];
+        return __ldcs(reinterpret_cast<const unsigned int*>(warp_base) + lane);
     } else {
-        const uint32_t w = words[lane];                           // lanes 24..31 read stale words, never used
+        uint32_t w = 0;
+        if (lane < 24) w = __ldcs(reinterpret_cast<const unsigned int*>(warp_base) + lane);
         const int a = (3 * lane) >> 2, o = ((3 * lane) & 3) * 8;
         const uint32_t lo = __shfl_sync(0xffffffffu, w, a);
         const uint32_t hi = __shfl_sync(0xffffffffu, w, (a + 1) & 31);
@@ -216,9 +208,10 @@ __device__ __forceinline__ uint32_t pop_round(uint32_t& head, int& off, const ui
     const uint32_t tgt = seg_min_v<G>(head, hi);
     // the lowest lane of the group whose head equals the minimum pops: its own bit is the lowest
     // set bit of the ballot within the lanes of its group up to itself
-    const bool pop = (__ballot_sync(0xffffffffu, head == tgt) & le) == self;
-    head = pop ? nxt : head;
-    off += pop ? CTA : 0;
+    const uint32_t upto = __ballot_sync(0xffffffffu, head == tgt) & le;
+    // if (upto == self) { head = nxt; off += CTA; }  as two predicated instructions
+    asm("{\n\t.reg .pred p;\n\tsetp.eq.u32 p, %2, %3;\n\t@p mov.u32 %0, %4;\n\t@p add.s32 %1, %1, %5;\n\t}"
+        : "+r"(head), "+r"(off) : "r"(upto), "r"(self), "r"(nxt), "n"(CTA));
     if constexpr (CLAMP) off = min(off, 7 * CTA);
     return tgt;
 }
@@ -269,50 +262,17 @@ __device__ __forceinline__ void bar_sync(int id) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(CTA) : "memory");
 }
 
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
-                 "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async4(void* smem_dst, const void* gmem_src) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
-                 "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
-
-// Starts the asynchronous copy of a full tile's inputs into the staging area: `pt` / `gt` the
-// tile's parameters / gradients, `jb_tile` its first state block.  The caller has made sure (by
-// __syncwarp after its own reads) that the warp no longer reads the area.
-template <int BM, int BV, int G>
-__device__ __forceinline__ void stage_full(const StepArgs& a, FastShared& s, const char* pt, const char* gt,
-                                           int64_t jb_tile) {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    cp_async16(&s.st_g[tid], gt + tid * 16);
-    cp_async16(&s.st_p0[tid], pt + tid * 32);
-    cp_async16(&s.st_p1[tid], pt + tid * 32 + 16);
-    const int64_t warp_slot0 = jb_tile * G + warp * 32;        // slot = 8 elements; 32 slots per warp
-    if (lane < 8 * BM) cp_async4(&s.st_cm[warp][lane], a.codes_m + warp_slot0 * BM + lane * 4);
-    if (lane < 8 * BV) cp_async4(&s.st_cv[warp][lane], a.codes_v + warp_slot0 * BV + lane * 4);
-    const int gl = tid & (G - 1), grp = tid / G;
-    if (gl < 3) {
-        const float* const src = gl == 0 ? a.scale_m : gl == 1 ? a.scale_v : a.alpha;
-        cp_async4(&s.st_sc[grp][gl], src + jb_tile + grp);
-    }
-    cp_async_commit();
-}
-
-// One tile.  FULL: all 2048 elements exist and both tensor pointers are 16-byte aligned.  A full
-// tile reads its inputs from the staging area; `staged` says whether the tile before it already
-// started that copy.  `next_full`: the tile this CTA visits next (`next_dtin` tiles further in
-// the same tensor) is full too, so its copy is started here and runs during this tile's
-// arithmetic.
+// One tile.  FULL: all 2048 elements exist and both tensor pointers are 16-byte aligned.
+// Inputs are loaded straight from global memory (128-bit streaming loads); staging the next
+// tile through shared memory with cp.async, or requesting its lines into L2 ahead of time,
+// was measured slower: the extra instructions cost more than the hidden latency gains, the
+// four resident CTAs per SM cover each other's load phases.
 
 template <int BM, int BV, int G, bool FULL>
 __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, const float* s_y,
                                           const float* s_mid, char* pbase, const char* gbase,
                                           const int64_t n, const int tin, const int64_t jb_tile,
-                                          const int tensor, const int par, bool& staged,
-                                          const bool next_full, const int next_dtin) {
+                                          const int tensor, const int par) {
     constexpr int KM = 1 << BM, KV = 1 << BV;
     constexpr int NG = CTA / G, B = G * EPT;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -340,11 +300,9 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     uint32_t cm = 0, cv = 0;
     float dm = 0.0f, dv = 0.0f, al = 0.5f;
     if (FULL) {
-        if (!staged) stage_full<BM, BV, G>(a, s, pt, gt, jb_tile);
-        cp_async_wait_all();                                     // this thread's copies have landed
-        __syncwarp();                                            // ... and those of the warp's other lanes
-        const uint4 gw = s.st_g[tid];
-        const float4 p0 = s.st_p0[tid], p1 = s.st_p1[tid];
+        const uint4 gw = __ldcs(reinterpret_cast<const uint4*>(gt) + tid);
+        const float4 p0 = __ldcs(reinterpret_cast<const float4*>(pt) + 2 * tid);
+        const float4 p1 = __ldcs(reinterpret_cast<const float4*>(pt) + 2 * tid + 1);
         const uint32_t gg[4] = {gw.x, gw.y, gw.z, gw.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -353,14 +311,11 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
         }
         p[0] = p0.x; p[1] = p0.y; p[2] = p0.z; p[3] = p0.w;
         p[4] = p1.x; p[5] = p1.y; p[6] = p1.z; p[7] = p1.w;
-        cm = warp_codes_from_words<BM>(s.st_cm[warp], lane);
-        cv = warp_codes_from_words<BV>(s.st_cv[warp], lane);
-        dm = s.st_sc[grp][0]; dv = s.st_sc[grp][1]; al = s.st_sc[grp][2];
-        __syncwarp();                                            // all reads done before the area is refilled
-        staged = next_full;
-        if (next_full)
-            stage_full<BM, BV, G>(a, s, pt + (int64_t)next_dtin * (TILE * 4), gt + (int64_t)next_dtin * (TILE * 2),
-                                  jb_tile + (int64_t)next_dtin * NG);
+        cm = warp_load_codes<BM>(wcm, lane);
+        cv = warp_load_codes<BV>(wcv, lane);
+        dm = __ldg(a.scale_m + jb);
+        dv = __ldg(a.scale_v + jb);
+        al = __ldg(a.alpha + jb);
     } else {
 #pragma unroll
         for (int i = 0; i < EPT; ++i) {
@@ -618,7 +573,7 @@ __global__ void __launch_bounds__(CTA, 4) solo_step_fast_kernel(const StepArgs a
     int64_t n = 0, jb0 = 0;
     char* pbase = nullptr;
     const char* gbase = nullptr;
-    bool skip = false, staged = false;
+    bool skip = false;
     int par = 0;
     for (int tile = blockIdx.x; tile < total_tiles; tile += stride) {
         if (tile >= t_hi) {
@@ -640,11 +595,9 @@ __global__ void __launch_bounds__(CTA, 4) solo_step_fast_kernel(const StepArgs a
         const int tin = tile - t_lo;
         const int64_t jb_tile = jb0 + (int64_t)tin * (CTA / G);
         if (tin < full_tiles)
-            fast_tile<BM, BV, G, true>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, staged,
-                                       tin + stride < full_tiles, stride);
+            fast_tile<BM, BV, G, true>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par);
         else
-            fast_tile<BM, BV, G, false>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, staged,
-                                        false, 0);
+            fast_tile<BM, BV, G, false>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par);
         par ^= 1;
     }
 }
