@@ -196,15 +196,11 @@ def run_ours(args, rank, world):
         sync_all()
         e2e_ms = e0.elapsed_time(e1) / k
 
-    times = torch.tensor([ms, e2e_ms or 0.0], dtype=torch.float64, device=device)
-    if world > 1:
-        import torch.distributed as dist
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms, e2e_max = float(times[0]), float(times[1])
+    ms, e2e_max = max_over_ranks([ms, e2e_ms or 0.0], device, world)
     if rank != 0:
         return None
     ms_per_step = ms / args.steps
-    value = world * n / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_gparams(world, n, ms_per_step)
     abytes = algorithmic_bytes_per_param(w.bits_m, w.bits_v, w.block)
     achieved = n * abytes / (ms_per_step * 1e-3) / 1e9
     peak, peak_kind = measured_peak()
@@ -232,6 +228,21 @@ def run_ours(args, rank, world):
     if world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(w, args.cpu_sample)
     return out
+
+
+def max_over_ranks(values, device, world: int) -> list:
+    """Element-wise maximum of `values` over all ranks (the slowest rank defines the job's time)."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def whole_job_gparams(world: int, params_per_rank: int, ms_per_step: float) -> float:
+    """Every rank steps its own replica of the workload (no data-path collective): the job's
+    throughput is all ranks' parameters over the slowest rank's time."""
+    return world * params_per_rank / (ms_per_step * 1e-3) / 1e9
 
 
 def cpu_baseline(w, sample_elems: int, steps: int = 1) -> dict:
