@@ -297,6 +297,7 @@ struct so_hyper {
     float lr, beta1, beta2, eps, weight_decay;
     float p_quantile;
     int32_t adamw, bias_correction, round_m, round_v, param_dtype;
+    int32_t belief;       // 0: Adam(W); 1: AdaBelief (second moment tracks (g - m^)^2 + eps)
     uint64_t seed;
 };
 
@@ -408,9 +409,12 @@ static void step_blocks(void* param, const uint16_t* grad, int64_t n, int64_t el
             // Eq. 2 (or, with the full-precision switch, the stored binary32 moments)
             float m_t = m32 ? m32[i] : ym[get_code(cm, e, bits_m)] * dm;
             float v_t = v32 ? v32[i] : pow_sm(al, get_code(cv, e, bits_v)) * dv;
-            // Eq. 3
+            // Eq. 3.  AdaBelief (Sec. 5.2, "AdaBelief"; Zhuang et al. 2020): the unsigned EMA's
+            // signal is (g - m^)^2 instead of g^2 and eps is added to the state at every step
             float m_h = std::fmaf(b1, m_t, omb1 * g);
-            float v_h = std::fmaf(b2, v_t, omb2 * (g * g));
+            float sig = h->belief ? g - m_h : g;
+            float v_h = std::fmaf(b2, v_t, omb2 * (sig * sig));
+            if (h->belief) v_h = v_h + h->eps;
             mh[e] = m_h;
             vh[e] = v_h;
             // Adam(W) with the un-requantized moments

@@ -48,6 +48,39 @@ def test_full_precision_switch_is_textbook_adam(adamw):
     assert np.all(st.codes_m == 0) and np.all(st.scale_m == 0)      # packed state untouched
 
 
+def test_full_precision_switch_is_textbook_adabelief():
+    """AdaBelief (Zhuang et al. 2020) written out in binary64 numpy: m = b1 m + (1-b1) g,
+    s = b2 s + (1-b2) (g - m)^2 + eps, p <- p (1 - lr wd) - lr (m / bc1) / (sqrt(s / bc2) + eps).
+    With quantization switched off the oracle's belief mode must follow it."""
+    n, steps = 1000, 12
+    p0, _, _ = rand_inputs(n, 7)
+    lr, wd, eps = 1e-2, 0.1, 1e-10
+    b1, b2 = float(np.float32(0.9)), float(np.float32(0.999))
+    h = oracle.hyper(lr=lr, beta1=0.9, beta2=0.999, eps=eps, weight_decay=wd, belief=1)
+    lr, wd, eps = float(np.float32(lr)), float(np.float32(wd)), float(np.float32(eps))
+    ref, m, sv = p0.astype(np.float64), np.zeros(n), np.zeros(n)
+    p = p0.copy()
+    st = oracle.State(n, 4, 4, 128)
+    m32, v32 = np.zeros(n, np.float32), np.zeros(n, np.float32)
+    for t in range(1, steps + 1):
+        _, gb, gf = rand_inputs(n, 300 + t)
+        g = gf.astype(np.float64)
+        m = b1 * m + (1 - b1) * g
+        sv = b2 * sv + (1 - b2) * (g - m) ** 2 + eps
+        ref = ref * (1 - lr * wd) - lr * (m / (1 - b1 ** t)) / (np.sqrt(sv / (1 - b2 ** t)) + eps)
+        oracle.step(p, gb, st, h, t, m32=m32, v32=v32)
+        assert np.all(np.abs(p - ref) <= 2e-6 * np.abs(ref) + 4e-9 * t), t
+    assert np.allclose(m32, m, rtol=1e-5, atol=1e-9) and np.allclose(v32, sv, rtol=1e-4, atol=1e-16)
+    # and it is not Adam: the same run without the flag ends elsewhere
+    q = p0.copy()
+    m32b, v32b = np.zeros(n, np.float32), np.zeros(n, np.float32)
+    hb = oracle.hyper(lr=lr, beta1=0.9, beta2=0.999, eps=eps, weight_decay=wd)
+    for t in range(1, steps + 1):
+        _, gb, _ = rand_inputs(n, 300 + t)
+        oracle.step(q, gb, st, hb, t, m32=m32b, v32=v32b)
+    assert np.abs(q - p).max() > 1e-4
+
+
 def test_first_step_from_zero_state():
     """From the zero state the EMA sees no quantization: m^ = (1-b1) g, v^ = (1-b2) g^2 and the
     parameter moves by the bias-corrected AdamW step."""
