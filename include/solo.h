@@ -72,6 +72,8 @@ typedef struct {
     int32_t round_m;       /* 0: nearest level (Eq. 1); 1: stochastic rounding (Eq. 5) */
     int32_t round_v;       /* 1: xi ~ U(-1/2,1/2) in Eq. 6; 0: xi = 0 (deterministic) */
     int32_t param_dtype;   /* 0: fp32 parameters; 1: bf16 parameters */
+    int32_t belief;        /* 0: Adam(W); 1: AdaBelief (Sec. 5.2): the unsigned EMA tracks
+                              (g - m^)^2 and eps is added to it at every step */
     uint64_t seed;         /* Philox key of the rounding noise */
 } solo_hyper_t;
 

@@ -124,6 +124,7 @@ void reduce_hyper(const solo_hyper_t* h, int64_t step, int block, StepArgs& a) {
     a.weight_decay = h->weight_decay;
     a.p_quantile = h->p_quantile;
     a.l2 = (!h->adamw && h->weight_decay != 0.0f) ? 1 : 0;
+    a.belief = h->belief ? 1 : 0;
     a.round_m = h->round_m ? 1 : 0;
     a.round_v = h->round_v ? 1 : 0;
     a.param_bf16 = h->param_dtype;

@@ -49,7 +49,7 @@ struct StepArgs {
     int* status;                       // device word: non-zero after a descriptor mismatch
     // hyper-parameters, already reduced to what the kernel multiplies with
     float beta1, beta2, omb1, omb2, step_size, inv_sqrt_bc2, eps, decay, weight_decay, p_quantile;
-    int32_t l2, round_m, round_v, param_bf16, block, k_full;
+    int32_t l2, round_m, round_v, param_bf16, block, k_full, belief;
     uint32_t seed_lo, seed_hi, step32;
     // Philox round keys (seed + r * Weyl constant), r = 0..9: [2r] low word, [2r+1] high word
     uint32_t rk[20];
@@ -359,7 +359,9 @@ __global__ void __launch_bounds__(CTA) solo_step_kernel(const StepArgs a) {
             float mt = s_y[qm] * dm;
             float vt = pow_sm<BV>(a2, qv) * dv;
             mh[i] = __fmaf_rn(a.beta1, mt, a.omb1 * gi);
-            vh[i] = __fmaf_rn(a.beta2, vt, a.omb2 * (gi * gi));
+            const float sig = a.belief ? gi - mh[i] : gi;            // AdaBelief: (g - m^)^2, plus eps
+            vh[i] = __fmaf_rn(a.beta2, vt, a.omb2 * (sig * sig));
+            if (a.belief) vh[i] = vh[i] + a.eps;
             float den = __fmaf_rn(sqrtf(vh[i]), a.inv_sqrt_bc2, a.eps);
             p[i] = __fmaf_rn(-a.step_size, mh[i] / den, p[i] * a.decay);
         }

@@ -27,6 +27,8 @@
 // value and reverses their order.
 #pragma once
 
+#include <type_traits>
+
 #include "solo_device.cuh"
 
 namespace solo {
@@ -359,17 +361,27 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     const char* const tab_m = reinterpret_cast<const char*>(tab + KV);
     const CodeOffsets<BM> om4(cm);
     const CodeOffsets<BV> ov4(cv);
+    // the loop is instantiated twice so that the optimizer variant costs nothing per element
+    auto ema = [&](auto belief_tag) {
+        constexpr bool BELIEF = decltype(belief_tag)::value;
 #pragma unroll
     for (int i = 0; i < EPT; ++i) {
         const float mt = *reinterpret_cast<const float*>(tab_m + om4(i));
         const float vt = *reinterpret_cast<const float*>(tab_v + ov4(i));
         const float gi = g[i];
         mh[i] = __fmaf_rn(a.beta1, mt, a.omb1 * gi);
-        vh[i] = __fmaf_rn(a.beta2, vt, a.omb2 * (gi * gi));
+        if (BELIEF) {                                            // AdaBelief: (g - m^)^2, plus eps
+            const float sig = gi - mh[i];
+            vh[i] = __fmaf_rn(a.beta2, vt, a.omb2 * (sig * sig)) + a.eps;
+        } else {
+            vh[i] = __fmaf_rn(a.beta2, vt, a.omb2 * (gi * gi));
+        }
         const bool valid = FULL || i < nv;
         mx_m_f = fmaxf(mx_m_f, valid ? fabsf(mh[i]) : 0.0f);
         mx_v = max(mx_v, valid ? __float_as_uint(vh[i]) : 0u);
     }
+    };
+    if (a.belief) ema(std::true_type{}); else ema(std::false_type{});
     uint32_t mx_m = __float_as_uint(mx_m_f);
 
     // Adam(W) update of element i and, after every fourth, the store; issued between the
