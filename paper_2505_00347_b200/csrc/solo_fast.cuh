@@ -1,5 +1,5 @@
 // Streamlined fused step for the common configurations: 2/3/4-bit states, blocks of
-// 128 or 256 elements, fp32 parameters, nearest rounding of the first moment, eps >= 1e-12.
+// 64, 128 or 256 elements, fp32 parameters, nearest rounding of the first moment, eps >= 1e-12.
 //
 // Same packed state as the general kernel (solo_device.cuh): every quantity that decides
 // a stored code (EMA values, block scales, p-quantile, base, rounded logarithm) is computed
@@ -15,7 +15,7 @@
 // sequence to a few 1e-7 of the update term, not bit for bit.
 //
 // Work split: a CTA of 256 threads owns a tile of 2048 consecutive elements, a thread
-// eight of them, a block of B elements G = B/8 consecutive lanes (half a warp or a warp).
+// eight of them, a block of B elements G = B/8 consecutive lanes (a quarter, half or whole warp).
 // The per-block scalar work (reciprocals of the scales, base of the logarithmic codebook
 // and its logarithm) is done once per block by the first warp for the whole tile and
 // passed through shared memory.
@@ -24,7 +24,8 @@
 // two halves of a warp are reduced by one minimum and one maximum over a transformed
 // value: all quantities reduced here are non-negative binary32 bit patterns (bit 31
 // clear), so complementing the upper half's values moves them above every lower-half
-// value and reverses their order.
+// value and reverses their order.  For G = 8 the same is done for each pair of groups, the
+// other pair's lanes contributing a neutral value.
 #pragma once
 
 #include <type_traits>
@@ -44,10 +45,10 @@ constexpr uint32_t KEY_MAX = 0x7FFFFFFFu;    // sentinel key: above or equal to 
 
 struct FastShared {
     uint32_t sort[16][CTA];                  // rows 0..6: 2nd..8th smallest key of a thread; rows 7..15: sentinel
-    float tab[CTA / 16][32];                 // per group: K_v second-moment levels, then K_m first-moment levels
-    uint4 xin[2][CTA / 16];                  // per group: bits of Delta_m', Delta_v', x_p
-    float4 xout[2][CTA / 16];                // per group: 1/Delta_m', 1/Delta_v', 1/log2(alpha'), rounding limit
-    uint32_t xflag[2][CTA / 16];             // bit 0: vanishing first moment, bit 1: vanishing second moment
+    float tab[CTA / 8][32];                 // per group: K_v second-moment levels, then K_m first-moment levels
+    uint4 xin[2][CTA / 8];                  // per group: bits of Delta_m', Delta_v', x_p
+    float4 xout[2][CTA / 8];                // per group: 1/Delta_m', 1/Delta_v', 1/log2(alpha'), rounding limit
+    uint32_t xflag[2][CTA / 8];             // bit 0: vanishing first moment, bit 1: vanishing second moment
 };
 
 __device__ __forceinline__ float lg2_approx(float x) {
@@ -113,41 +114,48 @@ __device__ __forceinline__ void philox_rk(uint32_t c0, uint32_t c1, uint32_t c2,
 
 // ---------------------------------------------------------------------------
 // Group collectives on 31-bit values, full-mask instructions only.
-// `hi`: the lane belongs to the upper half of its warp (G = 16 only).
+// `hi`: the lane belongs to the odd group of its pair of groups (G = 16: the upper half of the
+// warp; G = 8: lanes 8..15 and 24..31).  NEUTRAL neither lowers a minimum over the even group's
+// values (bit 31 clear) nor raises a maximum over the odd group's (bit 31 set).
 // ---------------------------------------------------------------------------
+constexpr uint32_t NEUTRAL = 0x7FFFFFFFu;
+
+// min over the even group and max over the odd group of `u`, for the calling lane's pair; returns
+// the one that belongs to the lane's own group
+template <int G>
+__device__ __forceinline__ uint32_t seg_pick(uint32_t u, bool hi) {
+    if constexpr (G == 16) {
+        const uint32_t lo = __reduce_min_sync(0xffffffffu, u);
+        const uint32_t up = __reduce_max_sync(0xffffffffu, u);
+        return hi ? up : lo;
+    } else {
+        static_assert(G == 8, "group of 8, 16 or 32 lanes");
+        const bool pair1 = (threadIdx.x & 16) != 0;
+        const uint32_t ua = pair1 ? NEUTRAL : u, ub = pair1 ? u : NEUTRAL;
+        const uint32_t a_lo = __reduce_min_sync(0xffffffffu, ua), a_up = __reduce_max_sync(0xffffffffu, ua);
+        const uint32_t b_lo = __reduce_min_sync(0xffffffffu, ub), b_up = __reduce_max_sync(0xffffffffu, ub);
+        return pair1 ? (hi ? b_up : b_lo) : (hi ? a_up : a_lo);
+    }
+}
 template <int G>
 __device__ __forceinline__ uint32_t seg_max31(uint32_t x, bool hi) {
     if constexpr (G == 32) {
         return __reduce_max_sync(0xffffffffu, x);
     } else {
-        // lower half: complement of the low 31 bits (order reversed, bit 31 clear);
-        // upper half: bit 31 set.  min = lower half's maximum, max = upper half's maximum.
+        // even group: complement of the low 31 bits (order reversed, bit 31 clear); odd group:
+        // bit 31 set.  min = even group's maximum, max = odd group's maximum.
         const uint32_t c = hi ? 0x80000000u : 0x7FFFFFFFu;
-        const uint32_t u = x ^ c;
-        const uint32_t lo = __reduce_min_sync(0xffffffffu, u);
-        const uint32_t up = __reduce_max_sync(0xffffffffu, u);
-        return (hi ? up : lo) ^ c;
+        return seg_pick<G>(x ^ c, hi) ^ c;
     }
 }
-template <int G>
-__device__ __forceinline__ int seg_sum16(int x, bool hi) {
-    if constexpr (G == 32) {
-        return __reduce_add_sync(0xffffffffu, x);
-    } else {
-        const int s = __reduce_add_sync(0xffffffffu, hi ? x << 16 : x);
-        return hi ? (int)((uint32_t)s >> 16) : s & 0xFFFF;
-    }
-}
-// Minimum of the group's keys in the "v domain": lower half keeps x, upper half holds ~x.
+// Minimum of the group's keys in the "v domain": even group keeps x, odd group holds ~x.
 // Returns the value a lane compares its own v with (equal <=> the lane holds the minimum).
 template <int G>
 __device__ __forceinline__ uint32_t seg_min_v(uint32_t v, bool hi) {
     if constexpr (G == 32) {
         return __reduce_min_sync(0xffffffffu, v);
     } else {
-        const uint32_t lo = __reduce_min_sync(0xffffffffu, v);
-        const uint32_t up = __reduce_max_sync(0xffffffffu, v);
-        return hi ? up : lo;
+        return seg_pick<G>(v, hi);
     }
 }
 
@@ -229,15 +237,24 @@ __device__ __forceinline__ uint32_t select_kth(uint32_t head, const uint32_t* co
     const int lane = threadIdx.x & 31;
     const uint32_t self = 1u << lane;
     const uint32_t upto = self | (self - 1u);
-    const uint32_t le = (G == 16 && hi) ? upto & 0xFFFF0000u : upto;
+    const uint32_t le = G == 32 ? upto : upto & (((1u << G) - 1u) << (lane & ~(G - 1)));
     int off = 0;
     uint32_t ans = 0;
-    if (UNIFORM_K && k == 13) {
+    if (UNIFORM_K && k == 13) {                                  // p = 0.1, block 128
 #pragma unroll
         for (int r = 0; r < 12; ++r) {
             pop_round<G, false>(head, off, col, le, self, hi);
             if (r < EPT) side(r);
         }
+        ans = pop_round<G, false, true>(head, off, col, le, self, hi);
+    } else if (UNIFORM_K && k == 7) {                            // p = 0.1, block 64
+#pragma unroll
+        for (int r = 0; r < 6; ++r) {
+            pop_round<G, false>(head, off, col, le, self, hi);
+            side(r);
+        }
+        side(6);
+        side(7);
         ans = pop_round<G, false, true>(head, off, col, le, self, hi);
     } else {
 #pragma unroll
@@ -279,7 +296,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     constexpr int NG = CTA / G, B = G * EPT;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gl = tid & (G - 1), grp = tid / G;
-    const bool hi = G == 16 && (lane & 16) != 0;
+    const bool hi = G < 32 && (lane & G) != 0;                  // odd group of its pair
     const uint32_t vflip = hi ? 0xFFFFFFFFu : 0u;               // x domain <-> v domain
 
     // validity (all true in a full tile)
@@ -343,8 +360,12 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
         a2[0] = al;
 #pragma unroll
         for (int i = 1; i < BV; ++i) a2[i] = a2[i - 1] * a2[i - 1];
-        if (gl < KV) tab[gl] = pow_sm<BV>(a2, (uint32_t)gl) * dv;
-        if (gl < KM) tab[KV + gl] = s_y[gl] * dm;
+#pragma unroll
+        for (int r0 = 0; r0 < KV; r0 += G)
+            if (r0 + gl < KV) tab[r0 + gl] = pow_sm<BV>(a2, (uint32_t)(r0 + gl)) * dv;
+#pragma unroll
+        for (int r0 = 0; r0 < KM; r0 += G)
+            if (r0 + gl < KM) tab[KV + r0 + gl] = s_y[r0 + gl] * dm;
     }
     __syncwarp();
 
@@ -574,7 +595,7 @@ __global__ void __launch_bounds__(CTA, 4) solo_step_fast_kernel(const StepArgs a
         s_y[i] = a.tables[i];
         if (i < KM - 1) s_mid[i] = a.tables[KM + i];
     }
-    for (int r = 7; r < 16; ++r) s.sort[r][tid] = (G == 16 && (tid & 16)) ? ~KEY_MAX : KEY_MAX;   // sentinels, v domain
+    for (int r = 7; r < 16; ++r) s.sort[r][tid] = (G < 32 && (tid & G)) ? ~KEY_MAX : KEY_MAX;   // sentinels, v domain
     __syncthreads();
 
     // Tile indices fit 32 bits (the host selects this kernel only below 2^31 tiles).  Tiles are

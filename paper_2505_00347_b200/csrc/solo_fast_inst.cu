@@ -12,13 +12,13 @@
 namespace solo {
 
 StepKernel SOLO_CAT(fast_kernel_bm, SOLO_BM)(int bv_index, int block) {
-    static const StepKernel table[3][2] = {
-        {solo_step_fast_kernel<SOLO_BM, 2, 16>, solo_step_fast_kernel<SOLO_BM, 2, 32>},
-        {solo_step_fast_kernel<SOLO_BM, 3, 16>, solo_step_fast_kernel<SOLO_BM, 3, 32>},
-        {solo_step_fast_kernel<SOLO_BM, 4, 16>, solo_step_fast_kernel<SOLO_BM, 4, 32>},
+    static const StepKernel table[3][3] = {
+        {solo_step_fast_kernel<SOLO_BM, 2, 8>, solo_step_fast_kernel<SOLO_BM, 2, 16>, solo_step_fast_kernel<SOLO_BM, 2, 32>},
+        {solo_step_fast_kernel<SOLO_BM, 3, 8>, solo_step_fast_kernel<SOLO_BM, 3, 16>, solo_step_fast_kernel<SOLO_BM, 3, 32>},
+        {solo_step_fast_kernel<SOLO_BM, 4, 8>, solo_step_fast_kernel<SOLO_BM, 4, 16>, solo_step_fast_kernel<SOLO_BM, 4, 32>},
     };
-    if (bv_index < 0 || bv_index > 2 || (block != 128 && block != 256)) return nullptr;
-    return table[bv_index][block == 256 ? 1 : 0];
+    if (bv_index < 0 || bv_index > 2 || (block != 64 && block != 128 && block != 256)) return nullptr;
+    return table[bv_index][block == 64 ? 0 : block == 128 ? 1 : 2];
 }
 
 #if SOLO_BM == 2
