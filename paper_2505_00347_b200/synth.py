@@ -191,20 +191,3 @@ def make_state(sizes, bits_m: int, bits_v: int, block: int, seed: int, device="c
     out["scale_v"] = loguniform(1e-14, 1e-2).masked_fill_(zero, 0.0)
     out["alpha"] = (torch.rand(nb, device=device, generator=g) * 0.78 + 0.2).float().masked_fill_(zero, 0.5)
     return out
-
-
-def pack_codes(codes: np.ndarray, b: int) -> np.ndarray:
-    """[n_blocks, block] integer codes -> bytes; element e takes bits [e*b, e*b+b) of its
-    block's little-endian bit string."""
-    nb, block = codes.shape
-    bitsarr = ((codes[:, :, None].astype(np.uint16) >> np.arange(b, dtype=np.uint16)) & 1)
-    return np.packbits(bitsarr.reshape(nb, block * b).astype(np.uint8), axis=1,
-                       bitorder="little").reshape(-1)
-
-
-def unpack_codes(packed: np.ndarray, b: int, block: int) -> np.ndarray:
-    """Inverse of pack_codes: bytes -> [n_blocks, block] codes."""
-    nb = packed.size // (block * b // 8)
-    bitsarr = np.unpackbits(packed.reshape(nb, -1), axis=1, bitorder="little")
-    bitsarr = bitsarr.reshape(nb, block, b).astype(np.uint16)
-    return (bitsarr << np.arange(b, dtype=np.uint16)).sum(axis=2).astype(np.uint8)

@@ -15,6 +15,24 @@ import oracle
 from paper_2505_00347_b200 import synth
 
 RTOL, ATOL = 1e-6, 1e-9
+
+
+def pack_codes(codes: np.ndarray, b: int) -> np.ndarray:
+    """[n_blocks, block] integer codes -> bytes; element e takes bits [e*b, e*b+b) of its
+    block's little-endian bit string."""
+    nb, block = codes.shape
+    bitsarr = ((codes[:, :, None].astype(np.uint16) >> np.arange(b, dtype=np.uint16)) & 1)
+    return np.packbits(bitsarr.reshape(nb, block * b).astype(np.uint8), axis=1,
+                       bitorder="little").reshape(-1)
+
+
+def unpack_codes(packed: np.ndarray, b: int, block: int) -> np.ndarray:
+    """Inverse of pack_codes: bytes -> [n_blocks, block] codes."""
+    nb = packed.size // (block * b // 8)
+    bitsarr = np.unpackbits(packed.reshape(nb, -1), axis=1, bitorder="little")
+    bitsarr = bitsarr.reshape(nb, block, b).astype(np.uint16)
+    return (bitsarr << np.arange(b, dtype=np.uint16)).sum(axis=2).astype(np.uint8)
+
 KEYS = ("codes_m", "codes_v", "scale_m", "scale_v", "alpha")
 
 
@@ -95,8 +113,8 @@ def compare_states(got: dict, want: dict, flags_per_block, bits_m, bits_v, block
     for key, b, bit in (("codes_m", bits_m, 1), ("codes_v", bits_v, 2)):
         if np.array_equal(got[key], want[key]):
             continue
-        g = synth.unpack_codes(got[key], b, block)
-        w = synth.unpack_codes(want[key], b, block)
+        g = unpack_codes(got[key], b, block)
+        w = unpack_codes(want[key], b, block)
         diff = g != w
         if flags_per_block is None:
             assert not diff.any(), (where, key, int(diff.sum()))

@@ -4,6 +4,7 @@ import numpy as np
 import torch
 
 import oracle
+import parity
 from paper_2505_00347_b200 import synth
 
 
@@ -43,12 +44,12 @@ def test_pack_helper_matches_oracle_layout():
         for block in (64, 128):
             rng = np.random.default_rng(b + block)
             codes = rng.integers(0, 1 << b, size=(3, block), dtype=np.uint8)
-            packed = synth.pack_codes(codes, b)
+            packed = parity.pack_codes(codes, b)
             slot = block * b // 8
             for j in range(3):
                 for e in range(block):
                     assert oracle.get_code(packed[j * slot:], e, b) == codes[j, e]
-            assert np.array_equal(synth.unpack_codes(packed, b, block), codes)
+            assert np.array_equal(parity.unpack_codes(packed, b, block), codes)
     st = synth.make_state((130, 64, 1), 2, 3, 64, seed=1)
     assert st["codes_m"].numel() == (3 + 1 + 1) * 16 and st["codes_v"].numel() == 5 * 24
     assert st["alpha"].numel() == 5 and st["codes_m"].dtype == torch.uint8
