@@ -6,6 +6,7 @@ import torch
 
 import oracle
 from paper_2505_00347_b200 import synth
+import parity
 from parity import run_lockstep
 
 pytestmark = pytest.mark.gpu
@@ -168,3 +169,79 @@ def test_argument_validation():
     assert multi.status() == 1 and float(ps[1].abs().sum()) == 0.0
     st.destroy()
     multi.destroy()
+
+
+def test_full_size_7b_set_sampled_blocks():
+    """The benchmark's workload at its full size (LLaMA-7B-shaped set, 6.74 B parameters, one
+    solo_multi_step launch, the configuration bench.py times), from a seeded random packed state.
+    Blocks are independent, so the oracle recomputes a sample of them one by one: the first and
+    the last block of every tensor plus random blocks, about 4,000 blocks in all."""
+    from paper_2505_00347_b200 import binding as B
+    free, _ = torch.cuda.mem_get_info()
+    if free < 60e9:
+        pytest.skip("needs about 55 GB of free device memory")
+    w = synth.workload(3)
+    bm, bv, block = w.bits_m, w.bits_v, w.block
+    dev = torch.device("cuda")
+    params = [synth.make_param(w, i, device=dev) for i in range(len(w.sizes))]
+    grads = [synth.make_grad(w, i, 1, device=dev) for i in range(len(w.sizes))]
+    st0 = synth.make_state(w.sizes, bm, bv, block, seed=33, device=dev)
+    gstate = B.State(list(w.sizes), bm, bv, block)
+    for key in parity.KEYS:
+        ptr, nbytes = gstate.raw_ptr(key)
+        src = st0[key].contiguous().view(torch.uint8)
+        assert src.numel() == nbytes
+        B._cuda_memcpy(ptr, src.data_ptr(), nbytes, 3)           # device to device
+    # the sample, and copies of its inputs taken before the step
+    rng = np.random.default_rng(5)
+    nblk = [-(-n // block) for n in w.sizes]
+    bstart = np.concatenate([[0], np.cumsum(nblk)])
+    sample = []
+    for t, nb in enumerate(nblk):
+        picks = {0, nb - 1} | set(int(x) for x in rng.integers(0, nb, size=12 if nb > 2 else 0))
+        sample += [(t, j) for j in sorted(picks)]
+    sm, sv = block * bm // 8, block * bv // 8
+    before = []
+    for t, j in sample:
+        lo, hi = j * block, min(w.sizes[t], (j + 1) * block)
+        jb = int(bstart[t]) + j
+        before.append(dict(
+            p=params[t][lo:hi].cpu().numpy().copy(), g=synth.bf16_bits(grads[t][lo:hi]),
+            codes_m=st0["codes_m"][jb * sm:(jb + 1) * sm].cpu().numpy().copy(),
+            codes_v=st0["codes_v"][jb * sv:(jb + 1) * sv].cpu().numpy().copy(),
+            scale_m=st0["scale_m"][jb:jb + 1].cpu().numpy().copy(),
+            scale_v=st0["scale_v"][jb:jb + 1].cpu().numpy().copy(),
+            alpha=st0["alpha"][jb:jb + 1].cpu().numpy().copy()))
+    del st0
+    kw = dict(lr=w.lr, beta1=w.beta1, beta2=w.beta2, weight_decay=w.weight_decay, seed=1234)
+    ho, hg = parity.hyper_pair(**kw)
+    step = 3
+    B.solo_multi_step(B.TensorSet(params, grads, gstate), hg, step)
+    torch.cuda.synchronize()
+    assert gstate.status() == 0
+    ptrs = {k: gstate.raw_ptr(k)[0] for k in parity.KEYS}
+
+    def fetch(key, off, nbytes, dtype):
+        out = torch.empty(nbytes, dtype=torch.uint8)
+        B._cuda_memcpy(out.data_ptr(), ptrs[key] + off, nbytes, 2)
+        return out.numpy().view(dtype)
+
+    worst = 0.0
+    for (t, j), b in zip(sample, before):
+        n = b["p"].size
+        ost = oracle.State(n, bm, bv, block)
+        for k in parity.KEYS:
+            getattr(ost, k)[:] = b[k]
+        p = b["p"].copy()
+        oracle.step(p, b["g"], ost, ho, step, tensor=t, elem_offset=j * block)
+        jb = int(bstart[t]) + j
+        assert np.array_equal(fetch("codes_m", jb * sm, sm, np.uint8), ost.codes_m), (t, j)
+        assert np.array_equal(fetch("codes_v", jb * sv, sv, np.uint8), ost.codes_v), (t, j)
+        for k in ("scale_m", "scale_v", "alpha"):
+            assert np.array_equal(fetch(k, jb * 4, 4, np.uint32), getattr(ost, k).view(np.uint32)), (t, j, k)
+        gp = params[t][j * block: j * block + n].cpu().numpy()
+        err = np.abs(gp.astype(np.float64) - p)
+        assert np.all(err <= parity.RTOL * np.abs(p) + parity.ATOL), (t, j, float(err.max()))
+        worst = max(worst, float(err.max()))
+    print(f"{len(sample)} blocks of {len(w.sizes)} tensors checked, largest parameter difference {worst:.3g}")
+    gstate.destroy()
