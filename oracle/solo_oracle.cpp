@@ -296,6 +296,7 @@ extern "C" {
 struct so_hyper {
     float lr, beta1, beta2, eps, weight_decay;
     float p_quantile;
+    float fixed_alpha;    // in (0,1): keep this base for every block (no quantile); otherwise 0
     int32_t adamw, bias_correction, round_m, round_v, param_dtype;
     int32_t belief;       // 0: Adam(W); 1: AdaBelief (second moment tracks (g - m^)^2 + eps)
     uint64_t seed;
@@ -469,15 +470,22 @@ static void step_blocks(void* param, const uint16_t* grad, int64_t n, int64_t el
         } else {
             scale_v[j] = dv_new;
             const float inv = 1.0f / dv_new;
-            // p-quantile as an order statistic: the k-th smallest, k = max(1, ceil(p n)).
-            int64_t k = (int64_t)std::ceil((double)h->p_quantile * (double)nb);
-            k = std::min<int64_t>(std::max<int64_t>(k, 1), nb);
-            std::copy(vh.begin(), vh.begin() + nb, sorted.begin());
-            std::sort(sorted.begin(), sorted.begin() + nb,
-                      [](float a, float b) { return f2u(a) < f2u(b); });
-            float x_p = sorted[k - 1];
-            float inv_lambda;
-            float al_new = log_base(x_p, inv, Kv, &inv_lambda);
+            float inv_lambda, al_new;
+            if (h->fixed_alpha > 0.0f && h->fixed_alpha < 1.0f) {
+                // standard logarithmic quantization with a fixed base (Sec. 3.2.2, the remark on
+                // alpha = 1/2; the setting of Prop. 3.5)
+                al_new = h->fixed_alpha;
+                inv_lambda = 1.0f / log2_sp(al_new);
+            } else {
+                // p-quantile as an order statistic: the k-th smallest, k = max(1, ceil(p n)).
+                int64_t k = (int64_t)std::ceil((double)h->p_quantile * (double)nb);
+                k = std::min<int64_t>(std::max<int64_t>(k, 1), nb);
+                std::copy(vh.begin(), vh.begin() + nb, sorted.begin());
+                std::sort(sorted.begin(), sorted.begin() + nb,
+                          [](float a, float b) { return f2u(a) < f2u(b); });
+                float x_p = sorted[k - 1];
+                al_new = log_base(x_p, inv, Kv, &inv_lambda);
+            }
             alpha[j] = al_new;
             for (int e = 0; e < nb; ++e) {
                 float r = vh[e] * inv;

@@ -81,6 +81,36 @@ def test_full_precision_switch_is_textbook_adabelief():
     assert np.abs(q - p).max() > 1e-4
 
 
+def test_fixed_base_mode_is_plain_logarithmic_quantization():
+    """fixed_alpha keeps the base (the standard logarithmic quantizer the paper contrasts with,
+    alpha = 1/2, and the setting of Prop. 3.5): every block stores that base and every code is
+    the rounded log_alpha(v^/Delta) + xi, re-derived here in binary64."""
+    n, block, bits = 128 * 5 + 40, 128, 3
+    p, _, _ = rand_inputs(n, 11)
+    st = oracle.State(n, 4, bits, block)
+    for alpha in (0.5, 0.8):
+        h = oracle.hyper(seed=5, fixed_alpha=alpha)
+        for t in (1, 2, 3):
+            _, gb, _ = rand_inputs(n, 40 + t)
+            _, vh, _ = oracle.step(p, gb, st, h, t, want_hat=True)
+            assert np.all(st.alpha == np.float32(alpha))
+            for j in range(st.nblk):
+                sl = slice(j * block, min(n, (j + 1) * block))
+                assert st.scale_v[j] == vh[sl].max()
+                r = vh[sl].astype(np.float64) / float(st.scale_v[j])
+                for e in range(sl.stop - sl.start):
+                    xi = oracle.xi(oracle.philox_draw16(5, t, 0, sl.start + e, 0))
+                    tt = math.log(r[e]) / math.log(float(np.float32(alpha))) + xi if r[e] > 0 else 99
+                    q_ref = int(min(max(round(tt), 0), (1 << bits) - 1))
+                    q = oracle.get_code(st.codes_v[j * (block * bits // 8):], e, bits)
+                    assert q == q_ref or abs(tt - math.floor(tt) - 0.5) < 2e-4, (alpha, t, j, e, tt, q)
+    # the quantile mode chooses its own base: a different state from the same inputs
+    st2 = oracle.State(n, 4, bits, block)
+    _, gb, _ = rand_inputs(n, 41)
+    oracle.step(p.copy(), gb, st2, oracle.hyper(seed=5), 1)
+    assert not np.all(st2.alpha == np.float32(0.8))
+
+
 def test_first_step_from_zero_state():
     """From the zero state the EMA sees no quantization: m^ = (1-b1) g, v^ = (1-b2) g^2 and the
     parameter moves by the bias-corrected AdamW step."""
