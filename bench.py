@@ -141,7 +141,8 @@ def run_ours(args, rank, world):
     B.set_kernel_policy(args.policy)
     state = B.State(list(w.sizes), w.bits_m, w.bits_v, w.block)
     ts = B.TensorSet(params, grads, state)
-    h = B.hyper(lr=w.lr, beta1=w.beta1, beta2=w.beta2, weight_decay=w.weight_decay, seed=1234)
+    h = B.hyper(lr=w.lr, beta1=w.beta1, beta2=w.beta2, weight_decay=w.weight_decay, seed=1234,
+                fixed_alpha=args.fixed_alpha)
     n = w.numel
     step_no = 0
 
@@ -209,7 +210,8 @@ def run_ours(args, rank, world):
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"{w.name}: {len(w.sizes)} tensors, {n} params, m {w.bits_m}-bit / v {w.bits_v}-bit, "
-                               f"block {w.block}, fp32 params, bf16 grads, one solo_multi_step launch per step",
+                               f"block {w.block}, fp32 params, bf16 grads, one solo_multi_step launch per step"
+                               + (f", fixed base {args.fixed_alpha}" if args.fixed_alpha else ""),
                    "l2": "working set (params+grads+state) far larger than the 126 MB L2; no flush needed"
                          if n * abytes > 1e9 else "working set fits L2: launch-bound point, not a bandwidth point",
                    "bytes_per_param": round(abytes, 4)},
@@ -297,6 +299,8 @@ def main():
     ap.add_argument("--bits-m", type=int, default=0, help="override the workload's first-moment width")
     ap.add_argument("--bits-v", type=int, default=0, help="override the workload's second-moment width")
     ap.add_argument("--block", type=int, default=0, help="override the workload's block size")
+    ap.add_argument("--fixed-alpha", type=float, default=0.0,
+                    help="fixed base of the logarithmic codebook (no quantile step); 0 = the paper's quantile rule")
     ap.add_argument("--cpu-sample", type=int, default=1 << 27)
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--policy", type=int, default=0, help="kernel policy: 0 streamlined where it applies, 1 general")

@@ -67,6 +67,8 @@ typedef struct {
     float eps;
     float weight_decay;
     float p_quantile;      /* p of the base alpha = (x_p/Delta)^(1/(2^b-1)); 0.1 in the paper; [0,1) */
+    float fixed_alpha;     /* in (0,1): every block keeps this base (standard logarithmic quantization,
+                              e.g. 1/2; Sec. 3.2.2, Prop. 3.5) and no quantile is taken; else 0 */
     int32_t adamw;         /* 1: decoupled decay (AdamW); 0: decay added to the gradient (Adam) */
     int32_t bias_correction; /* 1: divide by 1-beta^t; 0: no correction */
     int32_t round_m;       /* 0: nearest level (Eq. 1); 1: stochastic rounding (Eq. 5) */

@@ -102,7 +102,7 @@ int sm_count(int device) {
 int check_hyper(const solo_hyper_t* h, int64_t step) {
     if (!h || step < 1) return SOLO_EINVAL;
     auto unit = [](float b) { return b >= 0.0f && b < 1.0f; };
-    if (!unit(h->beta1) || !unit(h->beta2) || !unit(h->p_quantile)) return SOLO_EINVAL;
+    if (!unit(h->beta1) || !unit(h->beta2) || !unit(h->p_quantile) || !unit(h->fixed_alpha)) return SOLO_EINVAL;
     if (!(h->eps >= 0.0f) || !std::isfinite(h->lr) || !std::isfinite(h->weight_decay)) return SOLO_EINVAL;
     if (h->param_dtype != 0 && h->param_dtype != 1) return SOLO_EINVAL;
     return SOLO_OK;
@@ -123,6 +123,7 @@ void reduce_hyper(const solo_hyper_t* h, int64_t step, int block, StepArgs& a) {
     a.decay = h->adamw ? (float)(1.0 - (double)h->lr * (double)h->weight_decay) : 1.0f;
     a.weight_decay = h->weight_decay;
     a.p_quantile = h->p_quantile;
+    a.fixed_alpha = (h->fixed_alpha > 0.0f && h->fixed_alpha < 1.0f) ? h->fixed_alpha : 0.0f;
     a.l2 = (!h->adamw && h->weight_decay != 0.0f) ? 1 : 0;
     a.belief = h->belief ? 1 : 0;
     a.round_m = h->round_m ? 1 : 0;

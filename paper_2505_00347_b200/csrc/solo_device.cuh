@@ -49,6 +49,7 @@ struct StepArgs {
     int* status;                       // device word: non-zero after a descriptor mismatch
     // hyper-parameters, already reduced to what the kernel multiplies with
     float beta1, beta2, omb1, omb2, step_size, inv_sqrt_bc2, eps, decay, weight_decay, p_quantile;
+    float fixed_alpha;                 // in (0,1): base of every block; 0: base from the p-quantile
     int32_t l2, round_m, round_v, param_bf16, block, k_full, belief;
     uint32_t seed_lo, seed_hi, step32;
     // Philox round keys (seed + r * Weyl constant), r = 0..9: [2r] low word, [2r+1] high word
@@ -446,11 +447,15 @@ __global__ void __launch_bounds__(CTA) solo_step_kernel(const StepArgs a) {
                 k = (int)ceil((double)a.p_quantile * (double)nb);
                 k = min(max(k, 1), nb);
             }
-            const float x_p = __uint_as_float(group_select<CTA_GROUP>(key, k, mask, s_sort, s_hist));
             const float inv = 1.0f / dv_new;
-            float rho = fminf(fmaxf(x_p * inv, RHO_MIN), RHO_MAX);
-            const float lam = log2_sp(rho) * (1.0f / (float)(KV - 1));
-            al_new = exp2_sp(lam);
+            if (a.fixed_alpha > 0.0f) {                          // uniform: fixed base, no quantile
+                al_new = a.fixed_alpha;
+            } else {
+                const float x_p = __uint_as_float(group_select<CTA_GROUP>(key, k, mask, s_sort, s_hist));
+                float rho = fminf(fmaxf(x_p * inv, RHO_MIN), RHO_MAX);
+                const float lam = log2_sp(rho) * (1.0f / (float)(KV - 1));
+                al_new = exp2_sp(lam);
+            }
             const float inv_lambda = 1.0f / log2_sp(al_new);
             uint32_t wv[4];
             if (a.round_v) {

@@ -424,8 +424,11 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     // ---- block scales and the p-quantile of v^ (Sec. 3.2.2) ----
     mx_m = seg_max31<G>(mx_m, hi);
     mx_v = seg_max31<G>(mx_v, hi);
-    uint32_t x_p;
-    {
+    uint32_t x_p = 0;
+    if (a.fixed_alpha > 0.0f) {                                  // fixed base: no quantile to find
+#pragma unroll
+        for (int i = 0; i < EPT; ++i) update(i);
+    } else {
         uint32_t key[EPT];
 #pragma unroll
         for (int i = 0; i < EPT; ++i) key[i] = (FULL || i < nv) ? __float_as_uint(vh[i]) : KEY_MAX;
@@ -460,7 +463,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
         const float inv_dv = 1.0f / dv_new;
         const float rho = fminf(fmaxf(__uint_as_float(in.z) * inv_dv, RHO_MIN), RHO_MAX);
         const float lam = log2_sp(rho) * (1.0f / (float)(KV - 1));
-        const float al_new = exp2_sp(lam);
+        const float al_new = a.fixed_alpha > 0.0f ? a.fixed_alpha : exp2_sp(lam);
         const float inv_lambda = 1.0f / log2_sp(al_new);
         const float guard = __fmaf_rn(fabsf(inv_lambda), LG2_ABS, LG2_REL * (float)(KV + 1));
         s.xout[par][tid] = make_float4(inv_dm, inv_dv, inv_lambda, 0.5f - guard);

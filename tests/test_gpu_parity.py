@@ -53,6 +53,8 @@ def test_bits_and_blocks_random_state(bits_m, bits_v, block):
     dict(param_dtype=1, lr=1e-2),
     dict(eps=1e-3, lr=0.1, weight_decay=0.0),
     dict(belief=1),
+    dict(fixed_alpha=0.5),
+    dict(fixed_alpha=0.9, round_v=0),
     dict(belief=1, eps=1e-12, beta2=0.99, adamw=0, weight_decay=0.05),
 ])
 def test_hyper_parameter_modes(hk):
