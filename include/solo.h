@@ -204,7 +204,9 @@ int solo_debug_check_fast_log(uint32_t lo_bits, uint32_t hi_bits, float* max_exc
  * solo_multi_step_static.  Same layout as the library's own state (see the top of this
  * file): with n_blk = sum over tensors of ceil(numel / block),
  *   codes_m  n_blk * block * bits_m / 8 bytes     codes_v  n_blk * block * bits_v / 8 bytes
- *   scale_m, scale_v, alpha  n_blk floats each
+ *            (each followed by 16 bytes that may be read, never written)
+ *   scale_m, scale_v, alpha  n_blk floats each, allocated as a multiple of 16 bytes (round
+ *                            n_blk up to a multiple of 4; the padding is read, never written)
  * every buffer 16-byte aligned.  A fresh state is all-zero codes and scales and alpha = 0.5.
  */
 typedef struct {

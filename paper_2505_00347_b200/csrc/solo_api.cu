@@ -147,13 +147,14 @@ int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
     if (g_policy.load(std::memory_order_relaxed) == 0 && !a.round_m && !a.param_bf16 && a.eps >= 1e-12f &&
         s->tiles_total < (int64_t)1 << 31)
         k = solo::fast_kernel(s->bits_m, s->bits_v, s->block);
+    size_t dyn_smem = k ? solo::fast_kernel_smem() : 0;
     if (!k) k = solo::step_kernel(s->bits_m, s->bits_v, cta_group);
     if (!k) return SOLO_EINVAL;
-    int per_sm = solo::kernel_occupancy(k);
+    int per_sm = solo::kernel_occupancy(k, dyn_smem);
     if (per_sm <= 0) return SOLO_ECUDA;
     int64_t grid = std::min<int64_t>(s->tiles_total, (int64_t)sm_count(s->device) * per_sm);
     void* params[] = {(void*)&a};
-    cudaError_t e = cudaLaunchKernel((const void*)k, dim3((unsigned)grid), dim3(solo::CTA), params, 0, stream);
+    cudaError_t e = cudaLaunchKernel((const void*)k, dim3((unsigned)grid), dim3(solo::CTA), params, dyn_smem, stream);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return SOLO_ECUDA;
@@ -270,13 +271,16 @@ int solo_state_create_multi(const int64_t* numel_host, int num_tensors, int bits
     auto alloc = [&](void** p, size_t bytes) {
         if (ok && cudaMalloc(p, bytes ? bytes : 1) != cudaSuccess) { ok = false; cudaGetLastError(); }
     };
-    // +8 bytes of slack after the codes so that the widest per-thread access of a
-    // block's last slot never leaves the allocation
-    alloc((void**)&s->codes_m, s->bytes_codes_m + 8);
-    alloc((void**)&s->codes_v, s->bytes_codes_v + 8);
-    alloc((void**)&s->scale_m, (size_t)s->nblk_total * 4);
-    alloc((void**)&s->scale_v, (size_t)s->nblk_total * 4);
-    alloc((void**)&s->alpha, (size_t)s->nblk_total * 4);
+    // 16 bytes of slack after the codes: the streamlined kernel copies a tile's codes in
+    // 16-byte pieces starting at the 16-byte boundary at or below them
+    alloc((void**)&s->codes_m, s->bytes_codes_m + 16);
+    alloc((void**)&s->codes_v, s->bytes_codes_v + 16);
+    // the three per-block arrays are allocated in multiples of 16 bytes (the streamlined kernel
+    // copies them in 16-byte pieces)
+    const size_t scal_bytes = ((size_t)s->nblk_total + 3) / 4 * 16;
+    alloc((void**)&s->scale_m, scal_bytes);
+    alloc((void**)&s->scale_v, scal_bytes);
+    alloc((void**)&s->alpha, scal_bytes);
     alloc((void**)&s->geom, geom.size() * 8);
     alloc((void**)&s->tables_m, tm.size() * 4);
     alloc((void**)&s->tables_v, tv.size() * 4);
@@ -284,10 +288,11 @@ int solo_state_create_multi(const int64_t* numel_host, int num_tensors, int bits
     if (!ok) { solo_state_destroy(s); return SOLO_ENOMEM; }
     cudaError_t e = cudaSuccess;
     auto chk = [&](cudaError_t r) { if (e == cudaSuccess) e = r; };
-    chk(cudaMemset(s->codes_m, 0, s->bytes_codes_m + 8));
-    chk(cudaMemset(s->codes_v, 0, s->bytes_codes_v + 8));
-    chk(cudaMemset(s->scale_m, 0, (size_t)s->nblk_total * 4));
-    chk(cudaMemset(s->scale_v, 0, (size_t)s->nblk_total * 4));
+    chk(cudaMemset(s->codes_m, 0, s->bytes_codes_m + 16));
+    chk(cudaMemset(s->codes_v, 0, s->bytes_codes_v + 16));
+    chk(cudaMemset(s->scale_m, 0, scal_bytes));
+    chk(cudaMemset(s->scale_v, 0, scal_bytes));
+    chk(cudaMemset(s->alpha, 0, scal_bytes));
     chk(cudaMemset(s->status, 0, 4));
     chk(cudaMemcpy(s->geom, geom.data(), geom.size() * 8, cudaMemcpyHostToDevice));
     chk(cudaMemcpy(s->tables_m, tm.data(), tm.size() * 4, cudaMemcpyHostToDevice));

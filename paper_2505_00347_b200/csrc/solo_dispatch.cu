@@ -2,6 +2,7 @@
 #include "solo_dispatch.h"
 
 #include <map>
+#include <utility>
 #include <mutex>
 
 namespace solo {
@@ -28,19 +29,27 @@ StepKernel fast_kernel(int bits_m, int bits_v, int block) {
     }
 }
 
-int kernel_occupancy(StepKernel k) {
+int kernel_occupancy(StepKernel k, size_t dyn_smem) {
     static std::mutex mu;
-    static std::map<const void*, int> cache;
+    static std::map<std::pair<int, const void*>, int> cache;    // per device: the opt-in below is per context
     if (!k) return 0;
-    std::lock_guard<std::mutex> lk(mu);
-    auto it = cache.find((const void*)k);
-    if (it != cache.end()) return it->second;
-    int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k, CTA, 0) != cudaSuccess || n <= 0) {
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
-    cache[(const void*)k] = n;
+    std::lock_guard<std::mutex> lk(mu);
+    const auto key = std::make_pair(device, (const void*)k);
+    auto it = cache.find(key);
+    if (it != cache.end()) return it->second;
+    int n = 0;
+    if ((dyn_smem > 0 &&
+         cudaFuncSetAttribute((const void*)k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem) != cudaSuccess) ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k, CTA, dyn_smem) != cudaSuccess || n <= 0) {
+        cudaGetLastError();
+        return 0;
+    }
+    cache[key] = n;
     return n;
 }
 

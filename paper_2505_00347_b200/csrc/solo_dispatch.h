@@ -35,8 +35,11 @@ StepKernel fast_kernel_bm2(int bv_index, int block);
 StepKernel fast_kernel_bm3(int bv_index, int block);
 StepKernel fast_kernel_bm4(int bv_index, int block);
 StepKernel fast_kernel(int bits_m, int bits_v, int block);
-// Resident CTAs per SM of a step kernel (cached per kernel), 0 on error.
-int kernel_occupancy(StepKernel k);
+// Dynamic shared memory the streamlined kernels are launched with.
+size_t fast_kernel_smem();
+// Resident CTAs per SM of a step kernel launched with `dyn_smem` bytes of dynamic shared memory
+// (cached per device and kernel; opts the kernel in to that much shared memory), 0 on error.
+int kernel_occupancy(StepKernel k, size_t dyn_smem);
 
 // Exhaustive comparison of the hardware lg2 approximation with log2_sp (tests).
 cudaError_t launch_fast_log_check(uint32_t lo, uint32_t hi, float* out_max_excess, cudaStream_t stream);

@@ -49,7 +49,44 @@ struct FastShared {
     uint4 xin[2][CTA / 8];                  // per group: bits of Delta_m', Delta_v', x_p
     float4 xout[2][CTA / 8];                // per group: 1/Delta_m', 1/Delta_v', 1/log2(alpha'), rounding limit
     uint32_t xflag[2][CTA / 8];             // bit 0: vanishing first moment, bit 1: vanishing second moment
+    // Two stages for the inputs of a full tile, filled by bulk asynchronous copies (TMA, issued by
+    // one thread) one tile ahead of their use; each stage has its own mbarrier.
+    struct Stage {
+        float4 p[2 * CTA];                   // 2048 parameters
+        uint4 g[CTA];                        // 2048 bf16 gradients
+        uint32_t cm[CTA + 4];                // packed codes of the tile, from a 16-byte boundary (64 * bits words + 2)
+        uint32_t cv[CTA + 4];
+        float sc[3][CTA / 8 + 4];            // Delta_m, Delta_v, alpha of the tile's blocks, from a 16-byte boundary
+    };
+    alignas(16) Stage stage[2];
+    alignas(8) unsigned long long mbar[2];
 };
+
+// What a CTA carries from one tile to the next for the copy-ahead of inputs.
+struct Ahead {
+    uint32_t fill = 0;        // number of the next bulk copy to wait for (uniform over the CTA)
+    bool staged = false;      // that copy has already been issued (uniform)
+    bool failed = false;      // this thread once waited in vain for a copy
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// Waits until the phase with the given parity of an mbarrier has completed.  Bounded: gives up
+// (returns false) after 2^14 timed-out polls instead of spinning for ever.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (int it = 0; it < (1 << 14); ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void bulk_copy(void* smem_dst, const void* gmem_src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(bar) : "memory");
+}
 
 __device__ __forceinline__ float lg2_approx(float x) {
     float y;
@@ -177,6 +214,42 @@ __device__ __forceinline__ uint32_t warp_load_codes(const uint8_t* warp_base, in
         return __funnelshift_r(lo, hi, o) & 0xFFFFFFu;
     }
 }
+// Issues (one thread) the bulk copies of one full tile's inputs into stage `fill & 1`: parameters,
+// gradients, the packed codes of its blocks and their three per-block scalars.  Bulk copies need
+// 16-byte aligned addresses and sizes: codes (8 bytes off for 3-bit codes in blocks of 64 when the
+// first block is odd) and scalars are copied from the 16-byte boundary at or below them, with 16
+// bytes more when they do not start on it; readers add the offset.  The scalar arrays are
+// allocated in multiples of 16 bytes, so the copy never leaves them.
+template <int BM, int BV, int G>
+__device__ __forceinline__ void issue_tile_copy(const StepArgs& a, FastShared& s, uint32_t fill, const char* pt,
+                                                const char* gt, int64_t jb_tile) {
+    constexpr int NG = CTA / G;
+    FastShared::Stage& st = s.stage[fill & 1u];
+    const uint32_t bar = smem_u32(&s.mbar[fill & 1u]);
+    const int64_t bm0 = jb_tile * G * BM, bv0 = jb_tile * G * BV;   // byte offsets of the tile's codes
+    const uint32_t bytes_m = CTA * BM + ((bm0 & 15) ? 16u : 0u), bytes_v = CTA * BV + ((bv0 & 15) ? 16u : 0u);
+    const uint32_t bytes_s = (NG + ((jb_tile & 3) ? 4u : 0u)) * 4u;
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar),
+                 "r"((uint32_t)(TILE * 4 + TILE * 2) + bytes_m + bytes_v + 3u * bytes_s) : "memory");
+    bulk_copy(st.p, pt, TILE * 4, bar);
+    bulk_copy(st.g, gt, TILE * 2, bar);
+    bulk_copy(st.cm, a.codes_m + (bm0 & ~(int64_t)15), bytes_m, bar);
+    bulk_copy(st.cv, a.codes_v + (bv0 & ~(int64_t)15), bytes_v, bar);
+    const int64_t j0 = jb_tile & ~(int64_t)3;
+    bulk_copy(st.sc[0], a.scale_m + j0, bytes_s, bar);
+    bulk_copy(st.sc[1], a.scale_v + j0, bytes_s, bar);
+    bulk_copy(st.sc[2], a.alpha + j0, bytes_s, bar);
+}
+
+// From the warp's packed words (lane < 24 holds word `lane`) to the thread's own 3-bit codes.
+template <int BITS>
+__device__ __forceinline__ uint32_t warp_codes_finish(uint32_t w, int lane) {
+    static_assert(BITS == 3, "only the 3-bit layout needs the exchange");
+    const int a = (3 * lane) >> 2, o = ((3 * lane) & 3) * 8;
+    const uint32_t lo = __shfl_sync(0xffffffffu, w, a);
+    const uint32_t hi = __shfl_sync(0xffffffffu, w, (a + 1) & 31);
+    return __funnelshift_r(lo, hi, o) & 0xFFFFFFu;
+}
 template <int BITS>
 __device__ __forceinline__ void warp_store_codes(uint8_t* warp_base, int lane, uint32_t c) {
     if constexpr (BITS == 2) {
@@ -291,7 +364,8 @@ template <int BM, int BV, int G, bool FULL>
 __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, const float* s_y,
                                           const float* s_mid, char* pbase, const char* gbase,
                                           const int64_t n, const int tin, const int64_t jb_tile,
-                                          const int tensor, const int par) {
+                                          const int tensor, const int par, Ahead& ah, const bool next_full,
+                                          const int next_dtin) {
     constexpr int KM = 1 << BM, KV = 1 << BV;
     constexpr int NG = CTA / G, B = G * EPT;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -319,9 +393,39 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     uint32_t cm = 0, cv = 0;
     float dm = 0.0f, dv = 0.0f, al = 0.5f;
     if (FULL) {
-        const uint4 gw = __ldcs(reinterpret_cast<const uint4*>(gt) + tid);
-        const float4 p0 = __ldcs(reinterpret_cast<const float4*>(pt) + 2 * tid);
-        const float4 p1 = __ldcs(reinterpret_cast<const float4*>(pt) + 2 * tid + 1);
+        // Every full tile reads its inputs from a stage.  Copy number f uses stage f & 1 and
+        // completes phase f >> 1 of that stage's mbarrier.  The copy for this tile was issued
+        // while the tile before it was worked on (ah.staged), or is issued now (first full tile
+        // after a tensor change); the copy for the next tile is issued here.  Before a stage is
+        // refilled all threads have finished reading it: they read at the start of a tile and
+        // pass that tile's barriers before any thread starts the next one.
+        if (tid == 0) {
+            if (!ah.staged) issue_tile_copy<BM, BV, G>(a, s, ah.fill, pt, gt, jb_tile);
+            if (next_full)
+                issue_tile_copy<BM, BV, G>(a, s, ah.fill + 1u, pt + (int64_t)next_dtin * (TILE * 4),
+                                           gt + (int64_t)next_dtin * (TILE * 2), jb_tile + (int64_t)next_dtin * NG);
+        }
+        const uint32_t mine = ah.fill;
+        ah.fill += 1u;
+        ah.staged = next_full;
+        if (!mbar_wait(smem_u32(&s.mbar[mine & 1u]), (mine >> 1) & 1u)) {
+            // the copy was never seen to arrive: flag it; what the stage holds is used as it is
+            // (the step's results are then undefined, solo_state_status reports bit 1)
+            atomicOr(a.status, 2);
+            ah.failed = true;
+        }
+        const FastShared::Stage& st = s.stage[mine & 1u];
+        const uint4 gw = st.g[tid];
+        const float4 p0 = st.p[2 * tid], p1 = st.p[2 * tid + 1];
+        const int wm = (int)((jb_tile * G * BM) & 15) >> 2, wv = (int)((jb_tile * G * BV) & 15) >> 2;   // word offsets
+        if constexpr (BM == 2) cm = reinterpret_cast<const uint16_t*>(st.cm + wm)[tid];
+        else if constexpr (BM == 4) cm = st.cm[wm + tid];
+        else cm = warp_codes_finish<BM>(lane < 24 ? st.cm[wm + warp * 24 + lane] : 0u, lane);
+        if constexpr (BV == 2) cv = reinterpret_cast<const uint16_t*>(st.cv + wv)[tid];
+        else if constexpr (BV == 4) cv = st.cv[wv + tid];
+        else cv = warp_codes_finish<BV>(lane < 24 ? st.cv[wv + warp * 24 + lane] : 0u, lane);
+        const int so = (int)(jb_tile & 3) + grp;                 // the scalars were copied from a 16-byte boundary
+        dm = st.sc[0][so]; dv = st.sc[1][so]; al = st.sc[2][so];
         const uint32_t gg[4] = {gw.x, gw.y, gw.z, gw.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -330,11 +434,6 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
         }
         p[0] = p0.x; p[1] = p0.y; p[2] = p0.z; p[3] = p0.w;
         p[4] = p1.x; p[5] = p1.y; p[6] = p1.z; p[7] = p1.w;
-        cm = warp_load_codes<BM>(wcm, lane);
-        cv = warp_load_codes<BV>(wcv, lane);
-        dm = __ldg(a.scale_m + jb);
-        dv = __ldg(a.scale_v + jb);
-        al = __ldg(a.alpha + jb);
     } else {
 #pragma unroll
         for (int i = 0; i < EPT; ++i) {
@@ -590,7 +689,8 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
 template <int BM, int BV, int G>
 __global__ void __launch_bounds__(CTA, 4) solo_step_fast_kernel(const StepArgs a) {
     constexpr int KM = 1 << BM;
-    __shared__ FastShared s;
+    extern __shared__ __align__(16) unsigned char fast_smem[];   // sizeof(FastShared), above the static 48 KB limit
+    FastShared& s = *reinterpret_cast<FastShared*>(fast_smem);
     __shared__ float s_y[KM];
     __shared__ float s_mid[KM];
     const int tid = threadIdx.x;
@@ -599,6 +699,11 @@ __global__ void __launch_bounds__(CTA, 4) solo_step_fast_kernel(const StepArgs a
         if (i < KM - 1) s_mid[i] = a.tables[KM + i];
     }
     for (int r = 7; r < 16; ++r) s.sort[r][tid] = (G < 32 && (tid & G)) ? ~KEY_MAX : KEY_MAX;   // sentinels, v domain
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s.mbar[0])) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s.mbar[1])) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
     __syncthreads();
 
     // Tile indices fit 32 bits (the host selects this kernel only below 2^31 tiles).  Tiles are
@@ -610,6 +715,7 @@ __global__ void __launch_bounds__(CTA, 4) solo_step_fast_kernel(const StepArgs a
     char* pbase = nullptr;
     const char* gbase = nullptr;
     bool skip = false;
+    Ahead ah;
     int par = 0;
     for (int tile = blockIdx.x; tile < total_tiles; tile += stride) {
         if (tile >= t_hi) {
@@ -631,10 +737,17 @@ __global__ void __launch_bounds__(CTA, 4) solo_step_fast_kernel(const StepArgs a
         const int tin = tile - t_lo;
         const int64_t jb_tile = jb0 + (int64_t)tin * (CTA / G);
         if (tin < full_tiles)
-            fast_tile<BM, BV, G, true>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par);
+            fast_tile<BM, BV, G, true>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, ah,
+                                       tin + stride < full_tiles, stride);
         else
-            fast_tile<BM, BV, G, false>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par);
+            fast_tile<BM, BV, G, false>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, ah, false, 0);
         par ^= 1;
+    }
+    // every copy that was issued has been waited for by the thread that issued it, unless that
+    // thread gave up once: then it waits (bounded) once more for its last copy before the CTA exits
+    if (tid == 0 && ah.failed && ah.fill > 0) {
+        const uint32_t last = ah.fill - 1u;
+        mbar_wait(smem_u32(&s.mbar[last & 1u]), (last >> 1) & 1u);
     }
 }
 

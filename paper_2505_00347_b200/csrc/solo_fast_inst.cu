@@ -49,6 +49,7 @@ cudaError_t launch_fast_log_check(uint32_t lo, uint32_t hi, float* out_max_exces
     return cudaGetLastError();
 }
 float fast_log_abs_bound() { return LG2_ABS; }
+size_t fast_kernel_smem() { return sizeof(FastShared); }
 #endif
 
 }  // namespace solo

@@ -18,16 +18,32 @@ from paper_2505_00347_b200 import synth
 pytestmark = pytest.mark.gpu
 
 
+def pad4(n: int) -> int:
+    return (n + 3) // 4 * 4
+
+
 def _fresh_buffers(sizes, bits_m, bits_v, block, state0=None):
     nb = sum(-(-int(n) // block) for n in sizes)
     if state0 is not None:
-        return {k: v.clone().cuda() for k, v in state0.items()}
+        out = {}
+        for k, v in state0.items():
+            if v.dtype == torch.float32:                        # per-block arrays: padded allocation
+                buf = torch.zeros(pad4(v.numel()), dtype=torch.float32, device="cuda")
+                buf[: v.numel()] = v.cuda()
+                out[k] = buf[: v.numel()]
+            else:                                                # codes: 16 readable bytes follow
+                buf = torch.zeros(v.numel() + 16, dtype=torch.uint8, device="cuda")
+                buf[: v.numel()] = v.cuda()
+                out[k] = buf[: v.numel()]
+        return out
     return {
-        "codes_m": torch.zeros(nb * block * bits_m // 8, dtype=torch.uint8, device="cuda"),
-        "codes_v": torch.zeros(nb * block * bits_v // 8, dtype=torch.uint8, device="cuda"),
-        "scale_m": torch.zeros(nb, dtype=torch.float32, device="cuda"),
-        "scale_v": torch.zeros(nb, dtype=torch.float32, device="cuda"),
-        "alpha": torch.full((nb,), 0.5, dtype=torch.float32, device="cuda"),
+        # 16 readable bytes follow the codes
+        "codes_m": torch.zeros(nb * block * bits_m // 8 + 16, dtype=torch.uint8, device="cuda")[:nb * block * bits_m // 8],
+        "codes_v": torch.zeros(nb * block * bits_v // 8 + 16, dtype=torch.uint8, device="cuda")[:nb * block * bits_v // 8],
+        # the three per-block arrays are allocated in multiples of 16 bytes
+        "scale_m": torch.zeros(pad4(nb), dtype=torch.float32, device="cuda")[:nb],
+        "scale_v": torch.zeros(pad4(nb), dtype=torch.float32, device="cuda")[:nb],
+        "alpha": torch.full((pad4(nb),), 0.5, dtype=torch.float32, device="cuda")[:nb],
     }
 
 
