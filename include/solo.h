@@ -160,9 +160,12 @@ int solo_state_info(const solo_state_t* state, int64_t* numel, int64_t* num_bloc
                     int32_t* num_tensors, int32_t* bits_m, int32_t* bits_v, int32_t* block);
 
 /*
- * Reads the state's device status word into *status_out (0 = no problem seen;
- * bit 0 = a solo_multi_step descriptor's numel disagreed with the state and the
- * affected tensors were skipped).  Synchronizes the device.
+ * Reads the state's device status word into *status_out (0 = no problem seen).
+ *   bit 0  a solo_multi_step descriptor's numel disagreed with the state; the affected
+ *          tensors were skipped
+ *   bit 1  the streamlined kernel gave up waiting for an asynchronous copy of its inputs
+ *          (a bounded wait, so the kernel always ends); the results of that step are undefined
+ * Synchronizes the device.
  */
 int solo_state_status(solo_state_t* state, int* status_out);
 
