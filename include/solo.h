@@ -59,6 +59,14 @@ typedef enum {
 
 typedef struct solo_state solo_state_t; /* opaque; owns its device buffers */
 
+/* Quantizers of the unsigned (second-moment) state; Appendix A gives the codebooks. */
+enum {
+    SOLO_V_LOG = 0,           /* levels alpha^k with the per-block base of Sec. 3.2.2 (SOLO) */
+    SOLO_V_DE = 1,            /* unsigned dynamic exponent */
+    SOLO_V_LINEAR = 2,        /* {0, 1/(2^b-1), ..., 1} */
+    SOLO_V_LINEAR_NOZERO = 3  /* {1/2^b, ..., 1} */
+};
+
 /* Hyper-parameters of one step; plain data, read at the call and not retained. */
 typedef struct {
     float lr;
@@ -76,6 +84,14 @@ typedef struct {
     int32_t param_dtype;   /* 0: fp32 parameters; 1: bf16 parameters */
     int32_t belief;        /* 0: Adam(W); 1: AdaBelief (Sec. 5.2): the unsigned EMA tracks
                               (g - m^)^2 and eps is added to it at every step */
+    int32_t param_round;   /* bf16 parameters: 0 round to nearest even; 1 stochastic rounding with
+                              the element's Philox draw (purpose 2).  No counterpart in the paper,
+                              whose 16-bit baseline is plain BF16 (Sec. 5, "Baselines") */
+    int32_t v_codebook;    /* quantizer of the unsigned state: SOLO_V_LOG (Eq. 6, the paper's), or
+                              one of the baselines of Sec. 5 (block-wise absmax scaling, nearest
+                              level of a fixed codebook, Eq. 1): SOLO_V_DE, SOLO_V_LINEAR,
+                              SOLO_V_LINEAR_NOZERO.  A state must be stepped and dequantized
+                              with the selector it was written with */
     uint64_t seed;         /* Philox key of the rounding noise */
 } solo_hyper_t;
 

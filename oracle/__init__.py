@@ -59,14 +59,16 @@ class Hyper(C.Structure):
         ("weight_decay", C.c_float), ("p_quantile", C.c_float), ("fixed_alpha", C.c_float),
         ("adamw", C.c_int32), ("bias_correction", C.c_int32), ("round_m", C.c_int32),
         ("round_v", C.c_int32), ("param_dtype", C.c_int32), ("belief", C.c_int32),
+        ("param_round", C.c_int32), ("v_codebook", C.c_int32),
         ("seed", C.c_uint64),
     ]
 
 
 def hyper(lr=1e-3, beta1=0.8, beta2=0.999, eps=1e-8, weight_decay=0.01, p_quantile=0.1,
-          adamw=1, bias_correction=1, round_m=0, round_v=1, param_dtype=0, seed=0, belief=0, fixed_alpha=0.0) -> Hyper:
+          adamw=1, bias_correction=1, round_m=0, round_v=1, param_dtype=0, seed=0, belief=0, fixed_alpha=0.0,
+          param_round=0, v_codebook=0) -> Hyper:
     return Hyper(lr, beta1, beta2, eps, weight_decay, p_quantile, fixed_alpha, adamw, bias_correction,
-                 round_m, round_v, param_dtype, belief, seed)
+                 round_m, round_v, param_dtype, belief, param_round, v_codebook, seed)
 
 
 _lib = None
@@ -113,7 +115,11 @@ def lib() -> C.CDLL:
                           C.c_int, u8p, u8p, f32p, f32p, f32p, C.POINTER(Hyper), C.c_int64,
                           C.c_int, f32p, f32p, u8p, f32p, f32p]
     L.so_step.restype = C.c_int
-    L.so_dequant.argtypes = [C.c_int, C.c_int64, C.c_int, C.c_int, u8p, f32p, f32p, f32p]
+    L.so_dequant.argtypes = [C.c_int, C.c_int64, C.c_int, C.c_int, u8p, f32p, f32p, C.c_int, f32p]
+    L.so_bf16_sr.argtypes = [C.c_float, C.c_uint32]
+    L.so_bf16_sr.restype = C.c_uint32
+    L.so_bf16_rn.argtypes = [C.c_float]
+    L.so_bf16_rn.restype = C.c_uint32
     L.so_dequant.restype = C.c_int
     L.so_hardware_threads.argtypes = []
     L.so_hardware_threads.restype = C.c_int
@@ -163,6 +169,15 @@ def xi(draw16: int) -> float:
 
 def u01(draw16: int) -> float:
     return lib().so_u(draw16)
+
+
+def bf16_sr(x: float, draw16: int) -> int:
+    """bf16 bit pattern of ``x`` rounded stochastically with a 16-bit draw."""
+    return int(lib().so_bf16_sr(x, draw16))
+
+
+def bf16_rn(x: float) -> int:
+    return int(lib().so_bf16_rn(x))
 
 
 def quant_nearest(levels: np.ndarray, r: float) -> int:
@@ -224,6 +239,7 @@ class State:
         self.scale_m = np.zeros(self.nblk, np.float32)
         self.scale_v = np.zeros(self.nblk, np.float32)
         self.alpha = np.full(self.nblk, 0.5, np.float32)
+        self.v_codebook = 0          # selector the second moment was last written with
 
     def copy(self) -> "State":
         s = State.__new__(State)
@@ -255,6 +271,8 @@ def step(param: np.ndarray, grad_bf16: np.ndarray, st: State, h: Hyper, step_no:
                        _p(m32, C.c_float), _p(v32, C.c_float))
     if rc:
         raise ValueError("so_step rejected its arguments")
+    if m32 is None:
+        st.v_codebook = int(h.v_codebook)
     return mh, vh, fl
 
 
@@ -263,7 +281,8 @@ def dequant(st: State, which: int) -> np.ndarray:
     codes, scale, bits = ((st.codes_m, st.scale_m, st.bits_m) if which == 0
                           else (st.codes_v, st.scale_v, st.bits_v))
     rc = lib().so_dequant(which, st.numel, bits, st.block, _p(codes, C.c_uint8),
-                          _p(scale, C.c_float), _p(st.alpha, C.c_float), _p(out, C.c_float))
+                          _p(scale, C.c_float), _p(st.alpha, C.c_float), st.v_codebook,
+                          _p(out, C.c_float))
     if rc:
         raise ValueError("so_dequant rejected its arguments")
     return out

@@ -20,7 +20,9 @@
 // thresholds, the beta' table of Eq. 7 (Fig. 4), Theorem 3.1 as a property,
 // Proposition 3.5 decay statistics, Theorem 3.6 (unbiased SR, variance bound),
 // brute-force nearest-level search, Philox known answers, textbook AdamW,
-// memory accounting of Table 2.  Unpinned (paper silent; internal consistency
+// memory accounting of Table 2, the stochastic bf16 rounding over all 2^16
+// draws, the baseline second-moment codebooks by exhaustive search and the
+// swamping of Corollary 3.2 through the whole step.  Unpinned (paper silent; internal consistency
 // only): the rank convention of the p-quantile, the clamp constants of the
 // base, the 3-bit layout, the +1/-1 orientation of the signed DE codebook.
 //
@@ -164,7 +166,7 @@ void philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
-enum Purpose { PURPOSE_V = 0, PURPOSE_M = 1 };
+enum Purpose { PURPOSE_V = 0, PURPOSE_M = 1, PURPOSE_P = 2 };
 
 // The 16-bit draw that belongs to element `idx` of tensor `tensor` at `step`.
 // One Philox call serves eight consecutive elements:
@@ -279,6 +281,23 @@ inline uint16_t float_to_bf16(float x) {         // round to nearest, ties to ev
     return (uint16_t)((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
 }
 
+// Stochastic rounding of a binary32 value to bf16 with a 16-bit draw d: the two
+// neighbouring bf16 values are the truncation and the next pattern away from
+// zero; the upper one is taken with probability (dropped 16 bits) / 2^16, so the
+// expectation over d is the value itself.  Adding d to the pattern and
+// truncating does exactly that (the carry reaches bit 16 iff d >= 2^16 - low
+// bits).  A value already representable is returned unchanged; the largest
+// finite magnitudes can round to infinity; infinities and NaN are truncated
+// (NaN kept quiet).  Not from the paper: its 16-bit baseline is plain BF16
+// (Sec. 5, "Baselines"); this is the usual companion of bf16 parameters without
+// a binary32 master copy.
+inline uint16_t float_to_bf16_sr(float x, uint32_t d) {
+    uint32_t u = f2u(x);
+    if ((u & 0x7F800000u) == 0x7F800000u)
+        return (uint16_t)((u >> 16) | ((u & 0x007FFFFFu) ? 0x0040u : 0u));
+    return (uint16_t)((u + (d & 0xFFFFu)) >> 16);
+}
+
 // max over the block of the bit patterns of |x|: equal to the numerical maximum
 // for finite values, and a NaN if any element is NaN.
 inline float absmax_bits(const float* x, int n) {
@@ -287,9 +306,18 @@ inline float absmax_bits(const float* x, int n) {
     return u2f(m);
 }
 
+// Second-moment codebook selector of the hyper-parameter record -> Codebook, or
+// -1 for the logarithmic quantizer.
+inline int v_codebook_kind(int sel) {
+    return sel == 1 ? CB_DE_UNSIGNED : sel == 2 ? CB_LINEAR_UNSIGNED : sel == 3 ? CB_LINEAR_NOZERO : -1;
+}
+
 }  // namespace
 
 extern "C" {
+
+uint32_t so_bf16_sr(float x, uint32_t d) { return float_to_bf16_sr(x, d); }
+uint32_t so_bf16_rn(float x) { return float_to_bf16(x); }
 
 // Mirrors the hyper-parameter record of the library's C ABI (declared here
 // independently; the two must agree field by field).
@@ -299,6 +327,9 @@ struct so_hyper {
     float fixed_alpha;    // in (0,1): keep this base for every block (no quantile); otherwise 0
     int32_t adamw, bias_correction, round_m, round_v, param_dtype;
     int32_t belief;       // 0: Adam(W); 1: AdaBelief (second moment tracks (g - m^)^2 + eps)
+    int32_t param_round;  // bf16 parameters: 0 round to nearest even, 1 stochastic (Philox purpose 2)
+    int32_t v_codebook;   // second moment: 0 logarithmic, Eq. 6 (SOLO); 1 unsigned DE, 2 linear,
+                          // 3 linear without zero -- the baselines of Sec. 5, nearest rounding (Eq. 1)
     uint64_t seed;
 };
 
@@ -377,8 +408,10 @@ static void step_blocks(void* param, const uint16_t* grad, int64_t n, int64_t el
                         float* m_hat_out, float* v_hat_out, uint8_t* flags, float* m32,
                         float* v32) {
     const int Km = 1 << bits_m, Kv = 1 << bits_v;
-    float ym[256];
+    float ym[256], yv[256];
     build_codebook(CB_DE_SIGNED, bits_m, ym);
+    const int v_kind = v_codebook_kind(h->v_codebook);          // < 0: logarithmic (SOLO)
+    if (v_kind >= 0) build_codebook(v_kind, bits_v, yv);
 
     // Hyper-parameter scalars: binary64, rounded once.
     const double t = (double)step;
@@ -409,7 +442,9 @@ static void step_blocks(void* param, const uint16_t* grad, int64_t n, int64_t el
             if (l2) g = std::fmaf(h->weight_decay, p, g);       // Adam: L2 term in the gradient
             // Eq. 2 (or, with the full-precision switch, the stored binary32 moments)
             float m_t = m32 ? m32[i] : ym[get_code(cm, e, bits_m)] * dm;
-            float v_t = v32 ? v32[i] : pow_sm(al, get_code(cv, e, bits_v)) * dv;
+            float v_t = v32 ? v32[i]
+                      : v_kind >= 0 ? yv[get_code(cv, e, bits_v)] * dv
+                                    : pow_sm(al, get_code(cv, e, bits_v)) * dv;
             // Eq. 3.  AdaBelief (Sec. 5.2, "AdaBelief"; Zhuang et al. 2020): the unsigned EMA's
             // signal is (g - m^)^2 instead of g^2 and eps is added to the state at every step
             float m_h = std::fmaf(b1, m_t, omb1 * g);
@@ -421,8 +456,15 @@ static void step_blocks(void* param, const uint16_t* grad, int64_t n, int64_t el
             // Adam(W) with the un-requantized moments
             float den = std::fmaf(std::sqrt(v_h), inv_sqrt_bc2, h->eps);
             float p_new = std::fmaf(-step_size, m_h / den, p * decay);
-            if (h->param_dtype == 1) ((uint16_t*)param)[i] = float_to_bf16(p_new);
-            else ((float*)param)[i] = p_new;
+            if (h->param_dtype == 1) {
+                ((uint16_t*)param)[i] =
+                    h->param_round
+                        ? float_to_bf16_sr(p_new, philox_draw16(h->seed, step, tensor,
+                                                                elem_offset + i, PURPOSE_P))
+                        : float_to_bf16(p_new);
+            } else {
+                ((float*)param)[i] = p_new;
+            }
         }
         if (m_hat_out) std::copy(mh.begin(), mh.begin() + nb, m_hat_out + e0);
         if (v_hat_out) std::copy(vh.begin(), vh.begin() + nb, v_hat_out + e0);
@@ -467,6 +509,22 @@ static void step_blocks(void* param, const uint16_t* grad, int64_t n, int64_t el
         if (dv_new < TINY) {
             scale_v[j] = 0.0f;
             alpha[j] = 0.5f;
+        } else if (v_kind >= 0) {
+            // baseline: block-wise absmax scaling and the nearest level of a fixed codebook
+            // (Eq. 1; Sec. 5, "Baselines"); the base is not used and keeps its initial value
+            scale_v[j] = dv_new;
+            alpha[j] = 0.5f;
+            const float inv = 1.0f / dv_new;
+            for (int e = 0; e < nb; ++e) {
+                float r = vh[e] * inv;
+                set_code(cv, e, bits_v, quant_nearest(yv, Kv, r));
+                if (flags) {
+                    for (int k = 0; k + 1 < Kv; ++k) {
+                        double mid = 0.5 * ((double)yv[k] + (double)yv[k + 1]);
+                        if (std::fabs((double)r - mid) <= 1e-6 * std::fabs(mid)) flags[e0 + e] |= 2;
+                    }
+                }
+            }
         } else {
             scale_v[j] = dv_new;
             const float inv = 1.0f / dv_new;
@@ -516,6 +574,7 @@ int so_step(void* param, const uint16_t* grad, int64_t n, int64_t elem_offset, i
     if ((m32 == nullptr) != (v32 == nullptr)) return -1;
     if (n < 0 || block <= 0 || (block * bits_m) % 8 || (block * bits_v) % 8) return -1;
     if (bits_m < 2 || bits_m > 8 || bits_v < 1 || bits_v > 8 || elem_offset % block) return -1;
+    if (h->v_codebook < 0 || h->v_codebook > 3) return -1;
     const int64_t nblk = (n + block - 1) / block;
     if (nthreads <= 1 || nblk < 2) {
         step_blocks(param, grad, n, elem_offset, tensor, bits_m, bits_v, block, codes_m, codes_v,
@@ -537,10 +596,16 @@ int so_step(void* param, const uint16_t* grad, int64_t n, int64_t elem_offset, i
 }
 
 // Eq. 2 for inspection: which = 0 first moment, 1 second moment.
+// v_codebook: the selector the second moment was written with (0 = logarithmic).
 int so_dequant(int which, int64_t n, int bits, int block, const uint8_t* codes, const float* scale,
-               const float* alpha, float* out) {
+               const float* alpha, int v_codebook, float* out) {
     float ym[256];
     if (which == 0 && build_codebook(CB_DE_SIGNED, bits, ym) < 0) return -1;
+    const int v_kind = v_codebook_kind(v_codebook);
+    if (which == 1 && v_kind >= 0) {
+        if (build_codebook(v_kind, bits, ym) < 0) return -1;
+        which = 0;                                               // table lookup from here on
+    }
     const size_t slot = (size_t)block * bits / 8;
     for (int64_t i = 0; i < n; ++i) {
         int64_t j = i / block;

@@ -33,6 +33,7 @@ class Hyper(C.Structure):
         ("weight_decay", C.c_float), ("p_quantile", C.c_float), ("fixed_alpha", C.c_float),
         ("adamw", C.c_int32), ("bias_correction", C.c_int32), ("round_m", C.c_int32),
         ("round_v", C.c_int32), ("param_dtype", C.c_int32), ("belief", C.c_int32),
+        ("param_round", C.c_int32), ("v_codebook", C.c_int32),
         ("seed", C.c_uint64),
     ]
 
@@ -57,9 +58,10 @@ class RawState(C.Structure):
 
 
 def hyper(lr=1e-3, beta1=0.8, beta2=0.999, eps=1e-8, weight_decay=0.01, p_quantile=0.1,
-          adamw=1, bias_correction=1, round_m=0, round_v=1, param_dtype=0, seed=0, belief=0, fixed_alpha=0.0) -> Hyper:
+          adamw=1, bias_correction=1, round_m=0, round_v=1, param_dtype=0, seed=0, belief=0, fixed_alpha=0.0,
+          param_round=0, v_codebook=0) -> Hyper:
     return Hyper(lr, beta1, beta2, eps, weight_decay, p_quantile, fixed_alpha, adamw, bias_correction,
-                 round_m, round_v, param_dtype, belief, seed)
+                 round_m, round_v, param_dtype, belief, param_round, v_codebook, seed)
 
 
 _lib = None

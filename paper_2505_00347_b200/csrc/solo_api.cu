@@ -105,6 +105,7 @@ int check_hyper(const solo_hyper_t* h, int64_t step) {
     if (!unit(h->beta1) || !unit(h->beta2) || !unit(h->p_quantile) || !unit(h->fixed_alpha)) return SOLO_EINVAL;
     if (!(h->eps >= 0.0f) || !std::isfinite(h->lr) || !std::isfinite(h->weight_decay)) return SOLO_EINVAL;
     if (h->param_dtype != 0 && h->param_dtype != 1) return SOLO_EINVAL;
+    if (h->param_round != 0 || h->v_codebook != SOLO_V_LOG) return SOLO_EINVAL;
     return SOLO_OK;
 }
 

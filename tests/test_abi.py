@@ -58,7 +58,7 @@ def test_library_codebook_equals_oracle_codebook(B):
 
 def test_hyper_records_agree(B):
     """The oracle's and the library's hyper-parameter records have the same layout."""
-    assert C.sizeof(B.Hyper) == C.sizeof(oracle.Hyper) == 64
+    assert C.sizeof(B.Hyper) == C.sizeof(oracle.Hyper) == 72
     for (n1, t1), (n2, t2) in zip(B.Hyper._fields_, oracle.Hyper._fields_):
         assert n1 == n2 and t1 is t2
 

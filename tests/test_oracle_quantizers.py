@@ -211,3 +211,37 @@ def test_stochastic_rounding_brackets():
             assert oracle.quant_stochastic(y, float(r), min(float(frac) * 1.01 + 1e-6, 0.9999)) == lo
     for q in range(16):   # a value on a level stays there whatever u is
         assert oracle.quant_stochastic(y, float(y[q]), 0.5) == q
+
+
+def test_bf16_stochastic_rounding_probabilities_are_exact():
+    """Over all 2^16 draws the value goes to its upper bf16 neighbour exactly (dropped bits)
+    times, so the mean over the draws is the value itself; representable values never move."""
+    import struct
+    vals = [1.0, 1.00001, -3.14159, 0.1, -1e-3, 7e-41, 65504.0, -0.0, 2.0 ** -126 * 1.5]
+    for x in vals:
+        bits = struct.unpack("<I", struct.pack("<f", x))[0]
+        lo, hi = bits >> 16, bits & 0xffff
+        got = np.array([oracle.bf16_sr(x, d) for d in range(0, 65536, 1 if hi in (0, 1) else 7)])
+        assert set(np.unique(got)) <= {lo, lo + 1}
+        if hi == 0:
+            assert np.all(got == lo)                            # already bf16
+        # every draw: up iff d >= 2^16 - dropped bits
+        ds = np.arange(0, 65536, 1 if hi in (0, 1) else 7)
+        assert np.array_equal(got == lo + 1, ds >= 65536 - hi)
+    # counted in full for one value: ups == dropped bits, mean == value
+    x = 1.2345678
+    bits = struct.unpack("<I", struct.pack("<f", x))[0]
+    got = np.array([oracle.bf16_sr(x, d) for d in range(65536)], dtype=np.int64)
+    assert int((got == (bits >> 16) + 1).sum()) == bits & 0xffff
+    as_float = np.array([struct.unpack("<f", struct.pack("<I", int(b) << 16))[0] for b in np.unique(got)])
+    w = np.array([(got == b).sum() for b in np.unique(got)]) / 65536.0
+    assert float((as_float.astype(np.float64) * w).sum()) == float(np.float32(x))
+    # non-finite inputs are truncated, NaN stays NaN; the top finite bf16 binade can overflow
+    assert oracle.bf16_sr(float("inf"), 0xffff) == 0x7f80 and oracle.bf16_sr(float("-inf"), 1) == 0xff80
+    assert oracle.bf16_sr(float("nan"), 0) & 0x7fff > 0x7f80
+    assert oracle.bf16_sr(3.4e38, 0xffff) == 0x7f80 and oracle.bf16_sr(3.4e38, 0) == 0x7f7f
+    # nearest-even companion against torch
+    import torch
+    xs = np.random.default_rng(0).normal(0, 1, 2000).astype(np.float32)
+    want = torch.from_numpy(xs).to(torch.bfloat16).view(torch.int16).numpy().astype(np.uint16)
+    assert [oracle.bf16_rn(float(v)) for v in xs] == [int(v) for v in want]

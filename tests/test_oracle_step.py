@@ -280,3 +280,111 @@ def test_bf16_parameters_and_stochastic_m():
     a = np.array([oracle.get_code(ss.codes_m, e, 4) for e in range(128)])
     b = np.array([oracle.get_code(sn.codes_m, e, 4) for e in range(128)])
     assert np.max(np.abs(a - b)) <= 1 and np.any(a != b)
+
+
+def test_bf16_parameters_stochastic_rounding():
+    """bf16 parameters with param_round=1: each stored value is the binary32 result of the same
+    step rounded with the element's own purpose-2 draw; the states do not depend on the rounding
+    of the parameter; over many elements the rounding error averages out (nearest does not when
+    the update is far below half an ulp)."""
+    import struct
+    n, seed, tensor = 128 * 5 + 17, 0xABCDEF0123, 4
+    p, gb, _ = rand_inputs(n, 11)
+    pb = synth.bf16_bits(torch.from_numpy(p).to(torch.bfloat16))
+    pf = synth.bits_to_bf16(pb).float().numpy().copy()
+    hs = oracle.hyper(param_dtype=1, param_round=1, lr=1e-2, seed=seed)
+    hf = oracle.hyper(param_dtype=0, lr=1e-2, seed=seed)
+    s16, s32 = oracle.State(n, 2, 3, 128), oracle.State(n, 2, 3, 128)
+    for t in (1, 2):
+        before = synth.bits_to_bf16(pb).float().numpy().copy()
+        pf[:] = before
+        oracle.step(pb, gb, s16, hs, t, tensor=tensor, elem_offset=1280)
+        oracle.step(pf, gb, s32, hf, t, tensor=tensor, elem_offset=1280)
+        for i in range(n):
+            d = oracle.philox_draw16(seed, t, tensor, 1280 + i, 2)
+            bits = struct.unpack("<I", struct.pack("<f", float(pf[i])))[0]
+            assert int(pb[i]) == ((bits + d) >> 16) & 0xffff, (t, i)
+        assert np.array_equal(s16.codes_v, s32.codes_v) and np.array_equal(s16.codes_m, s32.codes_m)
+    # an update of 1/64 ulp: nearest rounding never moves the parameter, stochastic rounding
+    # moves it by the right amount on average
+    n = 1 << 15
+    ones = np.full(n, 0x3F80, np.uint16)                       # 1.0; ulp(bf16) = 2^-7 above 1
+    g = synth.bf16_bits(torch.full((n,), -1.0).to(torch.bfloat16))
+    lr = 2.0 ** -13
+    for rnd, moved in ((0, False), (1, True)):
+        pb = ones.copy()
+        h = oracle.hyper(param_dtype=1, param_round=rnd, lr=lr, weight_decay=0.0, seed=5,
+                         bias_correction=1, eps=0.0)
+        oracle.step(pb, g, oracle.State(n, 4, 4, 128), h, 1)   # first Adam step: p += lr exactly
+        val = synth.bits_to_bf16(pb).float().numpy().astype(np.float64)
+        if moved:
+            assert abs(val.mean() - (1.0 + lr)) < 4 * (2.0 ** -7) * math.sqrt(1 / 64 / n)
+        else:
+            assert np.all(val == 1.0)
+
+
+@pytest.mark.parametrize("sel,kind", [(1, "DE_UNSIGNED"), (2, "LINEAR_UNSIGNED"), (3, "LINEAR_NOZERO")])
+@pytest.mark.parametrize("bits_v", [2, 4])
+def test_baseline_second_moment_codebooks(sel, kind, bits_v):
+    """v_codebook != 0 (Sec. 5, "Baselines"): block-wise absmax scaling, codes are the nearest
+    level by exhaustive search, dequantization is level times scale, the base is not touched."""
+    n, block = 128 * 4 + 40, 128
+    p, _, _ = rand_inputs(n, 21)
+    y = oracle.codebook(getattr(oracle, kind), bits_v).astype(np.float64)
+    h = oracle.hyper(beta1=0.8, seed=3, v_codebook=sel)
+    st = oracle.State(n, 4, bits_v, block)
+    for t in range(1, 4):
+        _, gb, _ = rand_inputs(n, 40 + t)
+        prev = oracle.dequant(st, 1).astype(np.float64) if t > 1 else np.zeros(n)
+        _, vh, _ = oracle.step(p, gb, st, h, t, want_hat=True)
+        g = synth.bits_to_bf16(gb).float().numpy().astype(np.float64)
+        b2 = float(np.float32(0.999))
+        assert np.allclose(vh, b2 * prev + (1 - b2) * g * g, rtol=1e-5, atol=1e-20)   # Eq. 3 on Eq. 2
+        dv = oracle.dequant(st, 1)
+        for j in range(st.nblk):
+            sl = slice(j * block, min(n, (j + 1) * block))
+            assert st.scale_v[j] == vh[sl].max() and st.alpha[j] == 0.5
+            r = vh[sl].astype(np.float64) / float(st.scale_v[j])
+            dist = np.abs(r[:, None] - y[None, :])
+            q_ref = dist.argmin(1)
+            q = np.array([oracle.get_code(st.codes_v[j * (block * bits_v // 8):], e, bits_v)
+                          for e in range(sl.stop - sl.start)])
+            srt = np.sort(dist, axis=1)
+            tie = (srt[:, 1] - srt[:, 0]) < 1e-6
+            assert np.all((q == q_ref) | tie)
+            assert np.array_equal(dv[sl], (y[q].astype(np.float32) * st.scale_v[j]).astype(np.float32))
+
+
+def test_swamping_through_the_full_step():
+    """Sec. 3.2 (Corollary 3.2) on the whole step: one large element pins the block scale; with
+    the 4-bit linear codebook (beta2 = 0.999 >= 0.967) the small entries stay at level 0 under
+    a constant signal whose per-step increment is below half a gap, although the exact EMA
+    climbs to most of the scale; SOLO's logarithmic quantizer follows the exact EMA."""
+    n, b2 = 128, float(np.float32(0.999))
+    gvals = np.full(n, 1e-3, np.float32)
+    gvals[0] = 1.0
+    g_big = synth.bf16_bits(torch.from_numpy(gvals).to(torch.bfloat16))
+    gvals[1:] = 0.2
+    gvals[0] = 0.0                                              # the scale only decays from here
+    g_sig_t = torch.from_numpy(gvals).to(torch.bfloat16)
+    g_sig = synth.bf16_bits(g_sig_t)
+    gs = float(g_sig_t[1]) ** 2
+    exact, track = 0.0, {}
+    for t in range(1, 4):
+        exact = b2 * exact + (1 - b2) * 1e-6
+    for t in range(4, 64):
+        exact = b2 * exact + (1 - b2) * gs
+    for sel in (2, 0):
+        h = oracle.hyper(beta1=0.8, beta2=0.999, bias_correction=0, v_codebook=sel, seed=1, lr=0.0)
+        st = oracle.State(n, 4, 4, 128)
+        p = np.zeros(n, np.float32)
+        for t in range(1, 4):
+            oracle.step(p, g_big, st, h, t)
+        for t in range(4, 64):
+            oracle.step(p, g_sig, st, h, t)
+            # per-step increment relative to the scale: below half a gap of the linear codebook
+            assert (1 - b2) * gs / float(st.scale_v[0]) < 0.5 / 15
+        track[sel] = oracle.dequant(st, 1)[1:].astype(np.float64)
+        assert exact / float(st.scale_v[0]) > 0.5                  # the exact EMA is far from 0
+    assert np.all(track[2] == 0.0)                                  # swamped
+    assert abs(track[0].mean() / exact - 1) < 0.1                   # SOLO tracks
