@@ -121,7 +121,8 @@ def build_workload(cfg: int, device, args):
         over["block"] = args.block
     if over:
         w = synth.workload(cfg, **over)
-    params = [synth.make_param(w, i, device=device) for i in range(len(w.sizes))]
+    pdtype = torch.bfloat16 if args.param_bf16 else torch.float32
+    params = [synth.make_param(w, i, device=device, dtype=pdtype) for i in range(len(w.sizes))]
     grads = [synth.make_grad(w, i, 1, device=device) for i in range(len(w.sizes))]
     return w, params, grads
 
@@ -142,7 +143,8 @@ def run_ours(args, rank, world):
     state = B.State(list(w.sizes), w.bits_m, w.bits_v, w.block)
     ts = B.TensorSet(params, grads, state)
     h = B.hyper(lr=w.lr, beta1=w.beta1, beta2=w.beta2, weight_decay=w.weight_decay, seed=1234,
-                fixed_alpha=args.fixed_alpha)
+                fixed_alpha=args.fixed_alpha, v_codebook=args.v_codebook,
+                param_dtype=1 if args.param_bf16 else 0, param_round=1 if args.param_bf16 == 2 else 0)
     n = w.numel
     step_no = 0
 
@@ -177,11 +179,12 @@ def run_ours(args, rank, world):
     assert state.status() == 0
 
     # end to end: gradients come from pinned host memory, updated parameters go back to it
-    e2e_ms, h2d, d2h = None, 2 * n, 4 * n
+    pbytes = 2 if args.param_bf16 else 4
+    e2e_ms, h2d, d2h = None, 2 * n, pbytes * n
     if not args.no_e2e:
         big = max(w.sizes)
         hg = torch.empty(big, dtype=torch.bfloat16).pin_memory()
-        hp = torch.empty(big, dtype=torch.float32).pin_memory()
+        hp = torch.empty(big, dtype=params[0].dtype).pin_memory()
         hg[: grads[0].numel()].copy_(grads[0][: big].cpu())
         sync_all()
         k = max(1, min(args.steps, args.e2e_steps))
@@ -202,7 +205,7 @@ def run_ours(args, rank, world):
         return None
     ms_per_step = ms / args.steps
     value = whole_job_gparams(world, n, ms_per_step)
-    abytes = algorithmic_bytes_per_param(w.bits_m, w.bits_v, w.block)
+    abytes = algorithmic_bytes_per_param(w.bits_m, w.bits_v, w.block, pbytes)
     achieved = n * abytes / (ms_per_step * 1e-3) / 1e9
     peak, peak_kind = measured_peak()
     out = {
@@ -210,8 +213,11 @@ def run_ours(args, rank, world):
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"{w.name}: {len(w.sizes)} tensors, {n} params, m {w.bits_m}-bit / v {w.bits_v}-bit, "
-                               f"block {w.block}, fp32 params, bf16 grads, one solo_multi_step launch per step"
-                               + (f", fixed base {args.fixed_alpha}" if args.fixed_alpha else ""),
+                               f"block {w.block}, {'bf16' if args.param_bf16 else 'fp32'} params"
+                               f"{' (stochastic rounding)' if args.param_bf16 == 2 else ''}, bf16 grads, "
+                               "one solo_multi_step launch per step"
+                               + (f", fixed base {args.fixed_alpha}" if args.fixed_alpha else "")
+                               + (f", baseline v codebook {args.v_codebook}" if args.v_codebook else ""),
                    "l2": "working set (params+grads+state) far larger than the 126 MB L2; no flush needed"
                          if n * abytes > 1e9 else "working set fits L2: launch-bound point, not a bandwidth point",
                    "bytes_per_param": round(abytes, 4)},
@@ -220,6 +226,7 @@ def run_ours(args, rank, world):
                      "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
                      "traffic": (round(NCU_TRAFFIC_BYTES_PER_PARAM * n)
                                  if (NCU_TRAFFIC_BYTES_PER_PARAM is not None and args.policy == 0 and
+                                     not args.param_bf16 and not args.v_codebook and
                                      (w.bits_m, w.bits_v, w.block) == (2, 3, 128)) else None)},
         "gpu_launches": int(launches),
         "clocks": clk,
@@ -301,6 +308,10 @@ def main():
     ap.add_argument("--block", type=int, default=0, help="override the workload's block size")
     ap.add_argument("--fixed-alpha", type=float, default=0.0,
                     help="fixed base of the logarithmic codebook (no quantile step); 0 = the paper's quantile rule")
+    ap.add_argument("--v-codebook", type=int, default=0, choices=[0, 1, 2, 3],
+                    help="second-moment quantizer: 0 SOLO (default), 1 unsigned DE, 2 linear, 3 linear without zero")
+    ap.add_argument("--param-bf16", type=int, default=0, choices=[0, 1, 2],
+                    help="bf16 parameters: 1 nearest-even, 2 stochastic rounding (default 0: fp32)")
     ap.add_argument("--cpu-sample", type=int, default=1 << 27)
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--policy", type=int, default=0, help="kernel policy: 0 streamlined where it applies, 1 general")

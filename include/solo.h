@@ -158,7 +158,9 @@ int solo_multi_step(const solo_tensor_list_t* list, const solo_hyper_t* hyper, i
 /*
  * Eq. 2 for inspection: writes the dequantized moment of every element, tensors
  * concatenated without padding (sum of numel floats).
- *   which  0: first moment y[q] * Delta_m;  1: second moment alpha^q * Delta_v
+ *   which  0: first moment y[q] * Delta_m;  1: second moment alpha^q * Delta_v, or
+ *          y[q] * Delta_v with the baseline codebook of the state's last step
+ *          (hyper.v_codebook; a new state decodes as SOLO_V_LOG)
  *   out_dev  device, fp32
  * Asynchronous on `stream`.
  */
@@ -174,6 +176,26 @@ int solo_state_raw(const solo_state_t* state, int which, void** dev_ptr, size_t*
 /* Geometry of a state: total elements, total blocks, tensors, bits, block. */
 int solo_state_info(const solo_state_t* state, int64_t* numel, int64_t* num_blocks,
                     int32_t* num_tensors, int32_t* bits_m, int32_t* bits_v, int32_t* block);
+
+/*
+ * Checkpointing: the whole state as one HOST byte string, and back.  The paper stores
+ * exactly these arrays (codes, block scales, bases: Sec. 3.4 and the memory accounting
+ * of Table 2) but defines no file format; this one is the library's own.  Little-endian:
+ *   char    magic[8] = "SOLOST1"            int32 bits_m, bits_v, block, num_tensors,
+ *   int32   v_codebook, 0                   int64 num_blocks, numel[num_tensors]
+ *   (padding to a multiple of 16 bytes)
+ *   codes_m | codes_v | scale_m | scale_v | alpha, each padded to a multiple of 16 bytes
+ * solo_state_export_bytes gives the length.  export copies device -> host on `stream`
+ * and returns after the copy has completed (it synchronizes that stream); `bytes` must be
+ * at least the length.  import checks that the header describes the same widths, block
+ * size and tensor sizes as `state` (SOLO_ESTATE if not; SOLO_EINVAL for a short or
+ * foreign buffer), copies host -> device on `stream` and also returns after completion;
+ * the state then decodes and steps with the checkpoint's v_codebook.  Work queued on
+ * other streams that uses the state must be ordered by the caller.
+ */
+int solo_state_export_bytes(const solo_state_t* state, size_t* out);
+int solo_state_export(const solo_state_t* state, void* host_dst, size_t bytes, void* stream);
+int solo_state_import(solo_state_t* state, const void* host_src, size_t bytes, void* stream);
 
 /*
  * Reads the state's device status word into *status_out (0 = no problem seen).

@@ -99,6 +99,9 @@ def lib() -> C.CDLL:
     L.solo_multi_step_static.argtypes = [C.c_int32, vp, vp, C.POINTER(C.c_int64), C.POINTER(RawState),
                                          C.POINTER(Hyper), i64, vp]
     L.solo_multi_step_static.restype = C.c_int
+    L.solo_state_export_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
+    L.solo_state_export.argtypes = [vp, vp, C.c_size_t, vp]
+    L.solo_state_import.argtypes = [vp, vp, C.c_size_t, vp]
     L.solo_launch_count.argtypes = []
     L.solo_launch_count.restype = C.c_int64
     L.solo_strerror.argtypes = [i32]
@@ -106,7 +109,8 @@ def lib() -> C.CDLL:
     for name in ("solo_state_create", "solo_state_create_multi", "solo_state_destroy",
                  "solo_state_bytes", "solo_step", "solo_multi_step", "solo_dequant",
                  "solo_state_raw", "solo_state_info", "solo_state_status", "solo_codebook_m",
-                 "solo_set_kernel_policy", "solo_debug_check_fast_log"):
+                 "solo_set_kernel_policy", "solo_debug_check_fast_log", "solo_state_export_bytes",
+                 "solo_state_export", "solo_state_import"):
         getattr(L, name).restype = C.c_int
     _lib = L
     return L
@@ -188,6 +192,21 @@ class State:
             raise ValueError(f"expected {nbytes} bytes, got {v.numel()}")
         torch.cuda.synchronize()
         _cuda_memcpy(ptr, v.data_ptr(), nbytes, 1)
+
+    def export(self) -> torch.Tensor:
+        """The whole state as one CPU uint8 tensor (solo_state_export)."""
+        n = C.c_size_t()
+        _check(lib().solo_state_export_bytes(self.handle, C.byref(n)), "solo_state_export_bytes")
+        out = torch.empty(n.value, dtype=torch.uint8)
+        _check(lib().solo_state_export(self.handle, out.data_ptr(), n.value,
+                                       torch.cuda.current_stream().cuda_stream), "solo_state_export")
+        return out
+
+    def load(self, blob: torch.Tensor) -> None:
+        """Restores a state written by export() into this one (solo_state_import)."""
+        b = blob.contiguous().view(torch.uint8).cpu()
+        _check(lib().solo_state_import(self.handle, b.data_ptr(), b.numel(),
+                                       torch.cuda.current_stream().cuda_stream), "solo_state_import")
 
     def status(self) -> int:
         s = C.c_int()

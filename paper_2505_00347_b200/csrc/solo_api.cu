@@ -29,7 +29,8 @@ struct solo_state {
     float* alpha = nullptr;
     int64_t* geom = nullptr;      // numel[T] | block_start[T+1] | tile_start[T+1] | elem_start[T+1]
     float* tables_m = nullptr;    // first-moment codebook tables for bits_m
-    float* tables_v = nullptr;    // same construction for bits_v (solo_dequant of m only needs bits_m)
+    float* tables_v = nullptr;    // the three baseline second-moment codebooks for bits_v, each y[K] | mid[K-1]
+    int v_codebook = SOLO_V_LOG;  // selector of the last step (what solo_dequant decodes with)
     int* status = nullptr;
     size_t bytes_codes_m = 0, bytes_codes_v = 0;
 };
@@ -77,6 +78,44 @@ void codebook_tables(int bits, std::vector<float>& t) {
     }
 }
 
+// Unsigned codebooks of Appendix A for the baseline second-moment quantizers, ascending.
+//   SOLO_V_DE            {0, 1} and 10^-E times the midpoints of the 2^F cells of [0.1, 1],
+//                        E = 0..b-2 leading zero bits, one indicator bit, F = b-1-E fraction bits
+//   SOLO_V_LINEAR        k / (2^b - 1), k = 0..2^b-1
+//   SOLO_V_LINEAR_NOZERO k / 2^b, k = 1..2^b
+void unsigned_levels(int kind, int bits, std::vector<float>& y) {
+    const int K = 1 << bits;
+    y.clear();
+    if (kind == SOLO_V_LINEAR) {
+        for (int k = 0; k < K; ++k) y.push_back((float)((double)k / (double)(K - 1)));
+    } else if (kind == SOLO_V_LINEAR_NOZERO) {
+        for (int k = 1; k <= K; ++k) y.push_back((float)((double)k / (double)K));
+    } else {
+        y.push_back(0.0f);
+        for (int E = bits - 2; E >= 0; --E) {                 // smallest decade first
+            const int F = bits - 1 - E;
+            const double two = (double)(1 << (F + 1));
+            double ten = 10.0;
+            for (int i = 0; i < E; ++i) ten *= 10.0;
+            for (int j = 0; j < (1 << F); ++j)
+                y.push_back((float)((two + 9.0 * (double)(2 * j + 1)) / (ten * two)));
+        }
+        y.push_back(1.0f);
+    }
+}
+
+// The three baseline tables back to back, kind = 1, 2, 3: y[K] | mid[K-1] each.
+constexpr int v_table_floats(int bits) { return 2 * (1 << bits) - 1; }
+void baseline_v_tables(int bits, float* t) {
+    const int K = 1 << bits;
+    std::vector<float> y;
+    for (int kind = 1; kind <= 3; ++kind, t += v_table_floats(bits)) {
+        unsigned_levels(kind, bits, y);
+        for (int k = 0; k < K; ++k) t[k] = y[k];
+        for (int k = 0; k + 1 < K; ++k) t[K + k] = 0.5f * (y[k] + y[k + 1]);
+    }
+}
+
 __global__ void fill_f32(float* p, int64_t n, float v) {
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n;
          i += (int64_t)gridDim.x * blockDim.x)
@@ -105,7 +144,8 @@ int check_hyper(const solo_hyper_t* h, int64_t step) {
     if (!unit(h->beta1) || !unit(h->beta2) || !unit(h->p_quantile) || !unit(h->fixed_alpha)) return SOLO_EINVAL;
     if (!(h->eps >= 0.0f) || !std::isfinite(h->lr) || !std::isfinite(h->weight_decay)) return SOLO_EINVAL;
     if (h->param_dtype != 0 && h->param_dtype != 1) return SOLO_EINVAL;
-    if (h->param_round != 0 || h->v_codebook != SOLO_V_LOG) return SOLO_EINVAL;
+    if (h->param_round != 0 && h->param_round != 1) return SOLO_EINVAL;
+    if (h->v_codebook < SOLO_V_LOG || h->v_codebook > SOLO_V_LINEAR_NOZERO) return SOLO_EINVAL;
     return SOLO_OK;
 }
 
@@ -130,6 +170,7 @@ void reduce_hyper(const solo_hyper_t* h, int64_t step, int block, StepArgs& a) {
     a.round_m = h->round_m ? 1 : 0;
     a.round_v = h->round_v ? 1 : 0;
     a.param_bf16 = h->param_dtype;
+    a.param_sr = (h->param_dtype == 1 && h->param_round) ? 1 : 0;
     a.block = block;
     int64_t k = (int64_t)std::ceil((double)h->p_quantile * (double)block);
     a.k_full = (int)std::min<int64_t>(std::max<int64_t>(k, 1), block);
@@ -145,8 +186,8 @@ void reduce_hyper(const solo_hyper_t* h, int64_t step, int block, StepArgs& a) {
 int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
     const bool cta_group = s->block == 2048;
     solo::StepKernel k = nullptr;
-    if (g_policy.load(std::memory_order_relaxed) == 0 && !a.round_m && !a.param_bf16 && a.eps >= 1e-12f &&
-        s->tiles_total < (int64_t)1 << 31)
+    if (g_policy.load(std::memory_order_relaxed) == 0 && !a.round_m && !a.param_bf16 && !a.tables_v &&
+        a.eps >= 1e-12f && s->tiles_total < (int64_t)1 << 31)
         k = solo::fast_kernel(s->bits_m, s->bits_v, s->block);
     size_t dyn_smem = k ? solo::fast_kernel_smem() : 0;
     if (!k) k = solo::step_kernel(s->bits_m, s->bits_v, cta_group);
@@ -180,6 +221,14 @@ void fill_state_args(const solo_state* s, StepArgs& a) {
     a.status = s->status;
 }
 
+// Second-moment quantizer of this step; the state remembers it for solo_dequant.
+void select_v_codebook(solo_state* s, const solo_hyper_t* h, StepArgs& a) {
+    a.tables_v = h->v_codebook == SOLO_V_LOG
+                     ? nullptr
+                     : s->tables_v + (size_t)(h->v_codebook - 1) * v_table_floats(s->bits_v);
+    s->v_codebook = h->v_codebook;
+}
+
 bool on_state_device(const solo_state* s) {
     int dev = -1;
     return cudaGetDevice(&dev) == cudaSuccess && dev == s->device;
@@ -188,12 +237,15 @@ bool on_state_device(const solo_state* s) {
 // ---------------------------------------------------------------------------
 // Fixed scratch of the allocation-free entry point: per device, held until exit.
 //   int64 numel[MAX] | block_start[MAX+1] | tile_start[MAX+1]   then
-//   float tables[3*256-2] (y | mid | 1/gap of the first-moment codebook)   then   int status
+//   float tables[3*256-2] (y | mid | 1/gap of the first-moment codebook)   then
+//   float tables_v[2*256-1] (y | mid of a baseline second-moment codebook)   then   int status
 // ---------------------------------------------------------------------------
 constexpr int STATIC_MAX_T = SOLO_STATIC_MAX_TENSORS;
 constexpr size_t STATIC_GEOM_BYTES = (size_t)(3 * STATIC_MAX_T + 2) * sizeof(int64_t);
 constexpr size_t STATIC_TABLE_BYTES = (size_t)(3 * 256 - 2) * sizeof(float);
-constexpr size_t STATIC_STATUS_OFF = (STATIC_GEOM_BYTES + STATIC_TABLE_BYTES + 15) / 16 * 16;
+constexpr size_t STATIC_VTABLE_BYTES = (size_t)(2 * 256 - 1) * sizeof(float);
+constexpr size_t STATIC_STATUS_OFF =
+    (STATIC_GEOM_BYTES + STATIC_TABLE_BYTES + STATIC_VTABLE_BYTES + 15) / 16 * 16;
 constexpr size_t STATIC_BYTES = STATIC_STATUS_OFF + 16;
 static_assert(STATIC_BYTES <= 32 * 1024, "documented size of the fixed scratch");
 
@@ -266,7 +318,8 @@ int solo_state_create_multi(const int64_t* numel_host, int num_tensors, int bits
     geom.insert(geom.end(), s->elem_start.begin(), s->elem_start.end());
     std::vector<float> tm, tv;
     codebook_tables(bits_m, tm);
-    codebook_tables(bits_v, tv);
+    tv.assign(3 * v_table_floats(bits_v), 0.0f);
+    baseline_v_tables(bits_v, tv.data());
 
     bool ok = true;
     auto alloc = [&](void** p, size_t bytes) {
@@ -335,6 +388,7 @@ int solo_step(void* param_dev, const void* grad_dev, solo_state_t* s, const solo
     std::memset(&a, 0, sizeof(a));
     fill_state_args(s, a);
     reduce_hyper(hyper, step, s->block, a);
+    select_v_codebook(s, hyper, a);
     a.param_single = param_dev;
     a.grad_single = grad_dev;
     return launch_step(s, a, (cudaStream_t)stream);
@@ -351,6 +405,7 @@ int solo_multi_step(const solo_tensor_list_t* list, const solo_hyper_t* hyper, i
     std::memset(&a, 0, sizeof(a));
     fill_state_args(s, a);
     reduce_hyper(hyper, step, s->block, a);
+    select_v_codebook(s, hyper, a);
     a.param_list = list->param;
     a.grad_list = list->grad;
     a.numel_check = list->numel;
@@ -396,14 +451,25 @@ int solo_multi_step_static(int32_t num_tensors, void* const* param_dev, const vo
         codebook_tables(st->bits_m, tm);
         std::memcpy(tables, tm.data(), tm.size() * sizeof(float));
     }
+    float tables_v[2 * 256 - 1];
+    const bool vtab = hyper->v_codebook != SOLO_V_LOG;
+    if (vtab) {
+        float all[3 * (2 * 256 - 1)];
+        baseline_v_tables(st->bits_v, all);             // std::vector inside: host memory only
+        std::memcpy(tables_v, all + (size_t)(hyper->v_codebook - 1) * v_table_floats(st->bits_v),
+                    (size_t)v_table_floats(st->bits_v) * sizeof(float));
+    }
     const size_t geom_bytes = (size_t)(3 * T + 2) * sizeof(int64_t);
     const size_t table_bytes = (size_t)(3 * (1 << st->bits_m) - 2) * sizeof(float);
     int64_t* d_geom = (int64_t*)scratch;
     float* d_tables = (float*)(scratch + STATIC_GEOM_BYTES);
+    float* d_tables_v = (float*)(scratch + STATIC_GEOM_BYTES + STATIC_TABLE_BYTES);
     int* d_status = (int*)(scratch + STATIC_STATUS_OFF);
     // pageable sources: both copies are staged before cudaMemcpyAsync returns
     if (cudaMemcpyAsync(d_geom, geom, geom_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
         cudaMemcpyAsync(d_tables, tables, table_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        (vtab && cudaMemcpyAsync(d_tables_v, tables_v, (size_t)v_table_floats(st->bits_v) * sizeof(float),
+                                 cudaMemcpyHostToDevice, stream) != cudaSuccess) ||
         cudaMemsetAsync(d_status, 0, 16, stream) != cudaSuccess) {
         cudaGetLastError();
         return SOLO_ECUDA;
@@ -427,6 +493,7 @@ int solo_multi_step_static(int32_t num_tensors, void* const* param_dev, const vo
     a.scale_v = st->scale_v;
     a.alpha = st->alpha;
     a.tables = d_tables;
+    a.tables_v = vtab ? d_tables_v : nullptr;
     a.status = d_status;
     reduce_hyper(hyper, step, block, a);
     a.param_list = param_dev;
@@ -454,6 +521,10 @@ int solo_dequant(const solo_state_t* s, int which, float* out_dev, void* stream)
     a.out = out_dev;
     a.block = s->block;
     a.which = which;
+    if (which == 1 && s->v_codebook != SOLO_V_LOG) {          // level table times scale
+        a.tables = s->tables_v + (size_t)(s->v_codebook - 1) * v_table_floats(s->bits_v);
+        a.which = 0;
+    }
     const int bits = which == 0 ? s->bits_m : s->bits_v;
     int64_t grid = std::min<int64_t>(s->tiles_total, (int64_t)sm_count(s->device) * 8);
     cudaError_t e = solo::launch_dequant(bits, a, (unsigned)grid, (cudaStream_t)stream);
@@ -487,6 +558,92 @@ int solo_state_info(const solo_state_t* s, int64_t* numel, int64_t* num_blocks, 
     if (bits_m) *bits_m = s->bits_m;
     if (bits_v) *bits_v = s->bits_v;
     if (block) *block = s->block;
+    return SOLO_OK;
+}
+
+namespace {
+constexpr char CKPT_MAGIC[8] = {'S', 'O', 'L', 'O', 'S', 'T', '1', 0};
+size_t pad16(size_t n) { return (n + 15) / 16 * 16; }
+size_t ckpt_header_bytes(int T) { return pad16(8 + 6 * 4 + 8 + (size_t)T * 8); }
+struct CkptPart { void* dev; size_t bytes; };
+void ckpt_parts(const solo_state* s, CkptPart (&p)[5]) {
+    p[0] = {s->codes_m, s->bytes_codes_m};
+    p[1] = {s->codes_v, s->bytes_codes_v};
+    p[2] = {s->scale_m, (size_t)s->nblk_total * 4};
+    p[3] = {s->scale_v, (size_t)s->nblk_total * 4};
+    p[4] = {s->alpha, (size_t)s->nblk_total * 4};
+}
+size_t ckpt_bytes(const solo_state* s) {
+    CkptPart p[5];
+    ckpt_parts(s, p);
+    size_t n = ckpt_header_bytes(s->num_tensors);
+    for (const CkptPart& q : p) n += pad16(q.bytes);
+    return n;
+}
+}  // namespace
+
+int solo_state_export_bytes(const solo_state_t* s, size_t* out) {
+    if (!s || !out) return SOLO_EINVAL;
+    *out = ckpt_bytes(s);
+    return SOLO_OK;
+}
+
+int solo_state_export(const solo_state_t* s, void* host_dst, size_t bytes, void* stream_) {
+    if (!s || !host_dst) return SOLO_EINVAL;
+    if (bytes < ckpt_bytes(s)) return SOLO_EINVAL;
+    if (!on_state_device(s)) return SOLO_ESTATE;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    unsigned char* dst = (unsigned char*)host_dst;
+    const int T = s->num_tensors;
+    std::memset(dst, 0, ckpt_header_bytes(T));
+    std::memcpy(dst, CKPT_MAGIC, 8);
+    const int32_t head[6] = {s->bits_m, s->bits_v, s->block, T, s->v_codebook, 0};
+    std::memcpy(dst + 8, head, sizeof(head));
+    std::memcpy(dst + 32, &s->nblk_total, 8);
+    std::memcpy(dst + 40, s->numel.data(), (size_t)T * 8);
+    size_t off = ckpt_header_bytes(T);
+    CkptPart p[5];
+    ckpt_parts(s, p);
+    for (const CkptPart& q : p) {
+        if (cudaMemcpyAsync(dst + off, q.dev, q.bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess) {
+            cudaGetLastError();
+            return SOLO_ECUDA;
+        }
+        std::memset(dst + off + q.bytes, 0, pad16(q.bytes) - q.bytes);   // padding, outside the copy
+        off += pad16(q.bytes);
+    }
+    if (cudaStreamSynchronize(stream) != cudaSuccess) { cudaGetLastError(); return SOLO_ECUDA; }
+    return SOLO_OK;
+}
+
+int solo_state_import(solo_state_t* s, const void* host_src, size_t bytes, void* stream_) {
+    if (!s || !host_src) return SOLO_EINVAL;
+    const unsigned char* src = (const unsigned char*)host_src;
+    if (bytes < 40 || std::memcmp(src, CKPT_MAGIC, 8) != 0) return SOLO_EINVAL;
+    int32_t head[6];
+    int64_t nblk = 0;
+    std::memcpy(head, src + 8, sizeof(head));
+    std::memcpy(&nblk, src + 32, 8);
+    if (head[0] != s->bits_m || head[1] != s->bits_v || head[2] != s->block || head[3] != s->num_tensors ||
+        nblk != s->nblk_total)
+        return SOLO_ESTATE;
+    if (head[4] < SOLO_V_LOG || head[4] > SOLO_V_LINEAR_NOZERO) return SOLO_EINVAL;
+    if (bytes < ckpt_bytes(s)) return SOLO_EINVAL;
+    if (std::memcmp(src + 40, s->numel.data(), (size_t)s->num_tensors * 8) != 0) return SOLO_ESTATE;
+    if (!on_state_device(s)) return SOLO_ESTATE;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    size_t off = ckpt_header_bytes(s->num_tensors);
+    CkptPart p[5];
+    ckpt_parts(s, p);
+    for (const CkptPart& q : p) {
+        if (cudaMemcpyAsync(q.dev, src + off, q.bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+            cudaGetLastError();
+            return SOLO_ECUDA;
+        }
+        off += pad16(q.bytes);
+    }
+    if (cudaStreamSynchronize(stream) != cudaSuccess) { cudaGetLastError(); return SOLO_ECUDA; }
+    s->v_codebook = head[4];
     return SOLO_OK;
 }
 

@@ -46,11 +46,13 @@ struct StepArgs {
     float* scale_v;
     float* alpha;
     const float* tables;               // y[K], mid[K-1], inv_gap[K-1] of the first-moment codebook
+    const float* tables_v;             // baseline second-moment codebook y[K], mid[K-1]; null: Eq. 6
     int* status;                       // device word: non-zero after a descriptor mismatch
     // hyper-parameters, already reduced to what the kernel multiplies with
     float beta1, beta2, omb1, omb2, step_size, inv_sqrt_bc2, eps, decay, weight_decay, p_quantile;
     float fixed_alpha;                 // in (0,1): base of every block; 0: base from the p-quantile
     int32_t l2, round_m, round_v, param_bf16, block, k_full, belief;
+    int32_t param_sr;                  // bf16 parameters are rounded stochastically (Philox purpose 2)
     uint32_t seed_lo, seed_hi, step32;
     // Philox round keys (seed + r * Weyl constant), r = 0..9: [2r] low word, [2r+1] high word
     uint32_t rk[20];
@@ -113,6 +115,14 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
 }
 
 // 16-bit draw of element i (0..7) of a thread's eight: halfword i of the Philox block.
+// binary32 -> bf16 bit pattern with a 16-bit draw: the upper neighbour is taken with
+// probability (dropped bits) / 2^16; infinities and NaN are truncated (NaN kept quiet).
+__device__ __forceinline__ uint32_t bf16_sr(float x, uint32_t d) {
+    const uint32_t u = __float_as_uint(x);
+    if ((u & 0x7F800000u) == 0x7F800000u) return (u >> 16) | ((u & 0x007FFFFFu) ? 0x0040u : 0u);
+    return (u + d) >> 16;
+}
+
 __device__ __forceinline__ uint32_t draw16(const uint32_t (&w)[4], int i) {
     return (i & 1) ? (w[i >> 1] >> 16) : (w[i >> 1] & 0xFFFFu);
 }
@@ -265,6 +275,8 @@ __global__ void __launch_bounds__(CTA) solo_step_kernel(const StepArgs a) {
     __shared__ float s_y[KM];
     __shared__ float s_mid[KM];
     __shared__ float s_gap[KM];
+    __shared__ float s_yv[KV];
+    __shared__ float s_midv[KV];
     __shared__ uint32_t s_sort[CTA_GROUP ? 1 : EPT * CTA];
     __shared__ uint32_t s_hist[CTA_GROUP ? 256 + 16 : 1];
     __shared__ uint32_t s_red[8];
@@ -277,6 +289,12 @@ __global__ void __launch_bounds__(CTA) solo_step_kernel(const StepArgs a) {
             s_gap[i] = a.tables[2 * KM - 1 + i];
         }
     }
+    const bool vtab = a.tables_v != nullptr;                  // baseline codebook for the second moment
+    if (vtab)
+        for (int i = tid; i < KV; i += CTA) {
+            s_yv[i] = a.tables_v[i];
+            if (i < KV - 1) s_midv[i] = a.tables_v[KV + i];
+        }
     __syncthreads();
 
     const int B = CTA_GROUP ? TILE : a.block;
@@ -358,7 +376,7 @@ __global__ void __launch_bounds__(CTA) solo_step_kernel(const StepArgs a) {
             uint32_t qm = (uint32_t)(cm >> (i * BM)) & (KM - 1);
             uint32_t qv = (uint32_t)(cv >> (i * BV)) & (KV - 1);
             float mt = s_y[qm] * dm;
-            float vt = pow_sm<BV>(a2, qv) * dv;
+            float vt = (vtab ? s_yv[qv] : pow_sm<BV>(a2, qv)) * dv;
             mh[i] = __fmaf_rn(a.beta1, mt, a.omb1 * gi);
             const float sig = a.belief ? gi - mh[i] : gi;            // AdaBelief: (g - m^)^2, plus eps
             vh[i] = __fmaf_rn(a.beta2, vt, a.omb2 * (sig * sig));
@@ -368,13 +386,24 @@ __global__ void __launch_bounds__(CTA) solo_step_kernel(const StepArgs a) {
         }
 
         // ---- store parameters ----
+        const bool sr = bf16p && a.param_sr;
+        uint32_t wp[4] = {0u, 0u, 0u, 0u};
+        if (sr) {
+            const uint64_t c = (uint64_t)e0 >> 3;
+            philox4x32_10((uint32_t)c, (uint32_t)(c >> 32), a.step32, (uint32_t)tensor * 4u + 2u,
+                          a.seed_lo, a.seed_hi, wp);
+        }
         if (vec) {
             if (bf16p) {
                 uint32_t pp[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    __nv_bfloat162 h = __floats2bfloat162_rn(p[2 * i], p[2 * i + 1]);
-                    pp[i] = *reinterpret_cast<uint32_t*>(&h);
+                    if (sr) {
+                        pp[i] = bf16_sr(p[2 * i], wp[i] & 0xFFFFu) | (bf16_sr(p[2 * i + 1], wp[i] >> 16) << 16);
+                    } else {
+                        __nv_bfloat162 h = __floats2bfloat162_rn(p[2 * i], p[2 * i + 1]);
+                        pp[i] = *reinterpret_cast<uint32_t*>(&h);
+                    }
                 }
                 *reinterpret_cast<uint4*>(pbase + e0 * 2) = make_uint4(pp[0], pp[1], pp[2], pp[3]);
             } else {
@@ -385,7 +414,8 @@ __global__ void __launch_bounds__(CTA) solo_step_kernel(const StepArgs a) {
 #pragma unroll
             for (int i = 0; i < EPT; ++i) {
                 if (i < nv) {
-                    if (bf16p) reinterpret_cast<__nv_bfloat16*>(pbase)[e0 + i] = __float2bfloat16_rn(p[i]);
+                    if (sr) reinterpret_cast<uint16_t*>(pbase)[e0 + i] = (uint16_t)bf16_sr(p[i], draw16(wp, i));
+                    else if (bf16p) reinterpret_cast<__nv_bfloat16*>(pbase)[e0 + i] = __float2bfloat16_rn(p[i]);
                     else reinterpret_cast<float*>(pbase)[e0 + i] = p[i];
                 }
             }
@@ -441,7 +471,18 @@ __global__ void __launch_bounds__(CTA) solo_step_kernel(const StepArgs a) {
         // ---- second moment: p-quantile, base, Eq. 6 ----
         uint64_t ov = 0;
         float al_new = 0.5f;
-        if (!zero_v) {                                           // uniform over the group
+        if (!zero_v && vtab) {                                   // uniform: Eq. 1 on a fixed codebook
+            const float inv = 1.0f / dv_new;
+#pragma unroll
+            for (int i = 0; i < EPT; ++i) {
+                const float r = vh[i] * inv;
+                uint32_t q = 0;
+#pragma unroll
+                for (int s = KV / 2; s >= 1; s >>= 1)
+                    if (r > s_midv[q + s - 1]) q += s;
+                if (i < nv) ov |= (uint64_t)q << (i * BV);
+            }
+        } else if (!zero_v) {                                    // uniform over the group
             int k = a.k_full;
             if (nb != B) {
                 k = (int)ceil((double)a.p_quantile * (double)nb);
@@ -501,9 +542,9 @@ struct DequantArgs {
     const uint8_t* codes;
     const float* scale;
     const float* alpha;
-    const float* tables;
+    const float* tables;               // y[K] of the codebook when which == 0
     float* out;
-    int32_t block, which;
+    int32_t block, which;              // which: 0 level table times scale, 1 alpha^q times scale
 };
 
 template <int BITS>

@@ -56,6 +56,12 @@ def test_bits_and_blocks_random_state(bits_m, bits_v, block):
     dict(fixed_alpha=0.5),
     dict(fixed_alpha=0.9, round_v=0),
     dict(belief=1, eps=1e-12, beta2=0.99, adamw=0, weight_decay=0.05),
+    dict(param_dtype=1, param_round=1, lr=1e-2, seed=77),
+    dict(param_dtype=1, param_round=1, lr=3e-5, weight_decay=0.0, round_m=1),
+    dict(v_codebook=1),
+    dict(v_codebook=2, belief=1),
+    dict(v_codebook=3),
+    dict(v_codebook=3, param_dtype=1, param_round=1, adamw=0),
 ])
 def test_hyper_parameter_modes(hk):
     sizes = (128 * 40 + 17, 300)
@@ -68,6 +74,40 @@ def test_hyper_parameter_modes(hk):
     st0 = synth.make_state(sizes, 4, 3, 128, seed=17)
     run_lockstep(sizes, 4, 3, 128, base, 3, gf, params, state0=st0)
     run_lockstep(sizes, 4, 3, 128, base, 3, gf, params)
+
+
+@pytest.mark.parametrize("sel", [1, 2, 3])
+@pytest.mark.parametrize("bits_v,block", [(2, 64), (3, 128), (4, 2048), (8, 256)])
+def test_baseline_second_moment_codebooks(sel, bits_v, block):
+    """Sec. 5 baselines for the unsigned state (unsigned DE, linear, linear without zero;
+    Appendix A) at every width, from a random packed state and from zero, ragged sizes."""
+    sizes = (block * 5 + 3, 1, 2048 * 2 + 9, block - 1)
+    w = synth.workload(4, sizes=sizes)                            # zero blocks and zero elements
+    params, gf = _inputs(w)
+    hk = dict(lr=1e-3, beta1=0.8, beta2=0.999, weight_decay=0.01, seed=5, v_codebook=sel)
+    st0 = synth.make_state(sizes, 4, bits_v, block, seed=sel * 1000 + bits_v * 10 + block)
+    run_lockstep(sizes, 4, bits_v, block, hk, 2, gf, params, state0=st0)
+    run_lockstep(sizes, 4, bits_v, block, hk, 3, gf, params)
+
+
+def test_stochastic_bf16_rounding_is_unbiased_on_the_device():
+    """Updates of 1/64 ulp(bf16): nearest rounding leaves every parameter where it is, stochastic
+    rounding moves the mean by the update (first Adam step from zero state: p += lr exactly)."""
+    from paper_2505_00347_b200 import binding as B
+    n, lr = 1 << 20, 2.0 ** -13
+    g = torch.full((n,), -1.0, dtype=torch.bfloat16, device="cuda")
+    for rnd in (0, 1):
+        p = torch.ones(n, dtype=torch.bfloat16, device="cuda")
+        st = B.State(n, 4, 4, 128)
+        B.solo_step(p, g, st, B.hyper(param_dtype=1, param_round=rnd, lr=lr, weight_decay=0.0, seed=5, eps=0.0), 1)
+        torch.cuda.synchronize()
+        mean = float(p.double().mean())
+        if rnd:
+            assert abs(mean - (1.0 + lr)) < 5 * 2.0 ** -7 * (1 / 64 / n) ** 0.5
+            assert set(p.unique().tolist()) == {1.0, 1.0 + 2.0 ** -7}
+        else:
+            assert mean == 1.0
+        st.destroy()
 
 
 def test_streamlined_kernel_rounding_guard_is_sound():
@@ -138,6 +178,65 @@ def test_nan_and_inf_gradients_do_not_hang():
     assert torch.isfinite(out[256:]).all()          # untouched blocks stay finite
     assert st.status() == 0
     st.destroy()
+
+
+@pytest.mark.parametrize("v_codebook", [0, 3])
+def test_checkpoint_export_import(v_codebook):
+    """solo_state_export / solo_state_import: the byte string holds the header and the five
+    arrays in the documented order, equal to the oracle's state after the same steps; a state
+    restored from it continues bit-identically; a checkpoint of another geometry is refused."""
+    import struct
+    from paper_2505_00347_b200 import binding as B
+    sizes, bits_m, bits_v, block = (128 * 9 + 5, 77, 4096), 2, 3, 128
+    w = synth.workload(2, sizes=sizes)
+    hk = dict(lr=1e-3, beta1=0.6, beta2=0.999, weight_decay=0.01, seed=21, v_codebook=v_codebook)
+    ho, hg = parity.hyper_pair(**hk)
+    params = [synth.make_param(w, i) for i in range(3)]
+    gp = [p.clone().cuda() for p in params]
+    op = [p.numpy().copy() for p in params]
+    st = B.State(list(sizes), bits_m, bits_v, block)
+    ost = [oracle.State(n, bits_m, bits_v, block) for n in sizes]
+    for t in (1, 2):
+        grads = [synth.make_grad(w, i, t) for i in range(3)]
+        B.solo_multi_step(B.TensorSet(gp, [g.cuda() for g in grads], st), hg, t)
+        for i in range(3):
+            oracle.step(op[i], synth.bf16_bits(grads[i]), ost[i], ho, t, tensor=i)
+    blob = st.export().numpy()
+    nblk = sum(-(-n // block) for n in sizes)
+    assert bytes(blob[:8]) == b"SOLOST1\0"
+    assert struct.unpack("<6i", blob[8:32].tobytes()) == (bits_m, bits_v, block, 3, v_codebook, 0)
+    assert struct.unpack("<q3q", blob[32:64].tobytes()) == (nblk, *sizes)
+    off = 64
+    pad = lambda n: (n + 15) // 16 * 16
+    for key, per in (("codes_m", block * bits_m // 8), ("codes_v", block * bits_v // 8),
+                     ("scale_m", 4), ("scale_v", 4), ("alpha", 4)):
+        want = np.concatenate([getattr(o, key).view(np.uint8) for o in ost])
+        assert want.size == nblk * per
+        assert np.array_equal(blob[off:off + want.size], want), key
+        off += pad(want.size)
+    assert off == blob.size
+    # restore into a fresh state and continue on both
+    st2 = B.State(list(sizes), bits_m, bits_v, block)
+    st2.load(torch.from_numpy(blob))
+    gp2 = [p.clone() for p in gp]
+    grads = [synth.make_grad(w, i, 3).cuda() for i in range(3)]
+    B.solo_multi_step(B.TensorSet(gp, grads, st), hg, 3)
+    B.solo_multi_step(B.TensorSet(gp2, grads, st2), hg, 3)
+    torch.cuda.synchronize()
+    assert torch.equal(st.export(), st2.export())
+    assert all(torch.equal(a, b) for a, b in zip(gp, gp2))
+    assert torch.equal(B.solo_dequant(st, 1), B.solo_dequant(st2, 1))
+    # refused: other geometry, foreign bytes, short buffer
+    other = B.State(list(sizes), bits_m, 4, block)
+    with pytest.raises(B.SoloError) as e:
+        other.load(torch.from_numpy(blob))
+    assert e.value.status == B.SOLO_ESTATE
+    with pytest.raises(B.SoloError):
+        st2.load(torch.zeros(blob.size, dtype=torch.uint8))
+    with pytest.raises(B.SoloError):
+        st2.load(torch.from_numpy(blob[:100].copy()))
+    for s_ in (st, st2, other):
+        s_.destroy()
 
 
 def test_argument_validation():

@@ -47,9 +47,9 @@ def _fresh_buffers(sizes, bits_m, bits_v, block, state0=None):
     }
 
 
-def _run_pair(B, sizes, bits_m, bits_v, block, steps, seed, state0=None):
+def _run_pair(B, sizes, bits_m, bits_v, block, steps, seed, state0=None, **hyper_kw):
     w = synth.workload(2, sizes=tuple(sizes))
-    h = B.hyper(lr=1e-3, beta1=0.6, beta2=0.999, weight_decay=0.01, seed=seed)
+    h = B.hyper(lr=1e-3, beta1=0.6, beta2=0.999, weight_decay=0.01, seed=seed, **hyper_kw)
     params = [synth.make_param(w, i) for i in range(len(sizes))]
     p_lib = [p.clone().cuda() for p in params]
     p_sta = [p.clone().cuda() for p in params]
@@ -80,6 +80,8 @@ def test_static_entry_point_matches_library_state_twice():
     sizes = (2048 * 2 + 5, 300, 4097)
     st0 = synth.make_state(sizes, 8, 4, 2048, seed=99)
     _run_pair(B, sizes, 8, 4, 2048, steps=2, seed=8, state0=st0)
+    # third: a baseline codebook for the second moment (its table also lives in the fixed array)
+    _run_pair(B, (2048 + 9, 640), 4, 4, 128, steps=2, seed=9, v_codebook=3)
 
 
 def test_static_entry_point_rejects_what_it_cannot_hold():
