@@ -222,9 +222,10 @@ float solo_default_beta1(int bits_m, int from_scratch);
 
 /*
  * Kernel selection.  0 (default): configurations with 2/3/4-bit states, block 64, 128 or 256,
- * fp32 parameters, nearest rounding of the first moment and eps >= 1e-12 run the
- * streamlined kernel, everything else the general one.  1: always the general kernel.  Both produce the same
- * packed state; the streamlined kernel's parameters differ from the IEEE sequence of
+ * the logarithmic second-moment quantizer, nearest rounding of the first moment and
+ * eps >= 1e-12 run the streamlined kernel (fp32 or bf16 parameters), everything else the
+ * general one.  1: always the general kernel.  Both produce the same packed state and the same
+ * bf16 parameters; the streamlined kernel's fp32 parameters differ from the IEEE sequence of
  * divisions and square roots by at most a few 1e-7 of the update term.  Process-wide.
  */
 int solo_set_kernel_policy(int policy);

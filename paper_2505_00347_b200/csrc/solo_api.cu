@@ -186,9 +186,9 @@ void reduce_hyper(const solo_hyper_t* h, int64_t step, int block, StepArgs& a) {
 int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
     const bool cta_group = s->block == 2048;
     solo::StepKernel k = nullptr;
-    if (g_policy.load(std::memory_order_relaxed) == 0 && !a.round_m && !a.param_bf16 && !a.tables_v &&
-        a.eps >= 1e-12f && s->tiles_total < (int64_t)1 << 31)
-        k = solo::fast_kernel(s->bits_m, s->bits_v, s->block);
+    if (g_policy.load(std::memory_order_relaxed) == 0 && !a.round_m && !a.tables_v && a.eps >= 1e-12f &&
+        s->tiles_total < (int64_t)1 << 31)
+        k = solo::fast_kernel(s->bits_m, s->bits_v, s->block, a.param_bf16 != 0);
     size_t dyn_smem = k ? solo::fast_kernel_smem() : 0;
     if (!k) k = solo::step_kernel(s->bits_m, s->bits_v, cta_group);
     if (!k) return SOLO_EINVAL;

@@ -28,13 +28,13 @@ inline int bits_index(int bits) {
 
 StepKernel step_kernel(int bits_m, int bits_v, bool cta_group);
 
-// Streamlined kernel (2/3/4-bit states, block 64, 128 or 256); null outside that domain.  The
-// caller additionally requires fp32 parameters, nearest rounding of the first moment and
-// eps >= 1e-12.
-StepKernel fast_kernel_bm2(int bv_index, int block);
-StepKernel fast_kernel_bm3(int bv_index, int block);
-StepKernel fast_kernel_bm4(int bv_index, int block);
-StepKernel fast_kernel(int bits_m, int bits_v, int block);
+// Streamlined kernel (2/3/4-bit states, block 64, 128 or 256, fp32 or bf16 parameters); null
+// outside that domain.  The caller additionally requires the logarithmic second-moment
+// quantizer, nearest rounding of the first moment and eps >= 1e-12.
+StepKernel fast_kernel_bm2(int bv_index, int block, bool param_bf16);
+StepKernel fast_kernel_bm3(int bv_index, int block, bool param_bf16);
+StepKernel fast_kernel_bm4(int bv_index, int block, bool param_bf16);
+StepKernel fast_kernel(int bits_m, int bits_v, int block, bool param_bf16);
 // Dynamic shared memory the streamlined kernels are launched with.
 size_t fast_kernel_smem();
 // Resident CTAs per SM of a step kernel launched with `dyn_smem` bytes of dynamic shared memory

@@ -1,5 +1,6 @@
 // Streamlined fused step for the common configurations: 2/3/4-bit states, blocks of
-// 64, 128 or 256 elements, fp32 parameters, nearest rounding of the first moment, eps >= 1e-12.
+// 64, 128 or 256 elements, fp32 or bf16 parameters, the paper's logarithmic quantizer for the
+// second moment, nearest rounding of the first moment, eps >= 1e-12.
 //
 // Same packed state as the general kernel (solo_device.cuh): every quantity that decides
 // a stored code (EMA values, block scales, p-quantile, base, rounded logarithm) is computed
@@ -10,9 +11,11 @@
 //     sequence gives;
 //   * the k-th smallest v^ of a block is found exactly, duplicates included, by popping one
 //     minimum per round from per-thread sorted lists.
-// The parameter update uses an approximate square root and a reciprocal refined by one
-// Newton step (quotient error below 1.5 ulp); parameters therefore agree with the IEEE
-// sequence to a few 1e-7 of the update term, not bit for bit.
+// The update of fp32 parameters uses an approximate square root and a reciprocal refined by
+// one Newton step (quotient error below 1.5 ulp); they therefore agree with the IEEE sequence
+// to a few 1e-7 of the update term, not bit for bit.  bf16 parameters (PBF) are rounded from
+// the binary32 result, where such a difference could flip a whole bf16 ulp: that variant uses
+// the IEEE square root and division and stores the same patterns as the general kernel.
 //
 // Work split: a CTA of 256 threads owns a tile of 2048 consecutive elements, a thread
 // eight of them, a block of B elements G = B/8 consecutive lanes (a quarter, half or whole warp).
@@ -52,7 +55,7 @@ struct FastShared {
     // Two stages for the inputs of a full tile, filled by bulk asynchronous copies (TMA, issued by
     // one thread) one tile ahead of their use; each stage has its own mbarrier.
     struct Stage {
-        float4 p[2 * CTA];                   // 2048 parameters
+        float4 p[2 * CTA];                   // 2048 parameters (bf16: the first half)
         uint4 g[CTA];                        // 2048 bf16 gradients
         uint32_t cm[CTA + 4];                // packed codes of the tile, from a 16-byte boundary (64 * bits words + 2)
         uint32_t cv[CTA + 4];
@@ -220,18 +223,19 @@ __device__ __forceinline__ uint32_t warp_load_codes(const uint8_t* warp_base, in
 // first block is odd) and scalars are copied from the 16-byte boundary at or below them, with 16
 // bytes more when they do not start on it; readers add the offset.  The scalar arrays are
 // allocated in multiples of 16 bytes, so the copy never leaves them.
-template <int BM, int BV, int G>
+template <int BM, int BV, int G, bool PBF>
 __device__ __forceinline__ void issue_tile_copy(const StepArgs& a, FastShared& s, uint32_t fill, const char* pt,
                                                 const char* gt, int64_t jb_tile) {
     constexpr int NG = CTA / G;
+    constexpr uint32_t PBYTES = TILE * (PBF ? 2 : 4);
     FastShared::Stage& st = s.stage[fill & 1u];
     const uint32_t bar = smem_u32(&s.mbar[fill & 1u]);
     const int64_t bm0 = jb_tile * G * BM, bv0 = jb_tile * G * BV;   // byte offsets of the tile's codes
     const uint32_t bytes_m = CTA * BM + ((bm0 & 15) ? 16u : 0u), bytes_v = CTA * BV + ((bv0 & 15) ? 16u : 0u);
     const uint32_t bytes_s = (NG + ((jb_tile & 3) ? 4u : 0u)) * 4u;
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar),
-                 "r"((uint32_t)(TILE * 4 + TILE * 2) + bytes_m + bytes_v + 3u * bytes_s) : "memory");
-    bulk_copy(st.p, pt, TILE * 4, bar);
+                 "r"((uint32_t)(PBYTES + TILE * 2) + bytes_m + bytes_v + 3u * bytes_s) : "memory");
+    bulk_copy(st.p, pt, PBYTES, bar);
     bulk_copy(st.g, gt, TILE * 2, bar);
     bulk_copy(st.cm, a.codes_m + (bm0 & ~(int64_t)15), bytes_m, bar);
     bulk_copy(st.cv, a.codes_v + (bv0 & ~(int64_t)15), bytes_v, bar);
@@ -360,7 +364,7 @@ __device__ __forceinline__ void bar_sync(int id) {
 // was measured slower: the extra instructions cost more than the hidden latency gains, the
 // four resident CTAs per SM cover each other's load phases.
 
-template <int BM, int BV, int G, bool FULL>
+template <int BM, int BV, int G, bool FULL, bool PBF>
 __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, const float* s_y,
                                           const float* s_mid, char* pbase, const char* gbase,
                                           const int64_t n, const int tin, const int64_t jb_tile,
@@ -368,6 +372,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
                                           const int next_dtin) {
     constexpr int KM = 1 << BM, KV = 1 << BV;
     constexpr int NG = CTA / G, B = G * EPT;
+    constexpr int PSZ = PBF ? 2 : 4;                            // bytes per parameter
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gl = tid & (G - 1), grp = tid / G;
     const bool hi = G < 32 && (lane & G) != 0;                  // odd group of its pair
@@ -380,7 +385,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     const int nb = FULL ? B : (int)max((int64_t)0, min((int64_t)B, rem_tile - (int64_t)grp * B));
     const int nv = FULL ? EPT : (int)max((int64_t)0, min((int64_t)EPT, rem_tile - (int64_t)tid * EPT));
 
-    char* const pt = pbase + tile_elem0 * 4;                    // the tile's parameters and gradients
+    char* const pt = pbase + tile_elem0 * PSZ;                  // the tile's parameters and gradients
     const char* const gt = gbase + tile_elem0 * 2;
     const int64_t tile_slot0 = jb_tile * G;                     // slot = 8 elements = one thread's codes
     const int64_t jb = jb_tile + grp;
@@ -400,9 +405,9 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
         // refilled all threads have finished reading it: they read at the start of a tile and
         // pass that tile's barriers before any thread starts the next one.
         if (tid == 0) {
-            if (!ah.staged) issue_tile_copy<BM, BV, G>(a, s, ah.fill, pt, gt, jb_tile);
+            if (!ah.staged) issue_tile_copy<BM, BV, G, PBF>(a, s, ah.fill, pt, gt, jb_tile);
             if (next_full)
-                issue_tile_copy<BM, BV, G>(a, s, ah.fill + 1u, pt + (int64_t)next_dtin * (TILE * 4),
+                issue_tile_copy<BM, BV, G, PBF>(a, s, ah.fill + 1u, pt + (int64_t)next_dtin * (TILE * PSZ),
                                            gt + (int64_t)next_dtin * (TILE * 2), jb_tile + (int64_t)next_dtin * NG);
         }
         const uint32_t mine = ah.fill;
@@ -416,7 +421,19 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
         }
         const FastShared::Stage& st = s.stage[mine & 1u];
         const uint4 gw = st.g[tid];
-        const float4 p0 = st.p[2 * tid], p1 = st.p[2 * tid + 1];
+        if constexpr (PBF) {
+            const uint4 pw = reinterpret_cast<const uint4*>(st.p)[tid];
+            const uint32_t pp[4] = {pw.x, pw.y, pw.z, pw.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                p[2 * i] = __uint_as_float(pp[i] << 16);
+                p[2 * i + 1] = __uint_as_float(pp[i] & 0xffff0000u);
+            }
+        } else {
+            const float4 p0 = st.p[2 * tid], p1 = st.p[2 * tid + 1];
+            p[0] = p0.x; p[1] = p0.y; p[2] = p0.z; p[3] = p0.w;
+            p[4] = p1.x; p[5] = p1.y; p[6] = p1.z; p[7] = p1.w;
+        }
         const int wm = (int)((jb_tile * G * BM) & 15) >> 2, wv = (int)((jb_tile * G * BV) & 15) >> 2;   // word offsets
         if constexpr (BM == 2) cm = reinterpret_cast<const uint16_t*>(st.cm + wm)[tid];
         else if constexpr (BM == 4) cm = st.cm[wm + tid];
@@ -432,15 +449,16 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
             g[2 * i] = __uint_as_float(gg[i] << 16);
             g[2 * i + 1] = __uint_as_float(gg[i] & 0xffff0000u);
         }
-        p[0] = p0.x; p[1] = p0.y; p[2] = p0.z; p[3] = p0.w;
-        p[4] = p1.x; p[5] = p1.y; p[6] = p1.z; p[7] = p1.w;
     } else {
 #pragma unroll
         for (int i = 0; i < EPT; ++i) {
             p[i] = 0.0f; g[i] = 0.0f;
             if (i < nv) {
                 g[i] = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(gt)[tid * EPT + i] << 16);
-                p[i] = reinterpret_cast<const float*>(pt)[tid * EPT + i];
+                if constexpr (PBF)
+                    p[i] = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(pt)[tid * EPT + i] << 16);
+                else
+                    p[i] = reinterpret_cast<const float*>(pt)[tid * EPT + i];
             }
         }
         if (have_block) {
@@ -506,7 +524,39 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
 
     // Adam(W) update of element i and, after every fourth, the store; issued between the
     // rounds of the selection below, which it does not depend on
+    const uint64_t ctr = (uint64_t)(uint32_t)tin * (TILE / EPT) + (uint32_t)tid;   // element index / 8
+    uint32_t wp[4] = {0u, 0u, 0u, 0u};                          // draws of the stochastic bf16 rounding
+    const bool sr = PBF && a.param_sr;
+    if (PBF && !FULL && sr)
+        philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, (uint32_t)tensor * 4u + 2u, a.rk, wp);
     auto update = [&](int i) {
+        if constexpr (PBF) {
+            const float den = __fmaf_rn(__fsqrt_rn(vh[i]), a.inv_sqrt_bc2, a.eps);
+            p[i] = __fmaf_rn(-a.step_size, __fdiv_rn(mh[i], den), p[i] * a.decay);
+            if (FULL) {
+                if (i == 7) {
+                    uint32_t pp[4];
+                    if (sr) {
+                        philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, (uint32_t)tensor * 4u + 2u, a.rk, wp);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            pp[j] = bf16_sr(p[2 * j], wp[j] & 0xFFFFu) | (bf16_sr(p[2 * j + 1], wp[j] >> 16) << 16);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(p[2 * j], p[2 * j + 1]);
+                            pp[j] = *reinterpret_cast<const uint32_t*>(&h);
+                        }
+                    }
+                    __stcs(reinterpret_cast<uint4*>(pt) + tid, make_uint4(pp[0], pp[1], pp[2], pp[3]));
+                }
+            } else if (i < nv) {
+                reinterpret_cast<uint16_t*>(pt)[tid * EPT + i] =
+                    sr ? (uint16_t)bf16_sr(p[i], draw16(wp, i))
+                       : __bfloat16_as_ushort(__float2bfloat16_rn(p[i]));
+            }
+            return;
+        }
         const float den = __fmaf_rn(sqrt_approx(vh[i]), a.inv_sqrt_bc2, a.eps);
         const float rc = rcp_approx(den);
         const float q0 = mh[i] * rc;
@@ -551,7 +601,6 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     if (gl == 0) s.xin[par][grp] = make_uint4(mx_m, mx_v, x_p, 0u);
     bar_sync(1);
     uint32_t w[4] = {0u, 0u, 0u, 0u};
-    const uint64_t ctr = (uint64_t)(uint32_t)tin * (TILE / EPT) + (uint32_t)tid;   // element index / 8
     if (warp != 0) {
         if (a.round_v) philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, (uint32_t)tensor * 4u, a.rk, w);
     } else if (tid < NG) {
@@ -686,7 +735,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     }
 }
 
-template <int BM, int BV, int G>
+template <int BM, int BV, int G, bool PBF>
 __global__ void __launch_bounds__(CTA, 4) solo_step_fast_kernel(const StepArgs a) {
     constexpr int KM = 1 << BM;
     extern __shared__ __align__(16) unsigned char fast_smem[];   // sizeof(FastShared), above the static 48 KB limit
@@ -737,10 +786,10 @@ __global__ void __launch_bounds__(CTA, 4) solo_step_fast_kernel(const StepArgs a
         const int tin = tile - t_lo;
         const int64_t jb_tile = jb0 + (int64_t)tin * (CTA / G);
         if (tin < full_tiles)
-            fast_tile<BM, BV, G, true>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, ah,
+            fast_tile<BM, BV, G, true, PBF>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, ah,
                                        tin + stride < full_tiles, stride);
         else
-            fast_tile<BM, BV, G, false>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, ah, false, 0);
+            fast_tile<BM, BV, G, false, PBF>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, ah, false, 0);
         par ^= 1;
     }
     // every copy that was issued has been waited for by the thread that issued it, unless that

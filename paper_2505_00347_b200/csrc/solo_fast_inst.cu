@@ -11,14 +11,17 @@
 
 namespace solo {
 
-StepKernel SOLO_CAT(fast_kernel_bm, SOLO_BM)(int bv_index, int block) {
-    static const StepKernel table[3][3] = {
-        {solo_step_fast_kernel<SOLO_BM, 2, 8>, solo_step_fast_kernel<SOLO_BM, 2, 16>, solo_step_fast_kernel<SOLO_BM, 2, 32>},
-        {solo_step_fast_kernel<SOLO_BM, 3, 8>, solo_step_fast_kernel<SOLO_BM, 3, 16>, solo_step_fast_kernel<SOLO_BM, 3, 32>},
-        {solo_step_fast_kernel<SOLO_BM, 4, 8>, solo_step_fast_kernel<SOLO_BM, 4, 16>, solo_step_fast_kernel<SOLO_BM, 4, 32>},
+#define SOLO_ROW(BV, PBF)                                                                  \
+    {solo_step_fast_kernel<SOLO_BM, BV, 8, PBF>, solo_step_fast_kernel<SOLO_BM, BV, 16, PBF>, \
+     solo_step_fast_kernel<SOLO_BM, BV, 32, PBF>}
+
+StepKernel SOLO_CAT(fast_kernel_bm, SOLO_BM)(int bv_index, int block, bool param_bf16) {
+    static const StepKernel table[2][3][3] = {
+        {SOLO_ROW(2, false), SOLO_ROW(3, false), SOLO_ROW(4, false)},
+        {SOLO_ROW(2, true), SOLO_ROW(3, true), SOLO_ROW(4, true)},
     };
     if (bv_index < 0 || bv_index > 2 || (block != 64 && block != 128 && block != 256)) return nullptr;
-    return table[bv_index][block == 64 ? 0 : block == 128 ? 1 : 2];
+    return table[param_bf16 ? 1 : 0][bv_index][block == 64 ? 0 : block == 128 ? 1 : 2];
 }
 
 #if SOLO_BM == 2

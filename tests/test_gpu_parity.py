@@ -90,6 +90,23 @@ def test_baseline_second_moment_codebooks(sel, bits_v, block):
     run_lockstep(sizes, 4, bits_v, block, hk, 3, gf, params)
 
 
+@pytest.mark.parametrize("param_round", [0, 1])
+@pytest.mark.parametrize("bits_m,bits_v,block", [(2, 3, 128), (4, 4, 64), (3, 2, 256), (4, 3, 2048)])
+def test_bf16_parameters_every_kernel(bits_m, bits_v, block, param_round):
+    """bf16 parameters through the streamlined kernel (full tiles from the staged copies, ragged
+    tails from direct loads) and the general one, nearest and stochastic rounding; run_lockstep
+    compares the stored bf16 patterns bit for bit."""
+    sizes = (2048 * 5 + block * 3 + 1, 77, 2048 * 2, 2048 + 8)
+    w = synth.workload(2, sizes=sizes)
+    params = [synth.make_param(w, i, dtype=torch.bfloat16) for i in range(len(sizes))]
+    gf = lambda t: [synth.make_grad(w, i, t) for i in range(len(sizes))]
+    hk = dict(lr=1e-2, beta1=0.6, beta2=0.999, weight_decay=0.01, seed=41, param_dtype=1,
+              param_round=param_round)
+    st0 = synth.make_state(sizes, bits_m, bits_v, block, seed=block + bits_m)
+    run_lockstep(sizes, bits_m, bits_v, block, hk, 2, gf, params, state0=st0)
+    run_lockstep(sizes, bits_m, bits_v, block, hk, 3, gf, params)
+
+
 def test_stochastic_bf16_rounding_is_unbiased_on_the_device():
     """Updates of 1/64 ulp(bf16): nearest rounding leaves every parameter where it is, stochastic
     rounding moves the mean by the update (first Adam step from zero state: p += lr exactly)."""
@@ -272,11 +289,14 @@ def test_argument_validation():
     multi.destroy()
 
 
-def _full_size_sampled(cfg: int, random_per_tensor: int, need_bytes: float, overrides=None, step: int = 3):
+def _full_size_sampled(cfg: int, random_per_tensor: int, need_bytes: float, overrides=None, step: int = 3,
+                       param_bf16: int = 0):
     """A benchmark workload at its full size, one solo_multi_step launch in the configuration
     bench.py times, from a seeded random packed state.  Blocks are independent, so the oracle
     recomputes a sample of them one by one from copies of their inputs taken before the step:
-    the first and the last block of every tensor plus `random_per_tensor` random ones."""
+    the first and the last block of every tensor plus `random_per_tensor` random ones.
+    param_bf16: 0 fp32 parameters, 1 bf16 rounded to nearest, 2 bf16 rounded stochastically (the
+    stored patterns are then compared bit for bit)."""
     from paper_2505_00347_b200 import binding as B
     free, _ = torch.cuda.mem_get_info()
     if free < need_bytes:
@@ -284,7 +304,8 @@ def _full_size_sampled(cfg: int, random_per_tensor: int, need_bytes: float, over
     w = synth.workload(cfg, **(overrides or {}))
     bm, bv, block = w.bits_m, w.bits_v, w.block
     dev = torch.device("cuda")
-    params = [synth.make_param(w, i, device=dev) for i in range(len(w.sizes))]
+    pdtype = torch.bfloat16 if param_bf16 else torch.float32
+    params = [synth.make_param(w, i, device=dev, dtype=pdtype) for i in range(len(w.sizes))]
     grads = [synth.make_grad(w, i, 1, device=dev) for i in range(len(w.sizes))]
     st0 = synth.make_state(w.sizes, bm, bv, block, seed=33 + cfg, device=dev)
     gstate = B.State(list(w.sizes), bm, bv, block)
@@ -306,7 +327,8 @@ def _full_size_sampled(cfg: int, random_per_tensor: int, need_bytes: float, over
         lo, hi = j * block, min(w.sizes[t], (j + 1) * block)
         jb = int(bstart[t]) + j
         before.append(dict(
-            p=params[t][lo:hi].cpu().numpy().copy(), g=synth.bf16_bits(grads[t][lo:hi]),
+            p=(synth.bf16_bits(params[t][lo:hi]) if param_bf16 else params[t][lo:hi].cpu().numpy().copy()),
+            g=synth.bf16_bits(grads[t][lo:hi]),
             codes_m=st0["codes_m"][jb * sm:(jb + 1) * sm].cpu().numpy().copy(),
             codes_v=st0["codes_v"][jb * sv:(jb + 1) * sv].cpu().numpy().copy(),
             scale_m=st0["scale_m"][jb:jb + 1].cpu().numpy().copy(),
@@ -314,6 +336,8 @@ def _full_size_sampled(cfg: int, random_per_tensor: int, need_bytes: float, over
             alpha=st0["alpha"][jb:jb + 1].cpu().numpy().copy()))
     del st0
     kw = dict(lr=w.lr, beta1=w.beta1, beta2=w.beta2, weight_decay=w.weight_decay, seed=1234)
+    if param_bf16:
+        kw.update(param_dtype=1, param_round=1 if param_bf16 == 2 else 0)
     ho, hg = parity.hyper_pair(**kw)
     B.solo_multi_step(B.TensorSet(params, grads, gstate), hg, step)
     torch.cuda.synchronize()
@@ -338,6 +362,9 @@ def _full_size_sampled(cfg: int, random_per_tensor: int, need_bytes: float, over
         assert np.array_equal(fetch("codes_v", jb * sv, sv, np.uint8), ost.codes_v), (t, j)
         for k in ("scale_m", "scale_v", "alpha"):
             assert np.array_equal(fetch(k, jb * 4, 4, np.uint32), getattr(ost, k).view(np.uint32)), (t, j, k)
+        if param_bf16:
+            assert np.array_equal(synth.bf16_bits(params[t][j * block: j * block + n]), p), (t, j)
+            continue
         gp = params[t][j * block: j * block + n].cpu().numpy()
         err = np.abs(gp.astype(np.float64) - p)
         # random states pair huge first moments with tiny second moments: allow the streamlined
@@ -353,6 +380,11 @@ def _full_size_sampled(cfg: int, random_per_tensor: int, need_bytes: float, over
 def test_full_size_7b_set_sampled_blocks():
     """LLaMA-7B-shaped set, 6.74 B parameters, 2-bit / 3-bit, block 128 (the headline workload)."""
     _full_size_sampled(3, 12, 60e9)
+
+
+def test_full_size_7b_set_bf16_parameters_stochastic_rounding():
+    """The same set with bf16 parameters rounded stochastically (streamlined kernel, IEEE update)."""
+    _full_size_sampled(3, 6, 45e9, param_bf16=2)
 
 
 def test_full_size_ragged_set_sampled_blocks():
