@@ -28,7 +28,7 @@ inline int bits_index(int bits) {
 
 StepKernel step_kernel(int bits_m, int bits_v, bool cta_group);
 
-// Streamlined kernel (2/3/4-bit states, block 64, 128 or 256, fp32 or bf16 parameters); null
+// Streamlined kernel (2/3/4-bit states, block 64, 128, 256 or 2048, fp32 or bf16 parameters); null
 // outside that domain.  The caller additionally requires the logarithmic second-moment
 // quantizer, nearest rounding of the first moment and eps >= 1e-12.
 StepKernel fast_kernel_bm2(int bv_index, int block, bool param_bf16);

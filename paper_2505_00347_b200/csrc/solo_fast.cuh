@@ -1,5 +1,5 @@
 // Streamlined fused step for the common configurations: 2/3/4-bit states, blocks of
-// 64, 128 or 256 elements, fp32 or bf16 parameters, the paper's logarithmic quantizer for the
+// 64, 128, 256 or 2048 elements, fp32 or bf16 parameters, the paper's logarithmic quantizer for the
 // second moment, nearest rounding of the first moment, eps >= 1e-12.
 //
 // Same packed state as the general kernel (solo_device.cuh): every quantity that decides
@@ -18,7 +18,8 @@
 // the IEEE square root and division and stores the same patterns as the general kernel.
 //
 // Work split: a CTA of 256 threads owns a tile of 2048 consecutive elements, a thread
-// eight of them, a block of B elements G = B/8 consecutive lanes (a quarter, half or whole warp).
+// eight of them, a block of B elements G = B/8 consecutive lanes (a quarter, half or whole warp;
+// G = 256: the whole CTA, with CTA-wide maxima and a radix select instead of the warp collectives).
 // The per-block scalar work (reciprocals of the scales, base of the logarithmic codebook
 // and its logarithm) is done once per block by the first warp for the whole tile and
 // passed through shared memory.
@@ -52,6 +53,7 @@ struct FastShared {
     uint4 xin[2][CTA / 8];                  // per group: bits of Delta_m', Delta_v', x_p
     float4 xout[2][CTA / 8];                // per group: 1/Delta_m', 1/Delta_v', 1/log2(alpha'), rounding limit
     uint32_t xflag[2][CTA / 8];             // bit 0: vanishing first moment, bit 1: vanishing second moment
+    uint32_t red[2][16];                    // G = 256: per-warp maxima of |m^| (0..7) and v^ (8..15)
     // Two stages for the inputs of a full tile, filled by bulk asynchronous copies (TMA, issued by
     // one thread) one tile ahead of their use; each stage has its own mbarrier.
     struct Stage {
@@ -232,7 +234,9 @@ __device__ __forceinline__ void issue_tile_copy(const StepArgs& a, FastShared& s
     const uint32_t bar = smem_u32(&s.mbar[fill & 1u]);
     const int64_t bm0 = jb_tile * G * BM, bv0 = jb_tile * G * BV;   // byte offsets of the tile's codes
     const uint32_t bytes_m = CTA * BM + ((bm0 & 15) ? 16u : 0u), bytes_v = CTA * BV + ((bv0 & 15) ? 16u : 0u);
-    const uint32_t bytes_s = (NG + ((jb_tile & 3) ? 4u : 0u)) * 4u;
+    // NG >= 8 scalars from the boundary below the first (16 bytes more when it is not on it); a
+    // single block's scalar (NG = 1) lies within the 16 bytes that start at that boundary
+    const uint32_t bytes_s = NG >= 4 ? (NG + ((jb_tile & 3) ? 4u : 0u)) * 4u : 16u;
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar),
                  "r"((uint32_t)(PBYTES + TILE * 2) + bytes_m + bytes_v + 3u * bytes_s) : "memory");
     bulk_copy(st.p, pt, PBYTES, bar);
@@ -352,6 +356,49 @@ __device__ __forceinline__ uint32_t select_kth(uint32_t head, const uint32_t* co
         }
     }
     return ans;
+}
+
+// k-th smallest (1-based, duplicates counted) of the CTA's 2048 keys, eight per thread: radix
+// select from the top, 8 bits per pass, one histogram bin per thread.  Keys are below 2^31 or
+// the all-ones filler of elements that do not exist (k never reaches those).  `hist` is 272
+// words of shared memory.  Every thread of the CTA calls it; all return the same key.
+__device__ __forceinline__ uint32_t cta_select(const uint32_t (&key)[EPT], int k, uint32_t* hist) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint32_t* const scan = hist + 256;           // [0..7] warp totals, [8] chosen bin, [9] rank within it
+    uint32_t prefix = 0;
+    uint32_t kk = (uint32_t)k;
+#pragma unroll 1
+    for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        __syncthreads();                           // the bins and scan[] of the pass before are read
+        hist[tid] = 0;
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < EPT; ++i)
+            if (pass == 0 || (key[i] >> (shift + 8)) == prefix) atomicAdd(&hist[(key[i] >> shift) & 255u], 1u);
+        __syncthreads();
+        const uint32_t c = hist[tid];
+        uint32_t incl = c;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += t;
+        }
+        if (lane == 31) scan[warp] = incl;
+        __syncthreads();
+#pragma unroll
+        for (int w = 0; w < 7; ++w)
+            if (w < warp) incl += scan[w];
+        const uint32_t excl = incl - c;
+        if (kk > excl && kk <= incl) {             // exactly one bin holds the rank
+            scan[8] = (uint32_t)tid;
+            scan[9] = kk - excl;
+        }
+        __syncthreads();
+        prefix = (prefix << 8) | scan[8];
+        kk = scan[9];
+    }
+    return prefix;
 }
 
 __device__ __forceinline__ void bar_sync(int id) {
@@ -484,7 +531,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
         for (int r0 = 0; r0 < KM; r0 += G)
             if (r0 + gl < KM) tab[KV + r0 + gl] = s_y[r0 + gl] * dm;
     }
-    __syncwarp();
+    if constexpr (G == CTA) __syncthreads(); else __syncwarp();
 
     if (a.l2) {
 #pragma unroll
@@ -571,30 +618,57 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     };
 
     // ---- block scales and the p-quantile of v^ (Sec. 3.2.2) ----
-    mx_m = seg_max31<G>(mx_m, hi);
-    mx_v = seg_max31<G>(mx_v, hi);
     uint32_t x_p = 0;
-    if (a.fixed_alpha > 0.0f) {                                  // fixed base: no quantile to find
+    if constexpr (G == CTA) {
+        // one block per tile: maxima over the CTA through shared memory, radix select
+        mx_m = __reduce_max_sync(0xffffffffu, mx_m);
+        mx_v = __reduce_max_sync(0xffffffffu, mx_v);
+        if (lane == 0) {
+            s.red[par][warp] = mx_m;
+            s.red[par][8 + warp] = mx_v;
+        }
 #pragma unroll
         for (int i = 0; i < EPT; ++i) update(i);
-    } else {
-        uint32_t key[EPT];
+        __syncthreads();
+        const uint32_t t = s.red[par][lane & 15];
+        mx_m = __reduce_max_sync(0xffffffffu, (lane & 8) ? 0u : t);
+        mx_v = __reduce_max_sync(0xffffffffu, (lane & 8) ? t : 0u);
+        if (!(a.fixed_alpha > 0.0f)) {
+            uint32_t key[EPT];
 #pragma unroll
-        for (int i = 0; i < EPT; ++i) key[i] = (FULL || i < nv) ? __float_as_uint(vh[i]) : KEY_MAX;
-        sort8(key);
-        uint32_t* const col = &s.sort[0][tid];
-#pragma unroll
-        for (int j = 1; j < EPT; ++j) col[(j - 1) * CTA] = key[j] ^ vflip;
-        const uint32_t head = key[0] ^ vflip;
-        uint32_t xv;
-        if (FULL) {
-            xv = select_kth<G, true>(head, col, a.k_full, hi, update);
-        } else {
-            int k = (int)ceil((double)a.p_quantile * (double)nb);
-            k = min(max(k, 1), nb);                              // 0 for a group without a block
-            xv = select_kth<G, false>(head, col, k, hi, update);
+            for (int i = 0; i < EPT; ++i) key[i] = (FULL || i < nv) ? __float_as_uint(vh[i]) : 0xFFFFFFFFu;
+            int k = a.k_full;
+            if (!FULL) {
+                k = (int)ceil((double)a.p_quantile * (double)nb);
+                k = min(max(k, 1), nb);
+            }
+            x_p = cta_select(key, k, &s.sort[0][0]);
         }
-        x_p = xv ^ vflip;
+    } else {
+        mx_m = seg_max31<G>(mx_m, hi);
+        mx_v = seg_max31<G>(mx_v, hi);
+        if (a.fixed_alpha > 0.0f) {                                  // fixed base: no quantile to find
+#pragma unroll
+            for (int i = 0; i < EPT; ++i) update(i);
+        } else {
+            uint32_t key[EPT];
+#pragma unroll
+            for (int i = 0; i < EPT; ++i) key[i] = (FULL || i < nv) ? __float_as_uint(vh[i]) : KEY_MAX;
+            sort8(key);
+            uint32_t* const col = &s.sort[0][tid];
+#pragma unroll
+            for (int j = 1; j < EPT; ++j) col[(j - 1) * CTA] = key[j] ^ vflip;
+            const uint32_t head = key[0] ^ vflip;
+            uint32_t xv;
+            if (FULL) {
+                xv = select_kth<G, true>(head, col, a.k_full, hi, update);
+            } else {
+                int k = (int)ceil((double)a.p_quantile * (double)nb);
+                k = min(max(k, 1), nb);                              // 0 for a group without a block
+                xv = select_kth<G, false>(head, col, k, hi, update);
+            }
+            x_p = xv ^ vflip;
+        }
     }
 
     // ---- per-block scalars, once per block, by the first warp; the others draw xi meanwhile ----

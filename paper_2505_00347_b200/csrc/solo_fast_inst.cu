@@ -13,15 +13,16 @@ namespace solo {
 
 #define SOLO_ROW(BV, PBF)                                                                  \
     {solo_step_fast_kernel<SOLO_BM, BV, 8, PBF>, solo_step_fast_kernel<SOLO_BM, BV, 16, PBF>, \
-     solo_step_fast_kernel<SOLO_BM, BV, 32, PBF>}
+     solo_step_fast_kernel<SOLO_BM, BV, 32, PBF>, solo_step_fast_kernel<SOLO_BM, BV, 256, PBF>}
 
 StepKernel SOLO_CAT(fast_kernel_bm, SOLO_BM)(int bv_index, int block, bool param_bf16) {
-    static const StepKernel table[2][3][3] = {
+    static const StepKernel table[2][3][4] = {
         {SOLO_ROW(2, false), SOLO_ROW(3, false), SOLO_ROW(4, false)},
         {SOLO_ROW(2, true), SOLO_ROW(3, true), SOLO_ROW(4, true)},
     };
-    if (bv_index < 0 || bv_index > 2 || (block != 64 && block != 128 && block != 256)) return nullptr;
-    return table[param_bf16 ? 1 : 0][bv_index][block == 64 ? 0 : block == 128 ? 1 : 2];
+    const int g = block == 64 ? 0 : block == 128 ? 1 : block == 256 ? 2 : block == 2048 ? 3 : -1;
+    if (bv_index < 0 || bv_index > 2 || g < 0) return nullptr;
+    return table[param_bf16 ? 1 : 0][bv_index][g];
 }
 
 #if SOLO_BM == 2

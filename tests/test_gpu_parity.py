@@ -150,7 +150,8 @@ def test_quantile_ranks_and_ties_on_full_tiles():
         gs[1][2048:4096:2] = 0.0            # half zeros: the quantile sits on a tie
         return gs
 
-    for p_q, block in ((0.1, 128), (0.0, 64), (0.3, 256), (0.05, 128), (0.9, 64)):
+    for p_q, block in ((0.1, 128), (0.0, 64), (0.3, 256), (0.05, 128), (0.9, 64), (0.1, 2048), (0.0, 2048),
+                       (0.95, 2048)):
         hk = dict(seed=5, p_quantile=p_q, weight_decay=0.0)
         run_lockstep(sizes, 2, 3, block, hk, 3, gf, params)
         run_lockstep(sizes, 4, 2, block, hk, 2, gf, params)
