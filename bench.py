@@ -178,24 +178,34 @@ def run_ours(args, rank, world):
     clk = clocks.stop() if rank == 0 else None
     assert state.status() == 0
 
-    # end to end: gradients come from pinned host memory, updated parameters go back to it
+    # end to end through the host-buffer entry point: every step the gradients are read from pinned
+    # host memory and the updated parameters are written back to it (chunked, three streams)
     pbytes = 2 if args.param_bf16 else 4
-    e2e_ms, h2d, d2h = None, 2 * n, pbytes * n
+    e2e_ms, h2d, d2h, e2e_buffers = None, 2 * n, pbytes * n, None
     if not args.no_e2e:
-        big = max(w.sizes)
-        hg = torch.empty(big, dtype=torch.bfloat16).pin_memory()
-        hp = torch.empty(big, dtype=params[0].dtype).pin_memory()
-        hg[: grads[0].numel()].copy_(grads[0][: big].cpu())
+        try:                                     # one pinned buffer per tensor
+            hgs = [torch.empty(g.numel(), dtype=torch.bfloat16, pin_memory=True) for g in grads]
+            hps = [torch.empty(p.numel(), dtype=p.dtype, pin_memory=True) for p in params]
+            e2e_buffers = "one pinned host buffer per tensor"
+        except RuntimeError:                     # not enough page-locked memory: all tensors share one
+            hgs = hps = None
+            big = max(w.sizes)
+            hg = torch.empty(big, dtype=torch.bfloat16, pin_memory=True)
+            hp = torch.empty(big, dtype=params[0].dtype, pin_memory=True)
+            hgs = [hg[: g.numel()] for g in grads]
+            hps = [hp[: p.numel()] for p in params]
+            e2e_buffers = "all tensors share one pinned host buffer (same bytes moved)"
+        for hgt, g in zip(hgs, grads):
+            hgt.copy_(g)
         sync_all()
         k = max(1, min(args.steps, args.e2e_steps))
+        step_no += 1
+        B.solo_multi_step_host(params, hgs, hps, state, h, step_no)       # allocates the staging slots
+        sync_all()
         e0.record(stream)
         for _ in range(k):
             step_no += 1
-            for g in grads:
-                g.copy_(hg[: g.numel()], non_blocking=True)
-            B.solo_multi_step(ts, h, step_no)
-            for p in params:
-                hp[: p.numel()].copy_(p, non_blocking=True)
+            B.solo_multi_step_host(params, hgs, hps, state, h, step_no)
         e1.record(stream)
         sync_all()
         e2e_ms = e0.elapsed_time(e1) / k
@@ -233,7 +243,8 @@ def run_ours(args, rank, world):
     }
     if e2e_ms is not None:
         out["e2e"] = {"value": round(world * n / (e2e_max * 1e-3) / 1e9, 3), "unit": UNIT,
-                      "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+                      "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                      "call": "solo_multi_step_host", "buffers": e2e_buffers}
     if world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(w, args.cpu_sample)
     return out

@@ -156,6 +156,40 @@ int solo_multi_step(const solo_tensor_list_t* list, const solo_hyper_t* hyper, i
                     void* stream);
 
 /*
+ * The same step for a worker whose gradients arrive in HOST memory and that wants a HOST copy
+ * of the updated parameters (the paper has no counterpart: it does not discuss where the
+ * tensors live).  The parameters and the state stay resident on the device.  Every pointer
+ * of the descriptor is a HOST array of num_tensors entries:
+ *   param_dev[t]       DEVICE pointer of tensor t's parameters, 16-byte aligned, updated in place
+ *   grad_host[t]       HOST pointer of its bf16 gradients (page-locked memory for overlap)
+ *   param_out_host[t]  HOST pointer that receives the updated parameters (same type as the
+ *                      parameters); the array may be NULL: nothing is copied back
+ *   numel[t]           element counts, equal to the state's
+ *   chunk_elems        elements per pipeline chunk, rounded down to whole 2048-element tiles;
+ *                      0: 16 Mi
+ * The tensor list is cut into chunks of whole tiles.  For each chunk the gradients are copied to
+ * one of three device staging slots, the step kernel runs on the chunk's tiles, and the chunk's
+ * updated parameters are copied out; each slot has its own stream, so the upload of one chunk,
+ * the kernel of another and the download of a third overlap.  All of it is ordered after the
+ * work queued on `stream` at the call, and `stream` waits for the last chunk.  The call itself
+ * returns once all but the last three chunks have completed (it reuses page-locked staging).
+ * The first call on a state, and a call with another chunk size, synchronize the device and
+ * allocate the slots (3 x chunk_elems x 2 bytes) with cudaMalloc; they are freed with the state.
+ * Results are identical to solo_multi_step on the same inputs.
+ */
+typedef struct {
+    int32_t num_tensors;
+    void* const* param_dev;
+    const void* const* grad_host;
+    void* const* param_out_host;
+    const int64_t* numel;
+    int64_t chunk_elems;
+    solo_state_t* state;
+} solo_host_list_t;
+int solo_multi_step_host(const solo_host_list_t* list, const solo_hyper_t* hyper, int64_t step,
+                         void* stream);
+
+/*
  * Eq. 2 for inspection: writes the dequantized moment of every element, tensors
  * concatenated without padding (sum of numel floats).
  *   which  0: first moment y[q] * Delta_m;  1: second moment alpha^q * Delta_v, or

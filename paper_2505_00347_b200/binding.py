@@ -47,6 +47,16 @@ class TensorList(C.Structure):
     ]
 
 
+class HostList(C.Structure):
+    """solo_host_list_t: every pointer is a host array"""
+
+    _fields_ = [
+        ("num_tensors", C.c_int32), ("param_dev", C.c_void_p), ("grad_host", C.c_void_p),
+        ("param_out_host", C.c_void_p), ("numel", C.c_void_p), ("chunk_elems", C.c_int64),
+        ("state", C.c_void_p),
+    ]
+
+
 class RawState(C.Structure):
     """solo_raw_state_t: caller-owned state buffers for solo_multi_step_static"""
 
@@ -99,6 +109,8 @@ def lib() -> C.CDLL:
     L.solo_multi_step_static.argtypes = [C.c_int32, vp, vp, C.POINTER(C.c_int64), C.POINTER(RawState),
                                          C.POINTER(Hyper), i64, vp]
     L.solo_multi_step_static.restype = C.c_int
+    L.solo_multi_step_host.argtypes = [C.POINTER(HostList), C.POINTER(Hyper), i64, vp]
+    L.solo_multi_step_host.restype = C.c_int
     L.solo_state_export_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
     L.solo_state_export.argtypes = [vp, vp, C.c_size_t, vp]
     L.solo_state_import.argtypes = [vp, vp, C.c_size_t, vp]
@@ -316,6 +328,34 @@ def solo_multi_step_static(params: list[torch.Tensor], grads: list[torch.Tensor]
     _check(lib().solo_multi_step_static(len(sizes), param_ptrs.data_ptr(), grad_ptrs.data_ptr(), numel,
                                         C.byref(raw), C.byref(h), step, _stream()),
            "solo_multi_step_static")
+
+
+def solo_multi_step_host(params: list[torch.Tensor], grads_host: list[torch.Tensor],
+                         params_out_host, state: State, h: Hyper, step: int, chunk_elems: int = 0) -> None:
+    """The step with gradients in host memory (CPU bf16 tensors, pinned for overlap) and, when
+    `params_out_host` is a list of CPU tensors of the parameters' type, a host copy of the updated
+    parameters.  `params` are the resident CUDA tensors."""
+    T = len(params)
+    want = torch.bfloat16 if h.param_dtype == 1 else torch.float32
+    for i in range(T):
+        if not (params[i].is_cuda and params[i].is_contiguous() and params[i].dtype == want):
+            raise ValueError("params must be contiguous CUDA tensors of the type hyper.param_dtype names")
+        if grads_host[i].is_cuda or grads_host[i].dtype != torch.bfloat16 or not grads_host[i].is_contiguous() \
+                or grads_host[i].numel() != params[i].numel():
+            raise ValueError("grads_host must be contiguous CPU bf16 tensors of the parameters' sizes")
+        if params_out_host is not None:
+            o = params_out_host[i]
+            if o.is_cuda or o.dtype != want or not o.is_contiguous() or o.numel() != params[i].numel():
+                raise ValueError("params_out_host must be contiguous CPU tensors like the parameters")
+    vp = C.c_void_p * T
+    pd = vp(*[p.data_ptr() for p in params])
+    gh = vp(*[g.data_ptr() for g in grads_host])
+    po = vp(*[o.data_ptr() for o in params_out_host]) if params_out_host is not None else None
+    numel = (C.c_int64 * T)(*[int(p.numel()) for p in params])
+    lst = HostList(T, C.cast(pd, C.c_void_p), C.cast(gh, C.c_void_p),
+                   C.cast(po, C.c_void_p) if po is not None else None, C.cast(numel, C.c_void_p),
+                   int(chunk_elems), state.handle)
+    _check(lib().solo_multi_step_host(C.byref(lst), C.byref(h), step, _stream()), "solo_multi_step_host")
 
 
 def codebook_m(bits: int) -> torch.Tensor:

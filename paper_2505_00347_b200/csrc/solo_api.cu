@@ -33,6 +33,22 @@ struct solo_state {
     int v_codebook = SOLO_V_LOG;  // selector of the last step (what solo_dequant decodes with)
     int* status = nullptr;
     size_t bytes_codes_m = 0, bytes_codes_v = 0;
+    struct HostPipe* pipe = nullptr;   // staging of solo_multi_step_host, created at its first call
+};
+
+// Staging of the host-buffer entry point: three slots, each with its own stream, a device buffer
+// for one chunk of gradients and the device array of per-tensor gradient pointers of that chunk.
+struct HostPipe {
+    static constexpr int SLOTS = 3;
+    int64_t chunk_tiles = 0;
+    cudaStream_t stream[SLOTS] = {};
+    cudaEvent_t done[SLOTS] = {};          // end of the slot's last chunk
+    cudaEvent_t start = nullptr;           // the caller's stream at the call
+    unsigned char* d_grad[SLOTS] = {};     // chunk_tiles * (TILE * 2 + 16) bytes
+    void** d_grad_list[SLOTS] = {};        // [T] device
+    void** h_grad_list[SLOTS] = {};        // [T] pinned host
+    void** d_param_list = nullptr;         // [T] device
+    void** h_param_list = nullptr;         // [T] pinned host
 };
 
 namespace {
@@ -194,7 +210,8 @@ int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
     if (!k) return SOLO_EINVAL;
     int per_sm = solo::kernel_occupancy(k, dyn_smem);
     if (per_sm <= 0) return SOLO_ECUDA;
-    int64_t grid = std::min<int64_t>(s->tiles_total, (int64_t)sm_count(s->device) * per_sm);
+    int64_t grid = std::min<int64_t>(a.total_tiles - a.tile_first, (int64_t)sm_count(s->device) * per_sm);
+    if (grid < 1) return SOLO_EINVAL;
     void* params[] = {(void*)&a};
     cudaError_t e = cudaLaunchKernel((const void*)k, dim3((unsigned)grid), dim3(solo::CTA), params, dyn_smem, stream);
     if (e != cudaSuccess) {
@@ -369,6 +386,21 @@ int solo_state_create(int64_t numel, int bits_m, int bits_v, int block, solo_sta
 int solo_state_destroy(solo_state_t* s) {
     if (!s) return SOLO_OK;
     cudaDeviceSynchronize();
+    if (s->pipe) {
+        HostPipe* hp = s->pipe;
+        for (int i = 0; i < HostPipe::SLOTS; ++i) {
+            if (hp->stream[i]) cudaStreamDestroy(hp->stream[i]);
+            if (hp->done[i]) cudaEventDestroy(hp->done[i]);
+            if (hp->d_grad[i]) cudaFree(hp->d_grad[i]);
+            if (hp->d_grad_list[i]) cudaFree(hp->d_grad_list[i]);
+            if (hp->h_grad_list[i]) cudaFreeHost(hp->h_grad_list[i]);
+        }
+        if (hp->start) cudaEventDestroy(hp->start);
+        if (hp->d_param_list) cudaFree(hp->d_param_list);
+        if (hp->h_param_list) cudaFreeHost(hp->h_param_list);
+        delete hp;
+        s->pipe = nullptr;
+    }
     void* ptrs[] = {s->codes_m, s->codes_v, s->scale_m, s->scale_v, s->alpha,
                     s->geom, s->tables_m, s->tables_v, s->status};
     for (void* p : ptrs)
@@ -410,6 +442,137 @@ int solo_multi_step(const solo_tensor_list_t* list, const solo_hyper_t* hyper, i
     a.grad_list = list->grad;
     a.numel_check = list->numel;
     return launch_step(s, a, (cudaStream_t)stream);
+}
+
+namespace {
+
+// Creates (or, for another chunk size, re-creates) the staging of solo_multi_step_host.
+int host_pipe_prepare(solo_state* s, int64_t chunk_tiles) {
+    HostPipe* hp = s->pipe;
+    if (hp && hp->chunk_tiles == chunk_tiles) return SOLO_OK;
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return SOLO_ECUDA; }
+    if (!hp) {
+        hp = new (std::nothrow) HostPipe();
+        if (!hp) return SOLO_ENOMEM;
+        s->pipe = hp;
+        const size_t list_bytes = (size_t)s->num_tensors * sizeof(void*);
+        bool ok = cudaEventCreateWithFlags(&hp->start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaMalloc((void**)&hp->d_param_list, list_bytes) == cudaSuccess &&
+                  cudaMallocHost((void**)&hp->h_param_list, list_bytes) == cudaSuccess;
+        for (int i = 0; ok && i < HostPipe::SLOTS; ++i)
+            ok = cudaStreamCreateWithFlags(&hp->stream[i], cudaStreamNonBlocking) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&hp->done[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaMalloc((void**)&hp->d_grad_list[i], list_bytes) == cudaSuccess &&
+                 cudaMallocHost((void**)&hp->h_grad_list[i], list_bytes) == cudaSuccess;
+        if (!ok) { cudaGetLastError(); return SOLO_ENOMEM; }   // what exists is freed with the state
+    }
+    for (int i = 0; i < HostPipe::SLOTS; ++i) {
+        if (hp->d_grad[i]) cudaFree(hp->d_grad[i]);
+        hp->d_grad[i] = nullptr;
+    }
+    hp->chunk_tiles = 0;
+    const size_t slot_bytes = (size_t)chunk_tiles * (solo::TILE * 2 + 16);
+    for (int i = 0; i < HostPipe::SLOTS; ++i)
+        if (cudaMalloc((void**)&hp->d_grad[i], slot_bytes) != cudaSuccess) { cudaGetLastError(); return SOLO_ENOMEM; }
+    hp->chunk_tiles = chunk_tiles;
+    return SOLO_OK;
+}
+
+}  // namespace
+
+int solo_multi_step_host(const solo_host_list_t* list, const solo_hyper_t* hyper, int64_t step,
+                         void* stream_) {
+    if (!list || !list->state || !list->param_dev || !list->grad_host || !list->numel) return SOLO_EINVAL;
+    int rc = check_hyper(hyper, step);
+    if (rc) return rc;
+    solo_state* s = list->state;
+    const int T = s->num_tensors;
+    if (list->num_tensors != T || !on_state_device(s)) return SOLO_ESTATE;
+    if (list->chunk_elems < 0) return SOLO_EINVAL;
+    const int psz = hyper->param_dtype == 1 ? 2 : 4;
+    for (int t = 0; t < T; ++t) {
+        if (list->numel[t] != s->numel[t]) return SOLO_ESTATE;
+        if (!list->param_dev[t] || !list->grad_host[t] || (list->param_out_host && !list->param_out_host[t]))
+            return SOLO_EINVAL;
+        if (((uintptr_t)list->param_dev[t]) & 15u) return SOLO_EALIGN;
+    }
+    const int64_t chunk_elems = list->chunk_elems ? list->chunk_elems : (int64_t)16 << 20;
+    const int64_t chunk_tiles = std::max<int64_t>(1, chunk_elems / solo::TILE);
+    rc = host_pipe_prepare(s, chunk_tiles);
+    if (rc) return rc;
+    HostPipe* hp = s->pipe;
+    cudaStream_t user = (cudaStream_t)stream_;
+    bool ok = true;
+    auto chk = [&](cudaError_t e) { ok = ok && e == cudaSuccess; };
+
+    // the call before this one may still be using the pinned pointer arrays and the slots
+    for (int i = 0; i < HostPipe::SLOTS; ++i) chk(cudaEventSynchronize(hp->done[i]));
+    for (int t = 0; t < T; ++t) hp->h_param_list[t] = list->param_dev[t];
+    chk(cudaMemcpyAsync(hp->d_param_list, hp->h_param_list, (size_t)T * sizeof(void*), cudaMemcpyHostToDevice, user));
+    chk(cudaEventRecord(hp->start, user));
+    for (int i = 0; i < HostPipe::SLOTS; ++i) chk(cudaStreamWaitEvent(hp->stream[i], hp->start, 0));
+    if (!ok) { cudaGetLastError(); return SOLO_ECUDA; }
+
+    StepArgs base;
+    std::memset(&base, 0, sizeof(base));
+    fill_state_args(s, base);
+    reduce_hyper(hyper, step, s->block, base);
+    select_v_codebook(s, hyper, base);
+    base.param_list = hp->d_param_list;
+
+    int tensor = 0;
+    int64_t chunk = 0;
+    for (int64_t first = 0; first < s->tiles_total; first += chunk_tiles, ++chunk) {
+        const int64_t last = std::min<int64_t>(s->tiles_total, first + chunk_tiles);
+        const int slot = (int)(chunk % HostPipe::SLOTS);
+        cudaStream_t st = hp->stream[slot];
+        if (chunk >= HostPipe::SLOTS) chk(cudaEventSynchronize(hp->done[slot]));   // its pinned list is free again
+        while (s->tile_start[tensor + 1] <= first) ++tensor;
+        const int tensor_first = tensor;
+        // upload: one piece per tensor that the chunk touches, each from a 16-byte boundary of the slot
+        size_t off = 0;
+        int t = tensor;
+        for (; t < T && s->tile_start[t] < last; ++t) {
+            const int64_t e_lo = (std::max<int64_t>(s->tile_start[t], first) - s->tile_start[t]) * solo::TILE;
+            const int64_t e_hi = std::min<int64_t>(s->numel[t],
+                                                   (std::min<int64_t>(s->tile_start[t + 1], last) - s->tile_start[t]) * solo::TILE);
+            const size_t bytes = (size_t)(e_hi - e_lo) * 2;
+            chk(cudaMemcpyAsync(hp->d_grad[slot] + off, (const char*)list->grad_host[t] + e_lo * 2, bytes,
+                                cudaMemcpyHostToDevice, st));
+            // the kernel indexes gradients by the element's position in its tensor
+            hp->h_grad_list[slot][t] = (void*)((uintptr_t)hp->d_grad[slot] + off - (uintptr_t)(e_lo * 2));
+            off += (bytes + 15) / 16 * 16;
+        }
+        const int t_end = t;
+        chk(cudaMemcpyAsync(hp->d_grad_list[slot] + tensor_first, hp->h_grad_list[slot] + tensor_first,
+                            (size_t)(t_end - tensor_first) * sizeof(void*), cudaMemcpyHostToDevice, st));
+        if (!ok) break;
+        StepArgs a = base;
+        a.grad_list = (const void* const*)hp->d_grad_list[slot];
+        a.tile_first = first;
+        a.total_tiles = last;
+        a.tensor_first = tensor_first;
+        rc = launch_step(s, a, st);
+        if (rc) break;
+        if (list->param_out_host) {
+            for (t = tensor_first; t < t_end; ++t) {
+                const int64_t e_lo = (std::max<int64_t>(s->tile_start[t], first) - s->tile_start[t]) * solo::TILE;
+                const int64_t e_hi = std::min<int64_t>(s->numel[t],
+                                                       (std::min<int64_t>(s->tile_start[t + 1], last) - s->tile_start[t]) * solo::TILE);
+                chk(cudaMemcpyAsync((char*)list->param_out_host[t] + e_lo * psz, (const char*)list->param_dev[t] + e_lo * psz,
+                                    (size_t)(e_hi - e_lo) * psz, cudaMemcpyDeviceToHost, st));
+            }
+        }
+        chk(cudaEventRecord(hp->done[slot], st));
+    }
+    // the caller's stream continues after every slot's last chunk, also when something failed
+    for (int i = 0; i < HostPipe::SLOTS; ++i) {
+        cudaEventRecord(hp->done[i], hp->stream[i]);
+        cudaStreamWaitEvent(user, hp->done[i], 0);
+    }
+    if (rc) return rc;
+    if (!ok) { cudaGetLastError(); return SOLO_ECUDA; }
+    return SOLO_OK;
 }
 
 int solo_multi_step_static(int32_t num_tensors, void* const* param_dev, const void* const* grad_dev,

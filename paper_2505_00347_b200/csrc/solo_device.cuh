@@ -38,7 +38,9 @@ struct StepArgs {
     const int64_t* block_start;        // [T+1]
     const int64_t* tile_start;         // [T+1]
     int32_t num_tensors;
-    int64_t total_tiles;
+    int64_t total_tiles;               // the launch covers tiles [tile_first, total_tiles)
+    int64_t tile_first;
+    int32_t tensor_first;              // tensor that holds tile_first
     // state
     uint8_t* codes_m;
     uint8_t* codes_v;
@@ -304,7 +306,7 @@ __global__ void __launch_bounds__(CTA) solo_step_kernel(const StepArgs a) {
     const int gl = tid & (G - 1);                              // thread within its block
     const bool bf16p = a.param_bf16 != 0;
 
-    for (int64_t tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x) {
+    for (int64_t tile = a.tile_first + blockIdx.x; tile < a.total_tiles; tile += gridDim.x) {
         const int tensor = a.num_tensors > 1 ? find_tensor(a.tile_start, a.num_tensors, tile) : 0;
         const int64_t n = __ldg(a.numel + tensor);
         if (a.numel_check != nullptr && __ldg(a.numel_check + tensor) != n) {

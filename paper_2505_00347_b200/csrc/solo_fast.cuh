@@ -832,7 +832,7 @@ __global__ void __launch_bounds__(CTA, 4) solo_step_fast_kernel(const StepArgs a
     // Tile indices fit 32 bits (the host selects this kernel only below 2^31 tiles).  Tiles are
     // visited in increasing order, so the tensor of a tile is found by walking forward.
     const int total_tiles = (int)a.total_tiles, stride = (int)gridDim.x;
-    int tensor = -1;
+    int tensor = a.tensor_first - 1;
     int t_lo = 0, t_hi = 0, full_tiles = 0;      // the tensor's tiles [t_lo, t_hi); its first full_tiles are full
     int64_t n = 0, jb0 = 0;
     char* pbase = nullptr;
@@ -840,7 +840,7 @@ __global__ void __launch_bounds__(CTA, 4) solo_step_fast_kernel(const StepArgs a
     bool skip = false;
     Ahead ah;
     int par = 0;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += stride) {
+    for (int tile = (int)a.tile_first + blockIdx.x; tile < total_tiles; tile += stride) {
         if (tile >= t_hi) {
             do {
                 ++tensor;
@@ -861,7 +861,7 @@ __global__ void __launch_bounds__(CTA, 4) solo_step_fast_kernel(const StepArgs a
         const int64_t jb_tile = jb0 + (int64_t)tin * (CTA / G);
         if (tin < full_tiles)
             fast_tile<BM, BV, G, true, PBF>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, ah,
-                                       tin + stride < full_tiles, stride);
+                                       tin + stride < full_tiles && tile + stride < total_tiles, stride);
         else
             fast_tile<BM, BV, G, false, PBF>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, ah, false, 0);
         par ^= 1;

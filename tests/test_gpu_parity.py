@@ -198,6 +198,46 @@ def test_nan_and_inf_gradients_do_not_hang():
     st.destroy()
 
 
+@pytest.mark.parametrize("bits_m,bits_v,block,extra,chunk", [
+    (2, 3, 128, dict(), 2048 * 3),
+    (4, 4, 64, dict(param_dtype=1, param_round=1), 2048),
+    (8, 3, 2048, dict(round_m=1), 2048 * 2),
+    (3, 3, 256, dict(v_codebook=2), 2048 * 5),
+    (2, 3, 128, dict(), 0),
+])
+def test_host_buffer_entry_point(bits_m, bits_v, block, extra, chunk):
+    """solo_multi_step_host (gradients from host memory, parameters copied back, chunked over three
+    streams) against solo_multi_step on the same inputs: identical state and parameters, chunk
+    boundaries inside tensors, more chunks than staging slots, tiny tensors, two steps."""
+    from paper_2505_00347_b200 import binding as B
+    sizes = (2048 * 7 + 300, 5, 2048 * 2, 129, 2048 * 4 + 1, 2047)
+    w = synth.workload(2, sizes=sizes)
+    dtype = torch.bfloat16 if extra.get("param_dtype") == 1 else torch.float32
+    params = [synth.make_param(w, i, dtype=dtype) for i in range(len(sizes))]
+    p_dev = [p.clone().cuda() for p in params]
+    p_hst = [p.clone().cuda() for p in params]
+    out = [torch.zeros_like(p).pin_memory() for p in params]
+    h = B.hyper(lr=1e-3, beta1=0.6, beta2=0.999, weight_decay=0.01, seed=77, **extra)
+    st_dev = B.State(list(sizes), bits_m, bits_v, block)
+    st_hst = B.State(list(sizes), bits_m, bits_v, block)
+    for t in (1, 2):
+        grads = [synth.make_grad(w, i, t) for i in range(len(sizes))]
+        B.solo_multi_step(B.TensorSet(p_dev, [g.cuda() for g in grads], st_dev), h, t)
+        pinned = [g.pin_memory() for g in grads]
+        B.solo_multi_step_host(p_hst, pinned, out if t == 2 else None, st_hst, h, t, chunk_elems=chunk)
+        torch.cuda.synchronize()
+        assert st_hst.status() == 0
+        assert torch.equal(st_dev.export(), st_hst.export()), t
+        for a, b in zip(p_dev, p_hst):
+            assert torch.equal(a, b), t
+    for a, o in zip(p_dev, out):
+        assert torch.equal(a.cpu(), o)
+    with pytest.raises(B.SoloError):
+        B.solo_multi_step_host(p_hst[:2], pinned[:2], None, st_hst, h, 3)       # other list than the state's
+    st_dev.destroy()
+    st_hst.destroy()
+
+
 @pytest.mark.parametrize("v_codebook", [0, 3])
 def test_checkpoint_export_import(v_codebook):
     """solo_state_export / solo_state_import: the byte string holds the header and the five
