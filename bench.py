@@ -183,12 +183,18 @@ def run_ours(args, rank, world):
     pbytes = 2 if args.param_bf16 else 4
     e2e_ms, h2d, d2h, e2e_buffers = None, 2 * n, pbytes * n, None
     if not args.no_e2e:
-        try:                                     # one pinned buffer per tensor
-            hgs = [torch.empty(g.numel(), dtype=torch.bfloat16, pin_memory=True) for g in grads]
-            hps = [torch.empty(p.numel(), dtype=p.dtype, pin_memory=True) for p in params]
-            e2e_buffers = "one pinned host buffer per tensor"
-        except RuntimeError:                     # not enough page-locked memory: all tensors share one
-            hgs = hps = None
+        # one pinned buffer per tensor when this rank has the host to itself; with several ranks on the
+        # host, or when that much page-locked memory is refused, all tensors share one buffer
+        distinct = world == 1
+        if distinct:
+            try:
+                hgs = [torch.empty(g.numel(), dtype=torch.bfloat16, pin_memory=True) for g in grads]
+                hps = [torch.empty(p.numel(), dtype=p.dtype, pin_memory=True) for p in params]
+                e2e_buffers = "one pinned host buffer per tensor"
+            except RuntimeError:
+                hgs = hps = None
+                distinct = False
+        if not distinct:
             big = max(w.sizes)
             hg = torch.empty(big, dtype=torch.bfloat16, pin_memory=True)
             hp = torch.empty(big, dtype=params[0].dtype, pin_memory=True)
