@@ -405,12 +405,13 @@ __device__ __forceinline__ void bar_sync(int id) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(CTA) : "memory");
 }
 
-// One tile.  FULL: all 2048 elements exist and both tensor pointers are 16-byte aligned.
-// Inputs are loaded straight from global memory (128-bit streaming loads); staging the next
-// tile through shared memory with cp.async, or requesting its lines into L2 ahead of time,
-// was measured slower: the extra instructions cost more than the hidden latency gains, the
-// four resident CTAs per SM cover each other's load phases.
-
+// One tile.  FULL: all 2048 elements exist and both tensor pointers are 16-byte aligned; its
+// inputs come from a shared-memory stage that bulk asynchronous copies filled while the tile
+// before it was worked on (per-thread cp.async staging, L2 prefetch and register prefetch of the
+// next tile were all measured slower than plain 128-bit loads; the bulk copies, issued by one
+// thread, are faster).  Other tiles (tails, unaligned tensors) use masked plain loads.
+// `par` alternates between tiles (double buffering of the per-block exchange arrays); `ah`
+// carries the copy-ahead state; next_full / next_dtin describe the CTA's next tile.
 template <int BM, int BV, int G, bool FULL, bool PBF>
 __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, const float* s_y,
                                           const float* s_mid, char* pbase, const char* gbase,
