@@ -248,6 +248,13 @@ int solo_state_status(solo_state_t* state, int* status_out);
 int solo_codebook_m(int bits, float* levels_host);
 
 /*
+ * The same for a baseline codebook of the unsigned state (Appendix A): v_codebook is SOLO_V_DE,
+ * SOLO_V_LINEAR or SOLO_V_LINEAR_NOZERO (the logarithmic levels alpha^k depend on the block and
+ * have no fixed table).
+ */
+int solo_codebook_v(int v_codebook, int bits, float* levels_host);
+
+/*
  * Eq. 7 with the defaults of Sec. 3.4: the recommended beta1 for `bits_m`-bit first
  * moments, from_scratch = 0 (fine-tuning, b = 5 column of Fig. 4) or 1 (b = 8 column),
  * floored to one decimal like the paper's own defaults (4 bit: 0.8 / 0.3; 2 bit: 0.5 / 0.1).

@@ -101,6 +101,8 @@ def lib() -> C.CDLL:
                                   C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     L.solo_state_status.argtypes = [vp, C.POINTER(C.c_int)]
     L.solo_codebook_m.argtypes = [i32, C.POINTER(C.c_float)]
+    L.solo_codebook_v.argtypes = [i32, i32, C.POINTER(C.c_float)]
+    L.solo_codebook_v.restype = C.c_int
     L.solo_default_beta1.argtypes = [i32, i32]
     L.solo_default_beta1.restype = C.c_float
     L.solo_set_kernel_policy.argtypes = [i32]
@@ -361,6 +363,12 @@ def solo_multi_step_host(params: list[torch.Tensor], grads_host: list[torch.Tens
 def codebook_m(bits: int) -> torch.Tensor:
     buf = (C.c_float * (1 << bits))()
     _check(lib().solo_codebook_m(bits, buf), "solo_codebook_m")
+    return torch.tensor(list(buf), dtype=torch.float32)
+
+
+def codebook_v(v_codebook: int, bits: int) -> torch.Tensor:
+    buf = (C.c_float * (1 << bits))()
+    _check(lib().solo_codebook_v(v_codebook, bits, buf), "solo_codebook_v")
     return torch.tensor(list(buf), dtype=torch.float32)
 
 

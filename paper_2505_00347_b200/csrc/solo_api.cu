@@ -829,6 +829,15 @@ int solo_codebook_m(int bits, float* levels_host) {
     return SOLO_OK;
 }
 
+int solo_codebook_v(int v_codebook, int bits, float* levels_host) {
+    if (!valid_bits(bits) || !levels_host) return SOLO_EINVAL;
+    if (v_codebook < SOLO_V_DE || v_codebook > SOLO_V_LINEAR_NOZERO) return SOLO_EINVAL;
+    std::vector<float> y;
+    unsigned_levels(v_codebook, bits, y);
+    std::memcpy(levels_host, y.data(), y.size() * 4);
+    return SOLO_OK;
+}
+
 float solo_default_beta1(int bits_m, int from_scratch) {
     if (bits_m < 2 || bits_m > 8) return 0.0f;
     auto r_median = [](int bits) {

@@ -54,6 +54,10 @@ def test_library_codebook_equals_oracle_codebook(B):
     """Two independent constructions of the signed DE levels give the same binary32 values."""
     for b in (2, 3, 4, 8):
         assert np.array_equal(B.codebook_m(b).numpy(), oracle.codebook(oracle.DE_SIGNED, b))
+        for sel, kind in ((1, oracle.DE_UNSIGNED), (2, oracle.LINEAR_UNSIGNED), (3, oracle.LINEAR_NOZERO)):
+            assert np.array_equal(B.codebook_v(sel, b).numpy(), oracle.codebook(kind, b)), (sel, b)
+    with pytest.raises(B.SoloError):
+        B.codebook_v(0, 4)
 
 
 def test_hyper_records_agree(B):
