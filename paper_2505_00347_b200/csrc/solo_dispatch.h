@@ -31,10 +31,12 @@ StepKernel step_kernel(int bits_m, int bits_v, bool cta_group);
 // Streamlined kernel (2/3/4-bit states, block 64, 128, 256 or 2048, fp32 or bf16 parameters); null
 // outside that domain.  The caller additionally requires the logarithmic second-moment
 // quantizer, nearest rounding of the first moment and eps >= 1e-12.
-StepKernel fast_kernel_bm2(int bv_index, int block, bool param_bf16);
-StepKernel fast_kernel_bm3(int bv_index, int block, bool param_bf16);
-StepKernel fast_kernel_bm4(int bv_index, int block, bool param_bf16);
-StepKernel fast_kernel(int bits_m, int bits_v, int block, bool param_bf16);
+// `plain`: no L2 term in the gradient, no AdaBelief, base from the quantile, xi drawn (the
+// paper's step as it stands); that instantiation carries no code for the other modes.
+StepKernel fast_kernel_bm2(int bv_index, int block, bool param_bf16, bool plain);
+StepKernel fast_kernel_bm3(int bv_index, int block, bool param_bf16, bool plain);
+StepKernel fast_kernel_bm4(int bv_index, int block, bool param_bf16, bool plain);
+StepKernel fast_kernel(int bits_m, int bits_v, int block, bool param_bf16, bool plain);
 // Dynamic shared memory the streamlined kernels are launched with.
 size_t fast_kernel_smem();
 // Resident CTAs per SM of a step kernel launched with `dyn_smem` bytes of dynamic shared memory

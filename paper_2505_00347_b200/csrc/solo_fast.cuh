@@ -412,7 +412,7 @@ __device__ __forceinline__ void bar_sync(int id) {
 // thread, are faster).  Other tiles (tails, unaligned tensors) use masked plain loads.
 // `par` alternates between tiles (double buffering of the per-block exchange arrays); `ah`
 // carries the copy-ahead state; next_full / next_dtin describe the CTA's next tile.
-template <int BM, int BV, int G, bool FULL, bool PBF>
+template <int BM, int BV, int G, bool FULL, bool PBF, bool PLAIN>
 __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, const float* s_y,
                                           const float* s_mid, char* pbase, const char* gbase,
                                           const int64_t n, const int tin, const int64_t jb_tile,
@@ -421,6 +421,11 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     constexpr int KM = 1 << BM, KV = 1 << BV;
     constexpr int NG = CTA / G, B = G * EPT;
     constexpr int PSZ = PBF ? 2 : 4;                            // bytes per parameter
+    // PLAIN: the step of the paper as it stands (Adam(W) without an L2 term in the gradient, base
+    // from the p-quantile, xi drawn); the other modes cost branches and argument loads per tile
+    const bool l2 = !PLAIN && a.l2, belief = !PLAIN && a.belief;
+    const bool fixed_base = !PLAIN && a.fixed_alpha > 0.0f;
+    const bool round_v = PLAIN || a.round_v;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gl = tid & (G - 1), grp = tid / G;
     const bool hi = G < 32 && (lane & G) != 0;                  // odd group of its pair
@@ -534,7 +539,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     }
     if constexpr (G == CTA) __syncthreads(); else __syncwarp();
 
-    if (a.l2) {
+    if (l2) {
 #pragma unroll
         for (int i = 0; i < EPT; ++i) g[i] = __fmaf_rn(a.weight_decay, p[i], g[i]);
     }
@@ -567,7 +572,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
         mx_v = max(mx_v, valid ? __float_as_uint(vh[i]) : 0u);
     }
     };
-    if (a.belief) ema(std::true_type{}); else ema(std::false_type{});
+    if (belief) ema(std::true_type{}); else ema(std::false_type{});
     uint32_t mx_m = __float_as_uint(mx_m_f);
 
     // Adam(W) update of element i and, after every fourth, the store; issued between the
@@ -634,7 +639,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
         const uint32_t t = s.red[par][lane & 15];
         mx_m = __reduce_max_sync(0xffffffffu, (lane & 8) ? 0u : t);
         mx_v = __reduce_max_sync(0xffffffffu, (lane & 8) ? t : 0u);
-        if (!(a.fixed_alpha > 0.0f)) {
+        if (!fixed_base) {
             uint32_t key[EPT];
 #pragma unroll
             for (int i = 0; i < EPT; ++i) key[i] = (FULL || i < nv) ? __float_as_uint(vh[i]) : 0xFFFFFFFFu;
@@ -648,7 +653,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     } else {
         mx_m = seg_max31<G>(mx_m, hi);
         mx_v = seg_max31<G>(mx_v, hi);
-        if (a.fixed_alpha > 0.0f) {                                  // fixed base: no quantile to find
+        if (fixed_base) {                                            // no quantile to find
 #pragma unroll
             for (int i = 0; i < EPT; ++i) update(i);
         } else {
@@ -677,7 +682,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     bar_sync(1);
     uint32_t w[4] = {0u, 0u, 0u, 0u};
     if (warp != 0) {
-        if (a.round_v) philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, (uint32_t)tensor * 4u, a.rk, w);
+        if (round_v) philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, (uint32_t)tensor * 4u, a.rk, w);
     } else if (tid < NG) {
         const uint4 in = s.xin[par][tid];
         const float dm_new = __uint_as_float(in.x), dv_new = __uint_as_float(in.y);
@@ -686,7 +691,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
         const float inv_dv = 1.0f / dv_new;
         const float rho = fminf(fmaxf(__uint_as_float(in.z) * inv_dv, RHO_MIN), RHO_MAX);
         const float lam = log2_sp(rho) * (1.0f / (float)(KV - 1));
-        const float al_new = a.fixed_alpha > 0.0f ? a.fixed_alpha : exp2_sp(lam);
+        const float al_new = fixed_base ? a.fixed_alpha : exp2_sp(lam);
         const float inv_lambda = 1.0f / log2_sp(al_new);
         const float guard = __fmaf_rn(fabsf(inv_lambda), LG2_ABS, LG2_REL * (float)(KV + 1));
         s.xout[par][tid] = make_float4(inv_dm, inv_dv, inv_lambda, 0.5f - guard);
@@ -700,7 +705,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
         }
     }
     bar_sync(2);
-    if (warp == 0 && a.round_v)
+    if (warp == 0 && round_v)
         philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, (uint32_t)tensor * 4u, a.rk, w);
     float dr[EPT];                                               // the 16-bit draws d as binary32
 #pragma unroll
@@ -763,8 +768,8 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
         constexpr uint32_t MAGIC_BITS = 0x4B400000u;
         const float ils = il * (1.0f / KM1);
         // xi = (d + 1/2) / 2^16 - 1/2 (exact); scaled copy for the approximate path
-        const float xs1 = a.round_v ? (float)(0x1p-16 / (KV - 1)) : 0.0f;
-        const float xs0 = a.round_v ? (float)((-0.5 + 0x1p-17) / (KV - 1)) : 0.0f;
+        const float xs1 = round_v ? (float)(0x1p-16 / (KV - 1)) : 0.0f;
+        const float xs0 = round_v ? (float)((-0.5 + 0x1p-17) / (KV - 1)) : 0.0f;
         float worst = 0.0f;
         uint32_t acc = 0;
 #pragma unroll
@@ -782,7 +787,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
         if (__any_sync(0xffffffffu, worst > lim)) {
             // some element of the warp is too close to a rounding boundary for the
             // approximate logarithm: evaluate the exact sequence for all eight
-            const float x1 = a.round_v ? 0x1p-16f : 0.0f, x0 = a.round_v ? -0.5f + 0x1p-17f : 0.0f;
+            const float x1 = round_v ? 0x1p-16f : 0.0f, x0 = round_v ? -0.5f + 0x1p-17f : 0.0f;
             ov = 0;
 #pragma unroll
             for (int i = EPT - 1; i >= 0; --i) {
@@ -810,7 +815,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     }
 }
 
-template <int BM, int BV, int G, bool PBF>
+template <int BM, int BV, int G, bool PBF, bool PLAIN>
 __global__ void __launch_bounds__(CTA, 4) solo_step_fast_kernel(const StepArgs a) {
     constexpr int KM = 1 << BM;
     extern __shared__ __align__(16) unsigned char fast_smem[];   // sizeof(FastShared), above the static 48 KB limit
@@ -861,10 +866,10 @@ __global__ void __launch_bounds__(CTA, 4) solo_step_fast_kernel(const StepArgs a
         const int tin = tile - t_lo;
         const int64_t jb_tile = jb0 + (int64_t)tin * (CTA / G);
         if (tin < full_tiles)
-            fast_tile<BM, BV, G, true, PBF>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, ah,
+            fast_tile<BM, BV, G, true, PBF, PLAIN>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, ah,
                                        tin + stride < full_tiles && tile + stride < total_tiles, stride);
         else
-            fast_tile<BM, BV, G, false, PBF>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, ah, false, 0);
+            fast_tile<BM, BV, G, false, PBF, PLAIN>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, ah, false, 0);
         par ^= 1;
     }
     // every copy that was issued has been waited for by the thread that issued it, unless that

@@ -11,18 +11,19 @@
 
 namespace solo {
 
-#define SOLO_ROW(BV, PBF)                                                                  \
-    {solo_step_fast_kernel<SOLO_BM, BV, 8, PBF>, solo_step_fast_kernel<SOLO_BM, BV, 16, PBF>, \
-     solo_step_fast_kernel<SOLO_BM, BV, 32, PBF>, solo_step_fast_kernel<SOLO_BM, BV, 256, PBF>}
+#define SOLO_ROW(BV, PBF, PLAIN)                                                                            \
+    {solo_step_fast_kernel<SOLO_BM, BV, 8, PBF, PLAIN>, solo_step_fast_kernel<SOLO_BM, BV, 16, PBF, PLAIN>, \
+     solo_step_fast_kernel<SOLO_BM, BV, 32, PBF, PLAIN>, solo_step_fast_kernel<SOLO_BM, BV, 256, PBF, PLAIN>}
+#define SOLO_PLANE(PBF, PLAIN) {SOLO_ROW(2, PBF, PLAIN), SOLO_ROW(3, PBF, PLAIN), SOLO_ROW(4, PBF, PLAIN)}
 
-StepKernel SOLO_CAT(fast_kernel_bm, SOLO_BM)(int bv_index, int block, bool param_bf16) {
-    static const StepKernel table[2][3][4] = {
-        {SOLO_ROW(2, false), SOLO_ROW(3, false), SOLO_ROW(4, false)},
-        {SOLO_ROW(2, true), SOLO_ROW(3, true), SOLO_ROW(4, true)},
+StepKernel SOLO_CAT(fast_kernel_bm, SOLO_BM)(int bv_index, int block, bool param_bf16, bool plain) {
+    static const StepKernel table[2][2][3][4] = {
+        {SOLO_PLANE(false, false), SOLO_PLANE(true, false)},
+        {SOLO_PLANE(false, true), SOLO_PLANE(true, true)},
     };
     const int g = block == 64 ? 0 : block == 128 ? 1 : block == 256 ? 2 : block == 2048 ? 3 : -1;
     if (bv_index < 0 || bv_index > 2 || g < 0) return nullptr;
-    return table[param_bf16 ? 1 : 0][bv_index][g];
+    return table[plain ? 1 : 0][param_bf16 ? 1 : 0][bv_index][g];
 }
 
 #if SOLO_BM == 2

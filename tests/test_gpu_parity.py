@@ -43,6 +43,23 @@ def test_bits_and_blocks_random_state(bits_m, bits_v, block):
     assert rep.exempt_m + rep.exempt_v <= 3
 
 
+@pytest.mark.parametrize("bits_m,bits_v,block", [(2, 3, 128), (3, 2, 64), (4, 4, 256), (2, 2, 2048)])
+@pytest.mark.parametrize("hk", [dict(adamw=0, weight_decay=0.1), dict(round_v=0, belief=1),
+                                dict(fixed_alpha=0.5, param_dtype=1)])
+def test_mode_flags_at_other_widths(bits_m, bits_v, block, hk):
+    """The streamlined kernel has one instantiation for the paper's plain step and one that reads
+    the mode flags at run time; the latter at other widths and block sizes than the mode test."""
+    sizes = (2048 * 3 + block + 7, 500)
+    w = synth.workload(1, sizes=sizes)
+    dtype = torch.bfloat16 if hk.get("param_dtype") == 1 else torch.float32
+    params = [synth.make_param(w, i, dtype=dtype) for i in range(2)]
+    gf = lambda t: [synth.make_grad(w, i, t) for i in range(2)]
+    base = dict(lr=1e-3, beta1=0.6, beta2=0.999, weight_decay=0.01, seed=13)
+    base.update(hk)
+    st0 = synth.make_state(sizes, bits_m, bits_v, block, seed=19)
+    run_lockstep(sizes, bits_m, bits_v, block, base, 2, gf, params, state0=st0)
+
+
 @pytest.mark.parametrize("hk", [
     dict(adamw=0, weight_decay=0.1),
     dict(bias_correction=0),
