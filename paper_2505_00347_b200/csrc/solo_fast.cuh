@@ -328,6 +328,13 @@ __device__ __forceinline__ uint32_t select_kth(uint32_t head, const uint32_t* co
             if (r < EPT) side(r);
         }
         ans = pop_round<G, false, true>(head, off, col, le, self, hi);
+    } else if (UNIFORM_K && G == 32 && k == 26) {               // p = 0.1, block 256
+#pragma unroll
+        for (int r = 0; r < 25; ++r) {
+            pop_round<G, true>(head, off, col, le, self, hi);
+            if (r < EPT) side(r);
+        }
+        ans = pop_round<G, true, true>(head, off, col, le, self, hi);
     } else if (UNIFORM_K && k == 7) {                            // p = 0.1, block 64
 #pragma unroll
         for (int r = 0; r < 6; ++r) {
