@@ -29,6 +29,47 @@ def test_config1_lockstep_and_free_run():
     print("free run", rep)
 
 
+def test_gpt125m_set_free_run_100_steps():
+    """GPT-style 125M set (148 tensors, 124,439,808 parameters, 3-bit / 3-bit, block 128): the
+    library runs 100 steps on its own state, the oracle likewise; the packed state is compared bit
+    for bit at steps 10, 50 and 100 (any difference would compound, so equality at 100 covers every
+    step), the parameters within the per-step tolerance accumulated over the steps."""
+    from paper_2505_00347_b200 import binding as B
+    w = synth.workload(2)
+    T = len(w.sizes)
+    dev = torch.device("cuda")
+    gparams = [synth.make_param(w, i, device=dev) for i in range(T)]
+    oparams = [p.cpu().numpy().copy() for p in gparams]
+    prev = [p.clone() for p in gparams]
+    path = [torch.zeros_like(p) for p in gparams]                # sum over the steps of |update|
+    gstate = B.State(list(w.sizes), 3, 3, 128)
+    ostates = [oracle.State(n, 3, 3, 128) for n in w.sizes]
+    kw = dict(lr=w.lr, beta1=w.beta1, beta2=w.beta2, weight_decay=w.weight_decay, seed=2024)
+    ho, hg = parity.hyper_pair(**kw)
+    threads = oracle.hardware_threads()
+    for t in range(1, 101):
+        grads = [synth.make_grad(w, i, t, device=dev) for i in range(T)]
+        B.solo_multi_step(B.TensorSet(gparams, grads, gstate), hg, t)
+        for i in range(T):
+            path[i] += (gparams[i] - prev[i]).abs()
+            prev[i].copy_(gparams[i])
+            oracle.step(oparams[i], synth.bf16_bits(grads[i]), ostates[i], ho, t, tensor=i, nthreads=threads)
+        if t in (10, 50, 100):
+            torch.cuda.synchronize()
+            assert gstate.status() == 0
+            got = parity.download_state(gstate)
+            want = parity.join_state(ostates)
+            for k in parity.KEYS:
+                assert np.array_equal(got[k].view(np.uint8), want[k].view(np.uint8)), (t, k)
+            for i in range(T):
+                gp = gparams[i].cpu().numpy().astype(np.float64)
+                wp = oparams[i].astype(np.float64)
+                # per step: 1e-6 relative / 1e-9 absolute plus 3e-7 of the update term
+                tol = parity.RTOL * np.abs(wp) + parity.ATOL * t + 3e-7 * path[i].cpu().numpy().astype(np.float64)
+                assert np.all(np.abs(gp - wp) <= tol), (t, i, float(np.max(np.abs(gp - wp) - tol)))
+    gstate.destroy()
+
+
 @pytest.mark.parametrize("block", [64, 128, 256, 2048])
 @pytest.mark.parametrize("bits_m,bits_v", [(2, 2), (2, 3), (3, 3), (4, 2), (4, 4), (8, 8), (3, 8), (8, 2)])
 def test_bits_and_blocks_random_state(bits_m, bits_v, block):
