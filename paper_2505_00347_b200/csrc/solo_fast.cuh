@@ -365,27 +365,39 @@ __device__ __forceinline__ uint32_t select_kth(uint32_t head, const uint32_t* co
     return ans;
 }
 
-// k-th smallest (1-based, duplicates counted) of the CTA's 2048 keys, eight per thread: radix
-// select from the top, 8 bits per pass, one histogram bin per thread.  Keys are below 2^31 or
-// the all-ones filler of elements that do not exist (k never reaches those).  `hist` is 272
+// k-th smallest (1-based, duplicates counted) of the CTA's 2048 keys, eight per thread.  Keys are
+// below 2^31, or the all-ones filler of elements that do not exist (k never reaches those).
+// Radix select from the top in levels of 11, 11 and 9 bits with 2048 histogram bins (eight per
+// thread); as soon as the bin that holds the rank has at most 32 keys, those are collected and
+// ranked directly by the first warp, which is the usual case after the first level.  Exact for any
+// input: with many equal keys the levels run on until all 31 bits are fixed.  `hist` is 2096
 // words of shared memory.  Every thread of the CTA calls it; all return the same key.
 __device__ __forceinline__ uint32_t cta_select(const uint32_t (&key)[EPT], int k, uint32_t* hist) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    uint32_t* const scan = hist + 256;           // [0..7] warp totals, [8] chosen bin, [9] rank within it
-    uint32_t prefix = 0;
-    uint32_t kk = (uint32_t)k;
+    uint32_t* const scan = hist + 2048;      // [0..7] warp totals, [8] bin, [9] rank in it, [10] its count,
+                                             // [11] fill of `list`, [12] the answer
+    uint32_t* const list = hist + 2048 + 16; // the keys of a bin with at most 32 of them
+    uint32_t prefix = 0, kk = (uint32_t)k;
 #pragma unroll 1
-    for (int pass = 0; pass < 4; ++pass) {
-        const int shift = 24 - 8 * pass;
-        __syncthreads();                           // the bins and scan[] of the pass before are read
-        hist[tid] = 0;
+    for (int level = 0; level < 3; ++level) {
+        const int shift = level == 0 ? 20 : level == 1 ? 9 : 0;
+        const int width = level == 2 ? 9 : 11;
+        __syncthreads();                       // the bins, scan[] and list[] of earlier use are read
+        reinterpret_cast<uint4*>(hist)[2 * tid] = make_uint4(0u, 0u, 0u, 0u);
+        reinterpret_cast<uint4*>(hist)[2 * tid + 1] = make_uint4(0u, 0u, 0u, 0u);
+        if (tid == 0) scan[11] = 0;
         __syncthreads();
 #pragma unroll
-        for (int i = 0; i < EPT; ++i)
-            if (pass == 0 || (key[i] >> (shift + 8)) == prefix) atomicAdd(&hist[(key[i] >> shift) & 255u], 1u);
+        for (int i = 0; i < EPT; ++i)         // level 0: key >> 31 == 0 leaves the filler out
+            if ((key[i] >> (shift + width)) == prefix) atomicAdd(&hist[(key[i] >> shift) & ((1u << width) - 1u)], 1u);
         __syncthreads();
-        const uint32_t c = hist[tid];
-        uint32_t incl = c;
+        const uint4 c0 = reinterpret_cast<const uint4*>(hist)[2 * tid];
+        const uint4 c1 = reinterpret_cast<const uint4*>(hist)[2 * tid + 1];
+        const uint32_t c[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+        uint32_t mine = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) mine += c[j];
+        uint32_t incl = mine;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
             const uint32_t t = __shfl_up_sync(0xffffffffu, incl, d);
@@ -396,14 +408,43 @@ __device__ __forceinline__ uint32_t cta_select(const uint32_t (&key)[EPT], int k
 #pragma unroll
         for (int w = 0; w < 7; ++w)
             if (w < warp) incl += scan[w];
-        const uint32_t excl = incl - c;
-        if (kk > excl && kk <= incl) {             // exactly one bin holds the rank
-            scan[8] = (uint32_t)tid;
-            scan[9] = kk - excl;
+        uint32_t run = incl - mine;            // keys in the bins before this thread's
+        if (kk > run && kk <= incl) {          // exactly one thread holds the rank
+            int sel = 0;
+            uint32_t cnt = c[0];
+#pragma unroll
+            for (int j = 0; j < 7; ++j)
+                if (kk > run + c[j] && sel == j) {
+                    run += c[j];
+                    sel = j + 1;
+                    cnt = c[j + 1];
+                }
+            scan[8] = 8u * (uint32_t)tid + (uint32_t)sel;
+            scan[9] = kk - run;
+            scan[10] = cnt;
         }
         __syncthreads();
-        prefix = (prefix << 8) | scan[8];
+        prefix = (prefix << width) | scan[8];
         kk = scan[9];
+        const uint32_t cnt = scan[10];
+        if (level == 2) break;                 // all 31 bits are fixed
+        if (cnt <= 32u) {                      // uniform: rank the bin's keys directly
+#pragma unroll
+            for (int i = 0; i < EPT; ++i)
+                if ((key[i] >> shift) == prefix) list[atomicAdd(&scan[11], 1u)] = key[i];
+            __syncthreads();
+            if (warp == 0) {
+                const uint32_t my = (uint32_t)lane < cnt ? list[lane] : 0xFFFFFFFFu;
+                uint32_t below = 0;
+                for (uint32_t j = 0; j < cnt; ++j) {
+                    const uint32_t o = list[j];
+                    below += (o < my || (o == my && j < (uint32_t)lane)) ? 1u : 0u;
+                }
+                if ((uint32_t)lane < cnt && below == kk - 1u) scan[12] = my;
+            }
+            __syncthreads();
+            return scan[12];
+        }
     }
     return prefix;
 }
