@@ -262,7 +262,7 @@ int solo_codebook_v(int v_codebook, int bits, float* levels_host);
 float solo_default_beta1(int bits_m, int from_scratch);
 
 /*
- * Kernel selection.  0 (default): configurations with 2/3/4-bit states (any block size),
+ * Kernel selection.  0 (default): every width and block size with
  * the logarithmic second-moment quantizer, nearest rounding of the first moment and
  * eps >= 1e-12 run the streamlined kernel (fp32 or bf16 parameters), everything else the
  * general one.  1: always the general kernel.  Both produce the same packed state and the same

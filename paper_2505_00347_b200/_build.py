@@ -31,6 +31,7 @@ UNITS = [
     ("solo_fast_inst.cu", "solo_fast_bm2.o", ["-DSOLO_BM=2"]),
     ("solo_fast_inst.cu", "solo_fast_bm3.o", ["-DSOLO_BM=3"]),
     ("solo_fast_inst.cu", "solo_fast_bm4.o", ["-DSOLO_BM=4"]),
+    ("solo_fast_inst.cu", "solo_fast_bm8.o", ["-DSOLO_BM=8"]),
 ]
 
 

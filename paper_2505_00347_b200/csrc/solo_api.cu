@@ -206,7 +206,7 @@ int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
         s->tiles_total < (int64_t)1 << 31)
         k = solo::fast_kernel(s->bits_m, s->bits_v, s->block, a.param_bf16 != 0,
                               !a.l2 && !a.belief && a.fixed_alpha == 0.0f && a.round_v);
-    size_t dyn_smem = k ? solo::fast_kernel_smem() : 0;
+    size_t dyn_smem = k ? solo::fast_kernel_smem(s->bits_m, s->bits_v) : 0;
     if (!k) k = solo::step_kernel(s->bits_m, s->bits_v, cta_group);
     if (!k) return SOLO_EINVAL;
     int per_sm = solo::kernel_occupancy(k, dyn_smem);

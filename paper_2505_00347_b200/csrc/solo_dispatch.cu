@@ -20,11 +20,12 @@ StepKernel step_kernel(int bits_m, int bits_v, bool cta_group) {
 
 StepKernel fast_kernel(int bits_m, int bits_v, int block, bool param_bf16, bool plain) {
     const int bv = bits_index(bits_v);
-    if (bv < 0 || bv > 2) return nullptr;
+    if (bv < 0) return nullptr;
     switch (bits_m) {
         case 2: return fast_kernel_bm2(bv, block, param_bf16, plain);
         case 3: return fast_kernel_bm3(bv, block, param_bf16, plain);
         case 4: return fast_kernel_bm4(bv, block, param_bf16, plain);
+        case 8: return fast_kernel_bm8(bv, block, param_bf16, plain);
         default: return nullptr;
     }
 }

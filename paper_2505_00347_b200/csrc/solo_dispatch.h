@@ -28,7 +28,7 @@ inline int bits_index(int bits) {
 
 StepKernel step_kernel(int bits_m, int bits_v, bool cta_group);
 
-// Streamlined kernel (2/3/4-bit states, block 64, 128, 256 or 2048, fp32 or bf16 parameters); null
+// Streamlined kernel (2/3/4/8-bit states, block 64, 128, 256 or 2048, fp32 or bf16 parameters); null
 // outside that domain.  The caller additionally requires the logarithmic second-moment
 // quantizer, nearest rounding of the first moment and eps >= 1e-12.
 // `plain`: no L2 term in the gradient, no AdaBelief, base from the quantile, xi drawn (the
@@ -36,9 +36,10 @@ StepKernel step_kernel(int bits_m, int bits_v, bool cta_group);
 StepKernel fast_kernel_bm2(int bv_index, int block, bool param_bf16, bool plain);
 StepKernel fast_kernel_bm3(int bv_index, int block, bool param_bf16, bool plain);
 StepKernel fast_kernel_bm4(int bv_index, int block, bool param_bf16, bool plain);
+StepKernel fast_kernel_bm8(int bv_index, int block, bool param_bf16, bool plain);
 StepKernel fast_kernel(int bits_m, int bits_v, int block, bool param_bf16, bool plain);
-// Dynamic shared memory the streamlined kernels are launched with.
-size_t fast_kernel_smem();
+// Dynamic shared memory the streamlined kernel for these widths is launched with.
+size_t fast_kernel_smem(int bits_m, int bits_v);
 // Resident CTAs per SM of a step kernel launched with `dyn_smem` bytes of dynamic shared memory
 // (cached per device and kernel; opts the kernel in to that much shared memory), 0 on error.
 int kernel_occupancy(StepKernel k, size_t dyn_smem);

@@ -1,4 +1,4 @@
-// Streamlined fused step for the common configurations: 2/3/4-bit states, blocks of
+// Streamlined fused step for the common configurations: 2/3/4/8-bit states, blocks of
 // 64, 128, 256 or 2048 elements, fp32 or bf16 parameters, the paper's logarithmic quantizer for the
 // second moment, nearest rounding of the first moment, eps >= 1e-12.
 //
@@ -47,9 +47,12 @@ constexpr float LG2_REL = 0x1p-20f;
 
 constexpr uint32_t KEY_MAX = 0x7FFFFFFFu;    // sentinel key: above or equal to every valid key
 
-struct FastShared {
+// WM, WV: 32-bit words of packed codes per thread (1 up to 4-bit codes, 2 for 8-bit codes).
+template <int WM, int WV>
+struct FastSharedT {
     uint32_t sort[16][CTA];                  // rows 0..6: 2nd..8th smallest key of a thread; rows 7..15: sentinel
-    float tab[CTA / 8][32];                 // per group: K_v second-moment levels, then K_m first-moment levels
+    float tab[CTA / 8][32];                 // per group: second-moment levels (8-bit: alpha^0..15), then K_m
+                                            // first-moment levels (8-bit first moments use the codebook itself)
     uint4 xin[2][CTA / 8];                  // per group: bits of Delta_m', Delta_v', x_p
     float4 xout[2][CTA / 8];                // per group: 1/Delta_m', 1/Delta_v', 1/log2(alpha'), rounding limit
     uint32_t xflag[2][CTA / 8];             // bit 0: vanishing first moment, bit 1: vanishing second moment
@@ -59,13 +62,15 @@ struct FastShared {
     struct Stage {
         float4 p[2 * CTA];                   // 2048 parameters (bf16: the first half)
         uint4 g[CTA];                        // 2048 bf16 gradients
-        uint32_t cm[CTA + 4];                // packed codes of the tile, from a 16-byte boundary (64 * bits words + 2)
-        uint32_t cv[CTA + 4];
+        uint32_t cm[WM * CTA + 4];           // packed codes of the tile, from a 16-byte boundary (64 * bits words + 2)
+        uint32_t cv[WV * CTA + 4];
         float sc[3][CTA / 8 + 4];            // Delta_m, Delta_v, alpha of the tile's blocks, from a 16-byte boundary
     };
     alignas(16) Stage stage[2];
     alignas(8) unsigned long long mbar[2];
 };
+template <int BM, int BV>
+using FastShared = FastSharedT<(BM == 8 ? 2 : 1), (BV == 8 ? 2 : 1)>;
 
 // What a CTA carries from one tile to the next for the copy-ahead of inputs.
 struct Ahead {
@@ -122,7 +127,7 @@ __device__ __forceinline__ void halves_to_float(uint32_t w, float& lo, float& hi
 template <int W>
 struct CodeOffsets {
     uint32_t even, odd;
-    __device__ __forceinline__ explicit CodeOffsets(uint32_t c) {
+    __device__ __forceinline__ CodeOffsets(uint32_t c, uint32_t) {
         uint32_t me = 0;
 #pragma unroll
         for (int i = 0; i < 8; i += 2) me |= ((1u << W) - 1u) << (i * W);
@@ -135,6 +140,25 @@ struct CodeOffsets {
         asm("mul.lo.u32 %0, %1, %2;" : "=r"(top) : "r"(w), "r"(1u << (32 - (i + 1) * W)));
         return top >> (30 - W);
     }
+};
+
+// 8-bit codes: four per word (`lo`: elements 0..3, `hi`: elements 4..7); a byte is brought to
+// bits 2..9 by one shift and masked.  low4(i): byte offset of entry (code & 15) of a table of
+// floats; bit(i, k): bit k of the code.
+template <>
+struct CodeOffsets<8> {
+    uint32_t lo, hi;
+    __device__ __forceinline__ CodeOffsets(uint32_t l, uint32_t h) : lo(l), hi(h) {}
+    __device__ __forceinline__ uint32_t word(int i) const { return i < 4 ? lo : hi; }
+    __device__ __forceinline__ uint32_t operator()(int i) const {
+        const int j = i & 3;
+        return j == 0 ? (word(i) << 2) & 0x3FCu : (word(i) >> (8 * j - 2)) & 0x3FCu;
+    }
+    __device__ __forceinline__ uint32_t low4(int i) const {
+        const int j = i & 3;
+        return j == 0 ? (word(i) << 2) & 0x3Cu : (word(i) >> (8 * j - 2)) & 0x3Cu;
+    }
+    __device__ __forceinline__ bool bit(int i, int k) const { return ((word(i) >> (8 * (i & 3) + k)) & 1u) != 0; }
 };
 
 // Philox4x32-10 with the round keys taken from the kernel arguments.
@@ -226,11 +250,11 @@ __device__ __forceinline__ uint32_t warp_load_codes(const uint8_t* warp_base, in
 // bytes more when they do not start on it; readers add the offset.  The scalar arrays are
 // allocated in multiples of 16 bytes, so the copy never leaves them.
 template <int BM, int BV, int G, bool PBF>
-__device__ __forceinline__ void issue_tile_copy(const StepArgs& a, FastShared& s, uint32_t fill, const char* pt,
+__device__ __forceinline__ void issue_tile_copy(const StepArgs& a, FastShared<BM, BV>& s, uint32_t fill, const char* pt,
                                                 const char* gt, int64_t jb_tile) {
     constexpr int NG = CTA / G;
     constexpr uint32_t PBYTES = TILE * (PBF ? 2 : 4);
-    FastShared::Stage& st = s.stage[fill & 1u];
+    typename FastShared<BM, BV>::Stage& st = s.stage[fill & 1u];
     const uint32_t bar = smem_u32(&s.mbar[fill & 1u]);
     const int64_t bm0 = jb_tile * G * BM, bv0 = jb_tile * G * BV;   // byte offsets of the tile's codes
     const uint32_t bytes_m = CTA * BM + ((bm0 & 15) ? 16u : 0u), bytes_v = CTA * BV + ((bv0 & 15) ? 16u : 0u);
@@ -461,7 +485,7 @@ __device__ __forceinline__ void bar_sync(int id) {
 // `par` alternates between tiles (double buffering of the per-block exchange arrays); `ah`
 // carries the copy-ahead state; next_full / next_dtin describe the CTA's next tile.
 template <int BM, int BV, int G, bool FULL, bool PBF, bool PLAIN>
-__device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, const float* s_y,
+__device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>& s, const float* s_y,
                                           const float* s_mid, char* pbase, const char* gbase,
                                           const int64_t n, const int tin, const int64_t jb_tile,
                                           const int tensor, const int par, Ahead& ah, const bool next_full,
@@ -496,7 +520,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
 
     // ---- inputs ----
     float p[EPT], g[EPT];
-    uint32_t cm = 0, cv = 0;
+    uint32_t cm = 0, cv = 0, cm_hi = 0, cv_hi = 0;                // *_hi: elements 4..7 of 8-bit codes
     float dm = 0.0f, dv = 0.0f, al = 0.5f;
     if (FULL) {
         // Every full tile reads its inputs from a stage.  Copy number f uses stage f & 1 and
@@ -520,7 +544,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
             atomicOr(a.status, 2);
             ah.failed = true;
         }
-        const FastShared::Stage& st = s.stage[mine & 1u];
+        const typename FastShared<BM, BV>::Stage& st = s.stage[mine & 1u];
         const uint4 gw = st.g[tid];
         if constexpr (PBF) {
             const uint4 pw = reinterpret_cast<const uint4*>(st.p)[tid];
@@ -536,10 +560,16 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
             p[4] = p1.x; p[5] = p1.y; p[6] = p1.z; p[7] = p1.w;
         }
         const int wm = (int)((jb_tile * G * BM) & 15) >> 2, wv = (int)((jb_tile * G * BV) & 15) >> 2;   // word offsets
-        if constexpr (BM == 2) cm = reinterpret_cast<const uint16_t*>(st.cm + wm)[tid];
+        if constexpr (BM == 8) {
+            const uint2 c2 = reinterpret_cast<const uint2*>(st.cm + wm)[tid];
+            cm = c2.x; cm_hi = c2.y;
+        } else if constexpr (BM == 2) cm = reinterpret_cast<const uint16_t*>(st.cm + wm)[tid];
         else if constexpr (BM == 4) cm = st.cm[wm + tid];
         else cm = warp_codes_finish<BM>(lane < 24 ? st.cm[wm + warp * 24 + lane] : 0u, lane);
-        if constexpr (BV == 2) cv = reinterpret_cast<const uint16_t*>(st.cv + wv)[tid];
+        if constexpr (BV == 8) {
+            const uint2 c2 = reinterpret_cast<const uint2*>(st.cv + wv)[tid];
+            cv = c2.x; cv_hi = c2.y;
+        } else if constexpr (BV == 2) cv = reinterpret_cast<const uint16_t*>(st.cv + wv)[tid];
         else if constexpr (BV == 4) cv = st.cv[wv + tid];
         else cv = warp_codes_finish<BV>(lane < 24 ? st.cv[wv + warp * 24 + lane] : 0u, lane);
         const int so = (int)(jb_tile & 3) + grp;                 // the scalars were copied from a 16-byte boundary
@@ -563,8 +593,9 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
             }
         }
         if (have_block) {
-            cm = (uint32_t)load_codes<BM>(wcm + lane * BM);
-            cv = (uint32_t)load_codes<BV>(wcv + lane * BV);
+            const uint64_t cm64 = load_codes<BM>(wcm + lane * BM), cv64 = load_codes<BV>(wcv + lane * BV);
+            cm = (uint32_t)cm64; cm_hi = (uint32_t)(cm64 >> 32);
+            cv = (uint32_t)cv64; cv_hi = (uint32_t)(cv64 >> 32);
             dm = __ldg(a.scale_m + jb);
             dv = __ldg(a.scale_v + jb);
             al = __ldg(a.alpha + jb);
@@ -572,18 +603,31 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     }
 
     // ---- per-block level tables: alpha^k Delta_v and y_k Delta_m (Eq. 2) ----
+    // 8-bit second moments: the table holds the product of the first four factors of the
+    // square-and-multiply chain (alpha^(q & 15)); the other four are multiplied on per element.
+    // 8-bit first moments: no table, the codebook entry is scaled per element.
+    constexpr int KVT = BV == 8 ? 16 : KV;
     float* const tab = s.tab[grp];
+    float a2[BV];
+    a2[0] = al;
+#pragma unroll
+    for (int i = 1; i < BV; ++i) a2[i] = a2[i - 1] * a2[i - 1];
     {
-        float a2[BV];
-        a2[0] = al;
 #pragma unroll
-        for (int i = 1; i < BV; ++i) a2[i] = a2[i - 1] * a2[i - 1];
+        for (int r0 = 0; r0 < KVT; r0 += G)
+            if (r0 + gl < KVT) {
+                if constexpr (BV == 8) {
+                    const float a2lo[4] = {a2[0], a2[1], a2[2], a2[3]};
+                    tab[r0 + gl] = pow_sm<4>(a2lo, (uint32_t)(r0 + gl));
+                } else {
+                    tab[r0 + gl] = pow_sm<BV>(a2, (uint32_t)(r0 + gl)) * dv;
+                }
+            }
+        if constexpr (BM != 8) {
 #pragma unroll
-        for (int r0 = 0; r0 < KV; r0 += G)
-            if (r0 + gl < KV) tab[r0 + gl] = pow_sm<BV>(a2, (uint32_t)(r0 + gl)) * dv;
-#pragma unroll
-        for (int r0 = 0; r0 < KM; r0 += G)
-            if (r0 + gl < KM) tab[KV + r0 + gl] = s_y[r0 + gl] * dm;
+            for (int r0 = 0; r0 < KM; r0 += G)
+                if (r0 + gl < KM) tab[KVT + r0 + gl] = s_y[r0 + gl] * dm;
+        }
     }
     if constexpr (G == CTA) __syncthreads(); else __syncwarp();
 
@@ -597,16 +641,25 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     uint32_t mx_v = 0;
     float mx_m_f = 0.0f;                                         // max |m^| (a NaN element is passed over)
     const char* const tab_v = reinterpret_cast<const char*>(tab);
-    const char* const tab_m = reinterpret_cast<const char*>(tab + KV);
-    const CodeOffsets<BM> om4(cm);
-    const CodeOffsets<BV> ov4(cv);
+    const char* const tab_m = reinterpret_cast<const char*>(tab + KVT);
+    const CodeOffsets<BM> om4(cm, cm_hi);
+    const CodeOffsets<BV> ov4(cv, cv_hi);
     // the loop is instantiated twice so that the optimizer variant costs nothing per element
     auto ema = [&](auto belief_tag) {
         constexpr bool BELIEF = decltype(belief_tag)::value;
 #pragma unroll
     for (int i = 0; i < EPT; ++i) {
-        const float mt = *reinterpret_cast<const float*>(tab_m + om4(i));
-        const float vt = *reinterpret_cast<const float*>(tab_v + ov4(i));
+        float mt, vt;
+        if constexpr (BM == 8) mt = *reinterpret_cast<const float*>(reinterpret_cast<const char*>(s_y) + om4(i)) * dm;
+        else mt = *reinterpret_cast<const float*>(tab_m + om4(i));
+        if constexpr (BV == 8) {
+            float r = *reinterpret_cast<const float*>(tab_v + ov4.low4(i));
+#pragma unroll
+            for (int k = 4; k < 8; ++k) r = r * (ov4.bit(i, k) ? a2[k] : 1.0f);
+            vt = r * dv;
+        } else {
+            vt = *reinterpret_cast<const float*>(tab_v + ov4(i));
+        }
         const float gi = g[i];
         mh[i] = __fmaf_rn(a.beta1, mt, a.omb1 * gi);
         if (BELIEF) {                                            // AdaBelief: (g - m^)^2, plus eps
@@ -762,7 +815,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     const uint32_t zf = s.xflag[par][grp];
 
     // ---- first moment: nearest level (Eq. 1) ----
-    uint32_t om = 0;
+    uint32_t om = 0, om_hi = 0;                                   // om_hi: elements 4..7 of 8-bit codes
     {
         const float inv = sc.x;
         if constexpr (BM == 2 && FULL) {
@@ -800,7 +853,8 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
 #pragma unroll
                 for (int st = KM / 2; st >= 1; st >>= 1)
                     if (r > s_mid[q + st - 1]) q += st;
-                om = (om << BM) + ((FULL || i < nv) ? q : 0u);
+                uint32_t& dst = (BM == 8 && i >= 4) ? om_hi : om;
+                dst = (dst << BM) + ((FULL || i < nv) ? q : 0u);
             }
         }
     }
@@ -808,7 +862,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
     // ---- second moment: Eq. 6 ----
     // t = log_alpha(r) + xi is evaluated divided by K - 1, so that the clamp to [0, K-1] is the
     // saturation of the fused multiply-add; adding 1.5 * 2^23 to (K-1) * t rounds it to an integer.
-    uint32_t ov = 0;
+    uint32_t ov = 0, ov_hi = 0;
     {
         const float inv = sc.y, il = sc.z, lim = sc.w;
         constexpr float KM1 = (float)(KV - 1);
@@ -819,24 +873,27 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
         const float xs1 = round_v ? (float)(0x1p-16 / (KV - 1)) : 0.0f;
         const float xs0 = round_v ? (float)((-0.5 + 0x1p-17) / (KV - 1)) : 0.0f;
         float worst = 0.0f;
-        uint32_t acc = 0;
+        uint32_t acc = 0, acc_hi = 0;
 #pragma unroll
         for (int i = EPT - 1; i >= 0; --i) {
             const float r = vh[i] * inv;
             const float ts = __saturatef(__fmaf_rn(lg2_approx(r), ils, __fmaf_rn(dr[i], xs1, xs0)));
             const float u = __fmaf_rn(ts, KM1, MAGIC);
             worst = fmaxf(worst, fabsf(__fmaf_rn(ts, KM1, MAGIC - u)));
-            acc = acc * (1u << BV) + ((FULL || i < nv) ? __float_as_uint(u) : MAGIC_BITS);
+            uint32_t& dst = (BV == 8 && i >= 4) ? acc_hi : acc;
+            dst = dst * (1u << BV) + ((FULL || i < nv) ? __float_as_uint(u) : MAGIC_BITS);
         }
         uint32_t magic_sum = 0;
 #pragma unroll
-        for (int i = 0; i < EPT; ++i) magic_sum = (magic_sum << BV) + MAGIC_BITS;
+        for (int i = 0; i < (BV == 8 ? 4 : EPT); ++i) magic_sum = (magic_sum << BV) + MAGIC_BITS;
         ov = acc - magic_sum;
+        if constexpr (BV == 8) ov_hi = acc_hi - magic_sum;
         if (__any_sync(0xffffffffu, worst > lim)) {
             // some element of the warp is too close to a rounding boundary for the
             // approximate logarithm: evaluate the exact sequence for all eight
             const float x1 = round_v ? 0x1p-16f : 0.0f, x0 = round_v ? -0.5f + 0x1p-17f : 0.0f;
             ov = 0;
+            ov_hi = 0;
 #pragma unroll
             for (int i = EPT - 1; i >= 0; --i) {
                 const float r = vh[i] * inv;
@@ -846,28 +903,31 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared& s, cons
                     t = fminf(fmaxf(t, 0.0f), KM1);
                     q = (uint32_t)__float2int_rn(t);
                 }
-                ov = (ov << BV) + ((FULL || i < nv) ? q : 0u);
+                uint32_t& dst = (BV == 8 && i >= 4) ? ov_hi : ov;
+                dst = (dst << BV) + ((FULL || i < nv) ? q : 0u);
             }
         }
     }
-    if (zf & 1u) om = 0;
-    if (zf & 2u) ov = 0;
+    if (zf & 1u) { om = 0; om_hi = 0; }
+    if (zf & 2u) { ov = 0; ov_hi = 0; }
 
     // ---- store the codes ----
     if (FULL) {
-        warp_store_codes<BM>(wcm, lane, om);
-        warp_store_codes<BV>(wcv, lane, ov);
+        if constexpr (BM == 8) __stcs(reinterpret_cast<uint2*>(wcm) + lane, make_uint2(om, om_hi));
+        else warp_store_codes<BM>(wcm, lane, om);
+        if constexpr (BV == 8) __stcs(reinterpret_cast<uint2*>(wcv) + lane, make_uint2(ov, ov_hi));
+        else warp_store_codes<BV>(wcv, lane, ov);
     } else if (have_block) {
-        store_codes<BM>(wcm + lane * BM, om);
-        store_codes<BV>(wcv + lane * BV, ov);
+        store_codes<BM>(wcm + lane * BM, ((uint64_t)om_hi << 32) | om);
+        store_codes<BV>(wcv + lane * BV, ((uint64_t)ov_hi << 32) | ov);
     }
 }
 
 template <int BM, int BV, int G, bool PBF, bool PLAIN>
-__global__ void __launch_bounds__(CTA, 4) solo_step_fast_kernel(const StepArgs a) {
+__global__ void __launch_bounds__(CTA, (BM == 8 || BV == 8) ? 3 : 4) solo_step_fast_kernel(const StepArgs a) {
     constexpr int KM = 1 << BM;
-    extern __shared__ __align__(16) unsigned char fast_smem[];   // sizeof(FastShared), above the static 48 KB limit
-    FastShared& s = *reinterpret_cast<FastShared*>(fast_smem);
+    extern __shared__ __align__(16) unsigned char fast_smem[];   // sizeof(FastShared<BM, BV>), above the static 48 KB limit
+    FastShared<BM, BV>& s = *reinterpret_cast<FastShared<BM, BV>*>(fast_smem);
     __shared__ float s_y[KM];
     __shared__ float s_mid[KM];
     const int tid = threadIdx.x;

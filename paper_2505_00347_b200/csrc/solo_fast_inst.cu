@@ -1,9 +1,9 @@
-// Instantiations of the streamlined step kernel for one first-moment width (SOLO_BM = 2, 3, 4).
+// Instantiations of the streamlined step kernel for one first-moment width (SOLO_BM = 2, 3, 4, 8).
 #include "solo_dispatch.h"
 #include "solo_fast.cuh"
 
 #ifndef SOLO_BM
-#error "compile with -DSOLO_BM=2|3|4"
+#error "compile with -DSOLO_BM=2|3|4|8"
 #endif
 
 #define SOLO_CAT_(a, b) a##b
@@ -14,15 +14,16 @@ namespace solo {
 #define SOLO_ROW(BV, PBF, PLAIN)                                                                            \
     {solo_step_fast_kernel<SOLO_BM, BV, 8, PBF, PLAIN>, solo_step_fast_kernel<SOLO_BM, BV, 16, PBF, PLAIN>, \
      solo_step_fast_kernel<SOLO_BM, BV, 32, PBF, PLAIN>, solo_step_fast_kernel<SOLO_BM, BV, 256, PBF, PLAIN>}
-#define SOLO_PLANE(PBF, PLAIN) {SOLO_ROW(2, PBF, PLAIN), SOLO_ROW(3, PBF, PLAIN), SOLO_ROW(4, PBF, PLAIN)}
+#define SOLO_PLANE(PBF, PLAIN) \
+    {SOLO_ROW(2, PBF, PLAIN), SOLO_ROW(3, PBF, PLAIN), SOLO_ROW(4, PBF, PLAIN), SOLO_ROW(8, PBF, PLAIN)}
 
 StepKernel SOLO_CAT(fast_kernel_bm, SOLO_BM)(int bv_index, int block, bool param_bf16, bool plain) {
-    static const StepKernel table[2][2][3][4] = {
+    static const StepKernel table[2][2][4][4] = {
         {SOLO_PLANE(false, false), SOLO_PLANE(true, false)},
         {SOLO_PLANE(false, true), SOLO_PLANE(true, true)},
     };
     const int g = block == 64 ? 0 : block == 128 ? 1 : block == 256 ? 2 : block == 2048 ? 3 : -1;
-    if (bv_index < 0 || bv_index > 2 || g < 0) return nullptr;
+    if (bv_index < 0 || bv_index > 3 || g < 0) return nullptr;
     return table[plain ? 1 : 0][param_bf16 ? 1 : 0][bv_index][g];
 }
 
@@ -54,7 +55,11 @@ cudaError_t launch_fast_log_check(uint32_t lo, uint32_t hi, float* out_max_exces
     return cudaGetLastError();
 }
 float fast_log_abs_bound() { return LG2_ABS; }
-size_t fast_kernel_smem() { return sizeof(FastShared); }
+size_t fast_kernel_smem(int bits_m, int bits_v) {
+    const bool m8 = bits_m == 8, v8 = bits_v == 8;
+    return m8 ? (v8 ? sizeof(FastSharedT<2, 2>) : sizeof(FastSharedT<2, 1>))
+              : (v8 ? sizeof(FastSharedT<1, 2>) : sizeof(FastSharedT<1, 1>));
+}
 #endif
 
 }  // namespace solo

@@ -84,7 +84,8 @@ def test_bits_and_blocks_random_state(bits_m, bits_v, block):
     assert rep.exempt_m + rep.exempt_v <= 3
 
 
-@pytest.mark.parametrize("bits_m,bits_v,block", [(2, 3, 128), (3, 2, 64), (4, 4, 256), (2, 2, 2048)])
+@pytest.mark.parametrize("bits_m,bits_v,block", [(2, 3, 128), (3, 2, 64), (4, 4, 256), (2, 2, 2048), (8, 4, 64),
+                                                 (2, 8, 256)])
 @pytest.mark.parametrize("hk", [dict(adamw=0, weight_decay=0.1), dict(round_v=0, belief=1),
                                 dict(fixed_alpha=0.5, param_dtype=1)])
 def test_mode_flags_at_other_widths(bits_m, bits_v, block, hk):
@@ -149,7 +150,7 @@ def test_baseline_second_moment_codebooks(sel, bits_v, block):
 
 
 @pytest.mark.parametrize("param_round", [0, 1])
-@pytest.mark.parametrize("bits_m,bits_v,block", [(2, 3, 128), (4, 4, 64), (3, 2, 256), (4, 3, 2048)])
+@pytest.mark.parametrize("bits_m,bits_v,block", [(2, 3, 128), (4, 4, 64), (3, 2, 256), (4, 3, 2048), (8, 8, 128)])
 def test_bf16_parameters_every_kernel(bits_m, bits_v, block, param_round):
     """bf16 parameters through the streamlined kernel (full tiles from the staged copies, ragged
     tails from direct loads) and the general one, nearest and stochastic rounding; run_lockstep
