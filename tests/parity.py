@@ -208,7 +208,7 @@ def run_lockstep(sizes, bits_m, bits_v, block, hyper_kw, steps, grads_fn, params
                 ok |= np.abs(gp.astype(np.float64) - wp) <= RTOL * np.abs(wp) + ATOL + update_tol * upd
             assert ok.all(), (f"{where} tensor {i} params", int((~ok).sum()), gp[~ok][:4], wp[~ok][:4])
             if bf16p and not free_run:
-                # bf16 parameters take the general kernel (IEEE division and square root): the
+                # both kernels compute the update of bf16 parameters with IEEE division and square root: the
                 # binary32 value that is rounded, and with stochastic rounding its draw, are the
                 # oracle's, so the stored patterns are identical
                 assert np.array_equal(synth.bf16_bits(gparams[i].cpu()), oparams[i]), f"{where} tensor {i} bf16 bits"

@@ -76,10 +76,12 @@ def test_static_entry_point_matches_library_state_twice():
     from paper_2505_00347_b200 import binding as B
     # first call sequence: streamlined kernel (2/3 bit, block 128), ragged multi-tensor list
     _run_pair(B, (2048 * 3 + 77, 1, 128, 5000), 2, 3, 128, steps=2, seed=7)
-    # second, with another list and widths (general kernel: 8-bit, block 2048), from a random state
+    # second, with another list and widths (8-bit first moment, block 2048), from a random state
     sizes = (2048 * 2 + 5, 300, 4097)
     st0 = synth.make_state(sizes, 8, 4, 2048, seed=99)
     _run_pair(B, sizes, 8, 4, 2048, steps=2, seed=8, state0=st0)
+    # and through the general kernel (stochastic rounding of the first moment)
+    _run_pair(B, sizes, 8, 4, 2048, steps=2, seed=8, state0=st0, round_m=1)
     # third: a baseline codebook for the second moment (its table also lives in the fixed array)
     _run_pair(B, (2048 + 9, 640), 4, 4, 128, steps=2, seed=9, v_codebook=3)
 
