@@ -262,12 +262,16 @@ int solo_codebook_v(int v_codebook, int bits, float* levels_host);
 float solo_default_beta1(int bits_m, int from_scratch);
 
 /*
- * Kernel selection.  0 (default): every width and block size with
- * the logarithmic second-moment quantizer, nearest rounding of the first moment and
- * eps >= 1e-12 run the streamlined kernel (fp32 or bf16 parameters), everything else the
- * general one.  1: always the general kernel.  Both produce the same packed state and the same
- * bf16 parameters; the streamlined kernel's fp32 parameters differ from the IEEE sequence of
- * divisions and square roots by at most a few 1e-7 of the update term.  Process-wide.
+ * Kernel selection.  0 (default): every width and block size with the logarithmic
+ * second-moment quantizer, nearest rounding of the first moment and eps >= 1e-12 runs the
+ * streamlined kernel (fp32 or bf16 parameters), everything else the general one; the paper's
+ * default configuration (2-bit / 3-bit states, block 128, fp32 parameters, plain Adam(W) step,
+ * p = 0.1) runs its full tiles in a kernel with sixteen elements per thread and the remaining
+ * tiles in the streamlined kernel (two launches).  1: always the general kernel.  2: like 0
+ * without the sixteen-per-thread kernel.  All produce the same packed state and the same bf16
+ * parameters; the fp32 parameters of the two faster kernels are identical to each other and
+ * differ from the IEEE sequence of divisions and square roots by at most a few 1e-7 of the
+ * update term.  Process-wide.
  */
 int solo_set_kernel_policy(int policy);
 

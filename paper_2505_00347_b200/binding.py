@@ -377,7 +377,8 @@ def default_beta1(bits_m: int, from_scratch: bool = False) -> float:
 
 
 def set_kernel_policy(policy: int) -> None:
-    """0: streamlined kernel where it applies (default); 1: always the general kernel."""
+    """0: fastest kernel that applies (default); 1: always the general kernel; 2: like 0 without the
+    sixteen-elements-per-thread kernel."""
     _check(lib().solo_set_kernel_policy(policy), "solo_set_kernel_policy")
 
 

@@ -54,7 +54,7 @@ struct HostPipe {
 namespace {
 
 std::atomic<int64_t> g_launches{0};
-std::atomic<int> g_policy{0};          // 0: pick the streamlined kernel where it applies; 1: general kernel only
+std::atomic<int> g_policy{0};          // 0: fastest kernel that applies; 1: general kernel only; 2: no sixteen-per-thread kernel
 
 bool valid_bits(int b) { return b == 2 || b == 3 || b == 4 || b == 8; }
 bool valid_block(int b) { return b == 64 || b == 128 || b == 256 || b == 2048; }
@@ -199,28 +199,44 @@ void reduce_hyper(const solo_hyper_t* h, int64_t step, int block, StepArgs& a) {
     }
 }
 
-int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
-    const bool cta_group = s->block == 2048;
-    solo::StepKernel k = nullptr;
-    if (g_policy.load(std::memory_order_relaxed) == 0 && !a.round_m && !a.tables_v && a.eps >= 1e-12f &&
-        s->tiles_total < (int64_t)1 << 31)
-        k = solo::fast_kernel(s->bits_m, s->bits_v, s->block, a.param_bf16 != 0,
-                              !a.l2 && !a.belief && a.fixed_alpha == 0.0f && a.round_v);
-    size_t dyn_smem = k ? solo::fast_kernel_smem(s->bits_m, s->bits_v) : 0;
-    if (!k) k = solo::step_kernel(s->bits_m, s->bits_v, cta_group);
-    if (!k) return SOLO_EINVAL;
-    int per_sm = solo::kernel_occupancy(k, dyn_smem);
+int launch_kernel(solo::StepKernel k, const StepArgs& a, int device, int threads, size_t dyn_smem,
+                  cudaStream_t stream) {
+    int per_sm = solo::kernel_occupancy(k, dyn_smem, threads);
     if (per_sm <= 0) return SOLO_ECUDA;
-    int64_t grid = std::min<int64_t>(a.total_tiles - a.tile_first, (int64_t)sm_count(s->device) * per_sm);
+    int64_t grid = std::min<int64_t>(a.total_tiles - a.tile_first, (int64_t)sm_count(device) * per_sm);
     if (grid < 1) return SOLO_EINVAL;
     void* params[] = {(void*)&a};
-    cudaError_t e = cudaLaunchKernel((const void*)k, dim3((unsigned)grid), dim3(solo::CTA), params, dyn_smem, stream);
+    cudaError_t e = cudaLaunchKernel((const void*)k, dim3((unsigned)grid), dim3((unsigned)threads), params, dyn_smem, stream);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return SOLO_ECUDA;
     }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return SOLO_OK;
+}
+
+int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
+    const bool cta_group = s->block == 2048;
+    const int policy = g_policy.load(std::memory_order_relaxed);
+    const bool streamlined = policy != 1 && !a.round_m && !a.tables_v && a.eps >= 1e-12f &&
+                             s->tiles_total < (int64_t)1 << 31;
+    const bool plain = !a.l2 && !a.belief && a.fixed_alpha == 0.0f && a.round_v;
+    if (streamlined && policy == 0 && s->bits_m == 2 && s->bits_v == 3 && s->block == 128 && !a.param_bf16 &&
+        plain && a.k_full == 13) {
+        // the paper's default configuration: full tiles by the sixteen-per-thread kernel, whatever it
+        // leaves (tails, tensors that are not 16-byte aligned) by the streamlined kernel
+        int rc = launch_kernel(solo::fast16_kernel(), a, s->device, solo::CTA16, solo::fast16_kernel_smem(), stream);
+        if (rc) return rc;
+        const bool all_full = !a.param_list && s->num_tensors == 1 && s->numel[0] % solo::TILE == 0;
+        if (all_full) return SOLO_OK;
+        a.only_partial = 1;
+    }
+    solo::StepKernel k = nullptr;
+    if (streamlined) k = solo::fast_kernel(s->bits_m, s->bits_v, s->block, a.param_bf16 != 0, plain);
+    size_t dyn_smem = k ? solo::fast_kernel_smem(s->bits_m, s->bits_v) : 0;
+    if (!k) k = solo::step_kernel(s->bits_m, s->bits_v, cta_group);
+    if (!k) return SOLO_EINVAL;
+    return launch_kernel(k, a, s->device, solo::CTA, dyn_smem, stream);
 }
 
 void fill_state_args(const solo_state* s, StepArgs& a) {
@@ -858,7 +874,7 @@ float solo_default_beta1(int bits_m, int from_scratch) {
 }
 
 int solo_set_kernel_policy(int policy) {
-    if (policy != 0 && policy != 1) return SOLO_EINVAL;
+    if (policy < 0 || policy > 2) return SOLO_EINVAL;
     g_policy.store(policy, std::memory_order_relaxed);
     return SOLO_OK;
 }

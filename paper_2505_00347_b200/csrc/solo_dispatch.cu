@@ -30,7 +30,7 @@ StepKernel fast_kernel(int bits_m, int bits_v, int block, bool param_bf16, bool 
     }
 }
 
-int kernel_occupancy(StepKernel k, size_t dyn_smem) {
+int kernel_occupancy(StepKernel k, size_t dyn_smem, int threads) {
     static std::mutex mu;
     static std::map<std::pair<int, const void*>, int> cache;    // per device: the opt-in below is per context
     if (!k) return 0;
@@ -46,7 +46,7 @@ int kernel_occupancy(StepKernel k, size_t dyn_smem) {
     int n = 0;
     if ((dyn_smem > 0 &&
          cudaFuncSetAttribute((const void*)k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem) != cudaSuccess) ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k, CTA, dyn_smem) != cudaSuccess || n <= 0) {
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k, threads, dyn_smem) != cudaSuccess || n <= 0) {
         cudaGetLastError();
         return 0;
     }

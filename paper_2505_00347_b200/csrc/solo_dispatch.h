@@ -38,11 +38,17 @@ StepKernel fast_kernel_bm3(int bv_index, int block, bool param_bf16, bool plain)
 StepKernel fast_kernel_bm4(int bv_index, int block, bool param_bf16, bool plain);
 StepKernel fast_kernel_bm8(int bv_index, int block, bool param_bf16, bool plain);
 StepKernel fast_kernel(int bits_m, int bits_v, int block, bool param_bf16, bool plain);
+// Sixteen elements per thread: 2-bit / 3-bit states, block 128, fp32 parameters, the plain step
+// with p-quantile rank 13; full tiles of aligned tensors only (the rest is left to a launch of
+// the streamlined kernel with StepArgs::only_partial).  Launched with CTA16 = 128 threads.
+constexpr int CTA16 = 128;         // threads per CTA of that kernel
+StepKernel fast16_kernel();
+size_t fast16_kernel_smem();
 // Dynamic shared memory the streamlined kernel for these widths is launched with.
 size_t fast_kernel_smem(int bits_m, int bits_v);
 // Resident CTAs per SM of a step kernel launched with `dyn_smem` bytes of dynamic shared memory
 // (cached per device and kernel; opts the kernel in to that much shared memory), 0 on error.
-int kernel_occupancy(StepKernel k, size_t dyn_smem);
+int kernel_occupancy(StepKernel k, size_t dyn_smem, int threads = CTA);
 
 // Exhaustive comparison of the hardware lg2 approximation with log2_sp (tests).
 cudaError_t launch_fast_log_check(uint32_t lo, uint32_t hi, float* out_max_excess, cudaStream_t stream);

@@ -186,6 +186,23 @@ def test_stochastic_bf16_rounding_is_unbiased_on_the_device():
         st.destroy()
 
 
+def test_default_configuration_all_three_kernels():
+    """2-bit / 3-bit, block 128, plain step: the sixteen-per-thread kernel (policy 0: full tiles
+    there, the rest in the streamlined kernel), the streamlined kernel alone (2) and the general
+    kernel (1) against one oracle run; tensors with many full tiles, tails and tiny tensors, zero
+    blocks, ties, from a random state and from zero."""
+    sizes = (2048 * 9 + 700, 3, 2048 * 4, 2048 + 128, 127, 2048 * 2 + 1)
+    w = synth.workload(4, sizes=sizes)
+    params, gf = _inputs(w)
+    hk = dict(lr=2e-5, beta1=0.5, beta2=0.999, weight_decay=0.0, seed=1234)
+    st0 = synth.make_state(sizes, 2, 3, 128, seed=5)
+    run_lockstep(sizes, 2, 3, 128, hk, 3, gf, params, state0=st0, policies=(0, 2, 1))
+    run_lockstep(sizes, 2, 3, 128, hk, 4, gf, params, policies=(0, 2, 1))
+    w1 = synth.workload(1, sizes=(2048 * 6,))
+    p1, g1 = _inputs(w1)
+    run_lockstep(w1.sizes, 2, 3, 128, hk, 3, g1, p1, policies=(0, 2), multi=False)   # one launch: all tiles full
+
+
 def test_streamlined_kernel_rounding_guard_is_sound():
     """The streamlined kernel trusts lg2.approx to within abs + rel |log2 x| of the exact
     operation sequence; checked here for EVERY binary32 in [2^-100, 2) with half the constants."""
