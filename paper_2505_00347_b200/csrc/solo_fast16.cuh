@@ -23,9 +23,8 @@ static_assert(CTA16 * EPT16 == TILE, "same tile as the other kernels");
 
 struct Fast16Shared {
     // Sorted keys of the threads, one column per thread: row j holds the (j+2)-th smallest key.
-    // The column stride is CTA words (the pop advances by that constant); 128 columns are used.
     // Twelve rounds of popping read rows 0..11 at most.
-    uint32_t sort[12][CTA];
+    uint32_t sort[12][CTA16];
     float tab[16][16];                   // per block: 8 second-moment levels, then 4 first-moment levels
     uint4 xin[2][16];                    // per block: bits of Delta_m', Delta_v', x_p
     float4 xout[2][16];                  // per block: 1/Delta_m', 1/Delta_v', 1/log2(alpha'), rounding limit
@@ -76,6 +75,21 @@ __device__ __forceinline__ void sort16_low13(uint32_t (&k)[EPT16]) {
     SOLO_CS(3, 5); SOLO_CS(7, 9); SOLO_CS(11, 13);
     SOLO_CS(1, 2); SOLO_CS(3, 4); SOLO_CS(5, 6); SOLO_CS(7, 8); SOLO_CS(9, 10); SOLO_CS(11, 12);
 #undef SOLO_CS
+}
+
+// One selection round over groups of eight lanes, as pop_round in solo_fast.cuh (columns of
+// CTA16 words; at most twelve rounds, so no clamp).
+template <bool LAST>
+__device__ __forceinline__ uint32_t pop_round16(uint32_t& head, int& off, const uint32_t* col, uint32_t le,
+                                                uint32_t self, bool hi) {
+    if constexpr (LAST) return seg_min_v<8>(head, hi);
+    const uint32_t nxt = col[off];
+    const uint32_t tgt = seg_min_v<8>(head, hi);
+    const uint32_t upto = __ballot_sync(0xffffffffu, head == tgt) & le;
+    // if (upto == self) { head = nxt; off += CTA16; }
+    asm("{\n\t.reg .pred p;\n\tsetp.eq.u32 p, %2, %3;\n\t@p mov.u32 %0, %4;\n\t@p add.s32 %1, %1, %5;\n\t}"
+        : "+r"(head), "+r"(off) : "r"(upto), "r"(self), "r"(nxt), "n"(CTA16));
+    return tgt;
 }
 
 // Bulk copies of one full tile's inputs into stage `fill & 1` (one thread).  With blocks of 128
@@ -209,8 +223,19 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared& s, 
         sort16_low13(key);
         uint32_t* const col = &s.sort[0][tid];
 #pragma unroll
-        for (int j = 1; j <= 12; ++j) col[(j - 1) * CTA] = key[j] ^ vflip;
-        x_p = select_kth<G, true>(key[0] ^ vflip, col, 13, hi, update2) ^ vflip;
+        for (int j = 1; j <= 12; ++j) col[(j - 1) * CTA16] = key[j] ^ vflip;
+        // twelve rounds pop the twelve smallest keys of the block, the thirteenth minimum is x_p;
+        // the parameter updates are issued between the rounds
+        const uint32_t self = 1u << lane;
+        const uint32_t le = (self | (self - 1u)) & (0xFFu << (lane & ~(G - 1)));
+        uint32_t head = key[0] ^ vflip;
+        int off = 0;
+#pragma unroll
+        for (int r = 0; r < 12; ++r) {
+            pop_round16<false>(head, off, col, le, self, hi);
+            if (r < 8) update2(r);
+        }
+        x_p = pop_round16<true>(head, off, col, le, self, hi) ^ vflip;
     }
 
     // ---- per-block scalars by the first warp; the others draw xi meanwhile ----
@@ -334,7 +359,7 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared& s, 
     }
 }
 
-__global__ void __launch_bounds__(CTA16, 4) solo_step_fast16_kernel(const StepArgs a) {
+__global__ void __launch_bounds__(CTA16, 6) solo_step_fast16_kernel(const StepArgs a) {
     extern __shared__ __align__(16) unsigned char fast16_smem[];
     Fast16Shared& s = *reinterpret_cast<Fast16Shared*>(fast16_smem);
     __shared__ float s_y[4];
