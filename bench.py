@@ -339,7 +339,7 @@ def main():
                     help="bf16 parameters: 1 nearest-even, 2 stochastic rounding (default 0: fp32)")
     ap.add_argument("--cpu-sample", type=int, default=1 << 27)
     ap.add_argument("--e2e-steps", type=int, default=2)
-    ap.add_argument("--policy", type=int, default=0, help="kernel policy: 0 fastest that applies, 1 general, 2 without the sixteen-per-thread kernel")
+    ap.add_argument("--policy", type=int, default=0, help="kernel policy: 0 fastest that applies, 1 general, 2 without / 3 always with the sixteen-per-thread kernel")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -378,7 +378,7 @@ def default_beta1(bits_m: int, from_scratch: bool = False) -> float:
 
 def set_kernel_policy(policy: int) -> None:
     """0: fastest kernel that applies (default); 1: always the general kernel; 2: like 0 without the
-    sixteen-elements-per-thread kernel."""
+    sixteen-elements-per-thread kernel; 3: that kernel wherever it exists, whatever the tensor sizes."""
     _check(lib().solo_set_kernel_policy(policy), "solo_set_kernel_policy")
 
 

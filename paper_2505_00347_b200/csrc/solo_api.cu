@@ -54,7 +54,8 @@ struct HostPipe {
 namespace {
 
 std::atomic<int64_t> g_launches{0};
-std::atomic<int> g_policy{0};          // 0: fastest kernel that applies; 1: general kernel only; 2: no sixteen-per-thread kernel
+std::atomic<int> g_policy{0};          // 0: fastest kernel that applies; 1: general kernel only; 2: no sixteen-per-thread
+                                       // kernel; 3: sixteen-per-thread kernel wherever it exists
 
 bool valid_bits(int b) { return b == 2 || b == 3 || b == 4 || b == 8; }
 bool valid_block(int b) { return b == 64 || b == 128 || b == 256 || b == 2048; }
@@ -221,11 +222,17 @@ int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
     const bool streamlined = policy != 1 && !a.round_m && !a.tables_v && a.eps >= 1e-12f &&
                              s->tiles_total < (int64_t)1 << 31;
     const bool plain = !a.l2 && !a.belief && a.fixed_alpha == 0.0f && a.round_v;
-    if (streamlined && policy == 0 && s->bits_m == 2 && s->bits_v == 3 && s->block == 128 && !a.param_bf16 &&
-        plain && a.k_full == 13) {
-        // the paper's default configuration: full tiles by the sixteen-per-thread kernel, whatever it
-        // leaves (tails, tensors that are not 16-byte aligned) by the streamlined kernel
-        int rc = launch_kernel(solo::fast16_kernel(), a, s->device, solo::CTA16, solo::fast16_kernel_smem(), stream);
+    solo::StepKernel k16 = nullptr;
+    // worth its second launch and its 128-thread CTAs on large tensors only: measured faster on the
+    // 7B-shaped set and on one 268M-element tensor, slower on sets of small tensors
+    const bool large = s->tiles_total >= (int64_t)4096 * s->num_tensors;
+    if (streamlined && ((policy == 0 && large) || policy == 3) && s->block == 128 && !a.param_bf16 && plain &&
+        a.k_full == 13)
+        k16 = solo::fast16_kernel(s->bits_m, s->bits_v);
+    if (k16) {
+        // blocks of 128, plain step: full tiles by the sixteen-per-thread kernel, whatever it leaves
+        // (tails, tensors that are not 16-byte aligned) by the streamlined kernel
+        int rc = launch_kernel(k16, a, s->device, solo::CTA16, solo::fast16_kernel_smem(s->bits_m, s->bits_v), stream);
         if (rc) return rc;
         const bool all_full = !a.param_list && s->num_tensors == 1 && s->numel[0] % solo::TILE == 0;
         if (all_full) return SOLO_OK;
@@ -874,7 +881,7 @@ float solo_default_beta1(int bits_m, int from_scratch) {
 }
 
 int solo_set_kernel_policy(int policy) {
-    if (policy < 0 || policy > 2) return SOLO_EINVAL;
+    if (policy < 0 || policy > 3) return SOLO_EINVAL;
     g_policy.store(policy, std::memory_order_relaxed);
     return SOLO_OK;
 }

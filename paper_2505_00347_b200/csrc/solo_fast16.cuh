@@ -1,6 +1,7 @@
-// Sixteen elements per thread: the streamlined step for the paper's default configuration
-// (2-bit first moment, 3-bit second moment, blocks of 128, fp32 parameters, the plain step:
-// no L2 term in the gradient, no AdaBelief, base from the p = 0.1 quantile, xi drawn).
+// Sixteen elements per thread: the streamlined step for the paper's default block size and
+// plain step (2/3/4-bit states, of which 2-bit first moments are instantiated; blocks of 128,
+// fp32 parameters; no L2 term in the gradient, no AdaBelief, base from the p = 0.1 quantile, xi
+// drawn).
 //
 // Same arithmetic, element for element, as solo_step_fast_kernel (solo_fast.cuh); what changes
 // is the work split.  A CTA of 128 threads owns a tile of 2048 consecutive elements, a thread
@@ -21,20 +22,23 @@ namespace solo {
 constexpr int EPT16 = 16;               // elements per thread
 static_assert(CTA16 * EPT16 == TILE, "same tile as the other kernels");
 
+template <int BM, int BV>
 struct Fast16Shared {
     // Sorted keys of the threads, one column per thread: row j holds the (j+2)-th smallest key.
     // Twelve rounds of popping read rows 0..11 at most.
     uint32_t sort[12][CTA16];
-    float tab[16][16];                   // per block: 8 second-moment levels, then 4 first-moment levels
+    float tab[16][(1 << BV) + (1 << BM)]; // per block: K_v second-moment levels, then K_m first-moment levels
     uint4 xin[2][16];                    // per block: bits of Delta_m', Delta_v', x_p
     float4 xout[2][16];                  // per block: 1/Delta_m', 1/Delta_v', 1/log2(alpha'), rounding limit
     uint32_t xflag[2][16];
-    alignas(16) uint32_t cout[4][48];    // per warp: the packed 3-bit codes of its 512 elements, for 128-bit stores
+    // per 3-bit moment and warp: the packed codes of the warp's 512 elements, for 128-bit stores
+    static constexpr int N3 = (BM == 3 ? 1 : 0) + (BV == 3 ? 1 : 0);
+    alignas(16) uint32_t cout[N3 > 0 ? N3 : 1][4][48];
     struct Stage {
         float4 p[TILE / 4];              // 2048 parameters
         uint4 g[TILE / 8];               // 2048 bf16 gradients
-        uint32_t cm[CTA16 + 4];          // 2-bit codes of the tile: 512 bytes
-        uint32_t cv[192 + 4];            // 3-bit codes of the tile: 768 bytes
+        uint32_t cm[64 * BM + 4];        // packed codes of the tile: 256 * bits bytes
+        uint32_t cv[64 * BV + 4];
         float sc[3][16 + 4];             // Delta_m, Delta_v, alpha of the 16 blocks, from a 16-byte boundary
     };
     alignas(16) Stage stage[2];
@@ -56,6 +60,47 @@ struct CodeOffsets16x2 {
         return top >> 28;
     }
 };
+
+// The thread's sixteen BITS-bit codes as two words of eight codes each, from the tile's staged
+// code words (thread t owns bytes [2 * BITS * t, 2 * BITS * (t + 1)) of them).
+template <int BITS>
+__device__ __forceinline__ void load_codes16(const uint32_t* st, int tid, uint32_t (&h)[2]) {
+    if constexpr (BITS == 2) {
+        const uint32_t c = st[tid];
+        h[0] = c & 0xFFFFu; h[1] = c >> 16;
+    } else if constexpr (BITS == 4) {
+        const uint2 c = reinterpret_cast<const uint2*>(st)[tid];
+        h[0] = c.x; h[1] = c.y;
+    } else {
+        static_assert(BITS == 3, "2, 3 or 4 bits");
+        const int cw = (6 * tid) >> 2, cs = ((6 * tid) & 3) * 8;  // 48 bits from byte 6 * tid; cs is 0 or 16
+        const uint32_t w0 = st[cw], w1 = st[cw + 1];
+        const uint32_t c32 = __funnelshift_r(w0, w1, cs);         // bits 0..31
+        const uint32_t c16 = (w1 >> cs) & 0xFFFFu;                // bits 32..47
+        h[0] = c32 & 0xFFFFFFu; h[1] = (c32 >> 24) | (c16 << 8);
+    }
+}
+// The reverse, to the tile's codes in global memory (`tile_codes`: their first byte).  3-bit codes
+// (48 bits per thread) go through `stage` (48 words of the warp) so that twelve lanes store the
+// warp's 192 bytes as 128-bit words.
+template <int BITS>
+__device__ __forceinline__ void store_codes16(uint8_t* tile_codes, uint32_t* stage, int tid, const uint32_t (&h)[2]) {
+    if constexpr (BITS == 2) {
+        __stcs(reinterpret_cast<uint32_t*>(tile_codes) + tid, h[0] | (h[1] << 16));
+    } else if constexpr (BITS == 4) {
+        __stcs(reinterpret_cast<uint2*>(tile_codes) + tid, make_uint2(h[0], h[1]));
+    } else {
+        const int lane = tid & 31, warp = tid >> 5;
+        unsigned short* const half = reinterpret_cast<unsigned short*>(stage) + 3 * lane;
+        half[0] = (unsigned short)h[0];
+        half[1] = (unsigned short)((h[0] >> 16) | (h[1] << 8));
+        half[2] = (unsigned short)(h[1] >> 8);
+        __syncwarp();
+        if (lane < 12)
+            __stcs(reinterpret_cast<uint4*>(tile_codes + warp * 192) + lane, reinterpret_cast<const uint4*>(stage)[lane]);
+        __syncwarp();
+    }
+}
 
 // Sorts sixteen keys so that key[0..12] are the thirteen smallest in ascending order (Batcher's
 // odd-even merge sort without the one exchange that only orders key[13], key[14]).
@@ -93,19 +138,20 @@ __device__ __forceinline__ uint32_t pop_round16(uint32_t& head, int& off, const 
 }
 
 // Bulk copies of one full tile's inputs into stage `fill & 1` (one thread).  With blocks of 128
-// the tile's 2-bit and 3-bit codes start on 16-byte boundaries (32 and 48 bytes per block); the
-// per-block scalars are copied from the boundary at or below the first.
-__device__ __forceinline__ void issue_tile_copy16(const StepArgs& a, Fast16Shared& s, uint32_t fill, const char* pt,
-                                                  const char* gt, int64_t jb_tile) {
-    Fast16Shared::Stage& st = s.stage[fill & 1u];
+// the tile's codes start on 16-byte boundaries (16 * bits bytes per block); the per-block scalars
+// are copied from the boundary at or below the first.
+template <int BM, int BV>
+__device__ __forceinline__ void issue_tile_copy16(const StepArgs& a, Fast16Shared<BM, BV>& s, uint32_t fill,
+                                                  const char* pt, const char* gt, int64_t jb_tile) {
+    typename Fast16Shared<BM, BV>::Stage& st = s.stage[fill & 1u];
     const uint32_t bar = smem_u32(&s.mbar[fill & 1u]);
     const uint32_t bytes_s = (16u + ((jb_tile & 3) ? 4u : 0u)) * 4u;
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar),
-                 "r"((uint32_t)(TILE * 4 + TILE * 2 + 512 + 768) + 3u * bytes_s) : "memory");
+                 "r"((uint32_t)(TILE * 4 + TILE * 2 + 256 * BM + 256 * BV) + 3u * bytes_s) : "memory");
     bulk_copy(st.p, pt, TILE * 4, bar);
     bulk_copy(st.g, gt, TILE * 2, bar);
-    bulk_copy(st.cm, a.codes_m + jb_tile * 32, 512, bar);
-    bulk_copy(st.cv, a.codes_v + jb_tile * 48, 768, bar);
+    bulk_copy(st.cm, a.codes_m + jb_tile * (16 * BM), 256 * BM, bar);
+    bulk_copy(st.cv, a.codes_v + jb_tile * (16 * BV), 256 * BV, bar);
     const int64_t j0 = jb_tile & ~(int64_t)3;
     bulk_copy(st.sc[0], a.scale_m + j0, bytes_s, bar);
     bulk_copy(st.sc[1], a.scale_v + j0, bytes_s, bar);
@@ -113,11 +159,12 @@ __device__ __forceinline__ void issue_tile_copy16(const StepArgs& a, Fast16Share
 }
 
 // One full tile.  Arguments as for fast_tile.
-__device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared& s, const float* s_y, const float* s_mid,
+template <int BM, int BV>
+__device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, BV>& s, const float* s_y, const float* s_mid,
                                             char* pbase, const char* gbase, const int tin, const int64_t jb_tile,
                                             const int tensor, const int par, Ahead& ah, const bool next_full,
                                             const int next_dtin) {
-    constexpr int BV = 3, KV = 8, G = 8, NG = 16;                 // 2-bit m, 3-bit v, 8 lanes per block, 16 blocks per tile
+    constexpr int KM = 1 << BM, KV = 1 << BV, G = 8, NG = 16;     // 8 lanes per block, 16 blocks per tile
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gl = tid & (G - 1), grp = tid >> 3;
     const bool hi = (lane & G) != 0;                              // odd group of its pair
@@ -129,9 +176,9 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared& s, 
 
     // ---- inputs from the stage (see fast_tile for the protocol) ----
     if (tid == 0) {
-        if (!ah.staged) issue_tile_copy16(a, s, ah.fill, pt, gt, jb_tile);
+        if (!ah.staged) issue_tile_copy16<BM, BV>(a, s, ah.fill, pt, gt, jb_tile);
         if (next_full)
-            issue_tile_copy16(a, s, ah.fill + 1u, pt + (int64_t)next_dtin * (TILE * 4),
+            issue_tile_copy16<BM, BV>(a, s, ah.fill + 1u, pt + (int64_t)next_dtin * (TILE * 4),
                               gt + (int64_t)next_dtin * (TILE * 2), jb_tile + (int64_t)next_dtin * NG);
     }
     const uint32_t mine = ah.fill;
@@ -141,7 +188,7 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared& s, 
         atomicOr(a.status, 2);
         ah.failed = true;
     }
-    const Fast16Shared::Stage& st = s.stage[mine & 1u];
+    const typename Fast16Shared<BM, BV>::Stage& st = s.stage[mine & 1u];
     float p[EPT16], g[EPT16];
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
@@ -158,25 +205,24 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared& s, 
         const float4 pv = st.p[4 * tid + h];
         p[4 * h] = pv.x; p[4 * h + 1] = pv.y; p[4 * h + 2] = pv.z; p[4 * h + 3] = pv.w;
     }
-    const uint32_t cm = st.cm[tid];
-    // the thread's 48 bits of 3-bit codes start at byte 6 * tid
-    const int cw = (6 * tid) >> 2, cs = ((6 * tid) & 3) * 8;      // cs is 0 or 16
-    const uint32_t w0 = st.cv[cw], w1 = st.cv[cw + 1];
-    const uint32_t c32 = __funnelshift_r(w0, w1, cs);             // codes 0..9 and two bits of code 10
-    const uint32_t c16 = (w1 >> cs) & 0xFFFFu;                    // bits 32..47
-    const uint32_t cv_lo = c32 & 0xFFFFFFu, cv_hi = (c32 >> 24) | (c16 << 8);
+    uint32_t cm[2], cv[2];                                        // eight codes per word
+    load_codes16<BM>(st.cm, tid, cm);
+    load_codes16<BV>(st.cv, tid, cv);
     const int so = (int)(jb_tile & 3) + grp;
     const float dm = st.sc[0][so], dv = st.sc[1][so], al = st.sc[2][so];
 
-    // ---- per-block level tables (Eq. 2): one entry per lane ----
+    // ---- per-block level tables (Eq. 2), built by the block's eight lanes ----
     float* const tab = s.tab[grp];
     {
         float a2[BV];
         a2[0] = al;
 #pragma unroll
         for (int i = 1; i < BV; ++i) a2[i] = a2[i - 1] * a2[i - 1];
-        tab[gl] = pow_sm<BV>(a2, (uint32_t)gl) * dv;
-        if (gl < 4) tab[KV + gl] = s_y[gl] * dm;
+#pragma unroll
+        for (int r0 = 0; r0 < KV; r0 += G) tab[r0 + gl] = pow_sm<BV>(a2, (uint32_t)(r0 + gl)) * dv;
+#pragma unroll
+        for (int r0 = 0; r0 < KM; r0 += G)
+            if (r0 + gl < KM) tab[KV + r0 + gl] = s_y[r0 + gl] * dm;
     }
     __syncwarp();
 
@@ -186,11 +232,12 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared& s, 
     float mx_m_f = 0.0f;
     const char* const tab_v = reinterpret_cast<const char*>(tab);
     const char* const tab_m = reinterpret_cast<const char*>(tab + KV);
-    const CodeOffsets16x2 om4(cm);
-    const CodeOffsets<BV> ov4a(cv_lo, 0u), ov4b(cv_hi, 0u);
+    const CodeOffsets16x2 om16(cm[0] | (cm[1] << 16));            // used for 2-bit codes only
+    const CodeOffsets<BM> om4a(cm[0], 0u), om4b(cm[1], 0u);
+    const CodeOffsets<BV> ov4a(cv[0], 0u), ov4b(cv[1], 0u);
 #pragma unroll
     for (int i = 0; i < EPT16; ++i) {
-        const float mt = *reinterpret_cast<const float*>(tab_m + om4(i));
+        const float mt = *reinterpret_cast<const float*>(tab_m + (BM == 2 ? om16(i) : i < 8 ? om4a(i) : om4b(i - 8)));
         const float vt = *reinterpret_cast<const float*>(tab_v + (i < 8 ? ov4a(i) : ov4b(i - 8)));
         const float gi = g[i];
         mh[i] = __fmaf_rn(a.beta1, mt, a.omb1 * gi);
@@ -279,21 +326,34 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared& s, 
     const uint32_t zf = s.xflag[par][grp];
 
     // ---- first moment: nearest level (Eq. 1), see fast_tile ----
-    uint32_t om;
+    uint32_t om[2] = {0u, 0u};                                    // eight codes per word
     {
         const float inv = sc.x;
-        constexpr float BIG = 0x1p100f;
-        const float n0 = -s_mid[0] * BIG, n1 = -s_mid[1] * BIG, n2 = -s_mid[2] * BIG;
-        float omf[2] = {0.0f, 0.0f};
+        if constexpr (BM == 2) {
+            constexpr float BIG = 0x1p100f;
+            const float n0 = -s_mid[0] * BIG, n1 = -s_mid[1] * BIG, n2 = -s_mid[2] * BIG;
+            float omf[2] = {0.0f, 0.0f};
 #pragma unroll
-        for (int i = EPT16 - 1; i >= 0; --i) {
-            const float r = mh[i] * inv;
-            float& acc = omf[i >> 3];
-            acc = __fmaf_rn(acc, 4.0f, __saturatef(__fmaf_rn(r, BIG, n0)));
-            acc += __saturatef(__fmaf_rn(r, BIG, n1));
-            acc += __saturatef(__fmaf_rn(r, BIG, n2));
+            for (int i = EPT16 - 1; i >= 0; --i) {
+                const float r = mh[i] * inv;
+                float& acc = omf[i >> 3];
+                acc = __fmaf_rn(acc, 4.0f, __saturatef(__fmaf_rn(r, BIG, n0)));
+                acc += __saturatef(__fmaf_rn(r, BIG, n1));
+                acc += __saturatef(__fmaf_rn(r, BIG, n2));
+            }
+            om[0] = (uint32_t)omf[0];
+            om[1] = (uint32_t)omf[1];
+        } else {
+#pragma unroll
+            for (int i = EPT16 - 1; i >= 0; --i) {
+                const float r = mh[i] * inv;
+                uint32_t q = 0;
+#pragma unroll
+                for (int st = KM / 2; st >= 1; st >>= 1)
+                    if (r > s_mid[q + st - 1]) q += st;
+                om[i >> 3] = (om[i >> 3] << BM) + q;
+            }
         }
-        om = (uint32_t)omf[0] | ((uint32_t)omf[1] << 16);
     }
 
     // ---- second moment: Eq. 6, see fast_tile ----
@@ -340,34 +400,25 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared& s, 
             }
         }
     }
-    if (zf & 1u) om = 0;
+    if (zf & 1u) { om[0] = 0; om[1] = 0; }
     if (zf & 2u) { ov[0] = 0; ov[1] = 0; }
 
-    // ---- store the codes: 2-bit codes one word per thread; 3-bit codes (48 bits per thread)
-    // through shared memory so that twelve lanes store the warp's 192 bytes as 128-bit words ----
-    __stcs(reinterpret_cast<uint32_t*>(a.codes_m + jb_tile * 32) + tid, om);
-    {
-        unsigned short* const half = reinterpret_cast<unsigned short*>(s.cout[warp]) + 3 * lane;
-        half[0] = (unsigned short)ov[0];
-        half[1] = (unsigned short)((ov[0] >> 16) | (ov[1] << 8));
-        half[2] = (unsigned short)(ov[1] >> 8);
-        __syncwarp();
-        if (lane < 12)
-            __stcs(reinterpret_cast<uint4*>(a.codes_v + jb_tile * 48 + warp * 192) + lane,
-                   reinterpret_cast<const uint4*>(s.cout[warp])[lane]);
-        __syncwarp();
-    }
+    // ---- store the codes ----
+    store_codes16<BM>(a.codes_m + jb_tile * (16 * BM), s.cout[0][warp], tid, om);
+    store_codes16<BV>(a.codes_v + jb_tile * (16 * BV), s.cout[BM == 3 ? 1 : 0][warp], tid, ov);
 }
 
+template <int BM, int BV>
 __global__ void __launch_bounds__(CTA16, 6) solo_step_fast16_kernel(const StepArgs a) {
+    constexpr int KM = 1 << BM;
     extern __shared__ __align__(16) unsigned char fast16_smem[];
-    Fast16Shared& s = *reinterpret_cast<Fast16Shared*>(fast16_smem);
-    __shared__ float s_y[4];
-    __shared__ float s_mid[4];
+    Fast16Shared<BM, BV>& s = *reinterpret_cast<Fast16Shared<BM, BV>*>(fast16_smem);
+    __shared__ float s_y[KM];
+    __shared__ float s_mid[KM];
     const int tid = threadIdx.x;
-    if (tid < 4) {
+    if (tid < KM) {
         s_y[tid] = a.tables[tid];
-        if (tid < 3) s_mid[tid] = a.tables[4 + tid];
+        if (tid < KM - 1) s_mid[tid] = a.tables[KM + tid];
     }
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s.mbar[0])) : "memory");
@@ -403,7 +454,7 @@ __global__ void __launch_bounds__(CTA16, 6) solo_step_fast16_kernel(const StepAr
         }
         const int tin = tile - t_lo;
         if (skip || tin >= full_tiles) continue;
-        fast16_tile(a, s, s_y, s_mid, pbase, gbase, tin, jb0 + (int64_t)tin * 16, tensor, par, ah,
+        fast16_tile<BM, BV>(a, s, s_y, s_mid, pbase, gbase, tin, jb0 + (int64_t)tin * 16, tensor, par, ah,
                     tin + stride < full_tiles && tile + stride < total_tiles, stride);
         par ^= 1;
     }

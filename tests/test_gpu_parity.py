@@ -80,8 +80,11 @@ def test_bits_and_blocks_random_state(bits_m, bits_v, block):
     params, gf = _inputs(w)
     st0 = synth.make_state(sizes, bits_m, bits_v, block, seed=bits_m * 100 + bits_v * 10 + block)
     hk = dict(lr=1e-3, beta1=0.8, beta2=0.999, weight_decay=0.01, seed=5)
-    rep = run_lockstep(sizes, bits_m, bits_v, block, hk, 2, gf, params, state0=st0)
-    assert rep.exempt_m + rep.exempt_v <= 3
+    # block 128 with a 2-bit first moment: policy 3 is the sixteen-per-thread kernel plus the
+    # streamlined kernel for the tails (policy 0 picks it for large tensors only)
+    policies = (0, 3, 1) if block == 128 and bits_m == 2 and bits_v <= 4 else (0, 1)
+    rep = run_lockstep(sizes, bits_m, bits_v, block, hk, 2, gf, params, state0=st0, policies=policies)
+    assert rep.exempt_m + rep.exempt_v <= 3 * len(policies)
 
 
 @pytest.mark.parametrize("bits_m,bits_v,block", [(2, 3, 128), (3, 2, 64), (4, 4, 256), (2, 2, 2048), (8, 4, 64),
@@ -186,21 +189,22 @@ def test_stochastic_bf16_rounding_is_unbiased_on_the_device():
         st.destroy()
 
 
-def test_default_configuration_all_three_kernels():
-    """2-bit / 3-bit, block 128, plain step: the sixteen-per-thread kernel (policy 0: full tiles
-    there, the rest in the streamlined kernel), the streamlined kernel alone (2) and the general
-    kernel (1) against one oracle run; tensors with many full tiles, tails and tiny tensors, zero
-    blocks, ties, from a random state and from zero."""
+@pytest.mark.parametrize("bits_m,bits_v", [(2, 3), (2, 2), (2, 4)])
+def test_block_128_plain_step_all_three_kernels(bits_m, bits_v):
+    """Block 128, plain step: the sixteen-per-thread kernel (policy 3: full tiles there, the rest in
+    the streamlined kernel), the streamlined kernel alone (2) and the general kernel (1) against
+    one oracle run; tensors with many full tiles, tails and tiny tensors, zero blocks, ties, from a
+    random state and from zero."""
     sizes = (2048 * 9 + 700, 3, 2048 * 4, 2048 + 128, 127, 2048 * 2 + 1)
     w = synth.workload(4, sizes=sizes)
     params, gf = _inputs(w)
     hk = dict(lr=2e-5, beta1=0.5, beta2=0.999, weight_decay=0.0, seed=1234)
-    st0 = synth.make_state(sizes, 2, 3, 128, seed=5)
-    run_lockstep(sizes, 2, 3, 128, hk, 3, gf, params, state0=st0, policies=(0, 2, 1))
-    run_lockstep(sizes, 2, 3, 128, hk, 4, gf, params, policies=(0, 2, 1))
+    st0 = synth.make_state(sizes, bits_m, bits_v, 128, seed=5)
+    run_lockstep(sizes, bits_m, bits_v, 128, hk, 3, gf, params, state0=st0, policies=(3, 2, 1))
+    run_lockstep(sizes, bits_m, bits_v, 128, hk, 4, gf, params, policies=(3, 2, 1))
     w1 = synth.workload(1, sizes=(2048 * 6,))
     p1, g1 = _inputs(w1)
-    run_lockstep(w1.sizes, 2, 3, 128, hk, 3, g1, p1, policies=(0, 2), multi=False)   # one launch: all tiles full
+    run_lockstep(w1.sizes, bits_m, bits_v, 128, hk, 3, g1, p1, policies=(3, 2), multi=False)   # one launch: all tiles full
 
 
 def test_streamlined_kernel_rounding_guard_is_sound():
