@@ -220,7 +220,7 @@ int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
     const bool cta_group = s->block == 2048;
     const int policy = g_policy.load(std::memory_order_relaxed);
     const bool streamlined = policy != 1 && !a.round_m && !a.tables_v && a.eps >= 1e-12f &&
-                             s->tiles_total < (int64_t)1 << 31;
+                             s->tiles_total < ((int64_t)1 << 31) - ((int64_t)1 << 20);   // 32-bit tile arithmetic with headroom
     const bool plain = !a.l2 && !a.belief && a.fixed_alpha == 0.0f && a.round_v;
     solo::StepKernel k16 = nullptr;
     // worth its second launch and its 128-thread CTAs on large tensors only: measured faster on the

@@ -943,25 +943,34 @@ __global__ void __launch_bounds__(CTA, (BM == 8 || BV == 8) ? 3 : 4) solo_step_f
     }
     __syncthreads();
 
-    // Tile indices fit 32 bits (the host selects this kernel only below 2^31 tiles).  Tiles are
-    // visited in increasing order, so the tensor of a tile is found by walking forward.
-    const int total_tiles = (int)a.total_tiles, stride = (int)gridDim.x;
-    int tensor = a.tensor_first - 1;
+    // Tile indices fit 32 bits (the host selects this kernel only below 2^31 - 2^20 tiles).  With
+    // sub-CTA blocks a CTA takes a contiguous share of the launch's tiles, so that its next tile is
+    // nearly always the next tile of the same tensor and can be copied ahead even in sets of small
+    // tensors (with tiles dealt out in turn it rarely was; measured +7 % on the GPT-125M set, +16 %
+    // on the ragged set, +2 % on the 7B set).  Blocks of 2048 measured 7 % slower that way and keep
+    // tiles dealt in turn.  Tiles are visited in increasing order, so the tensor of a tile is found by
+    // a search for the CTA's first tile and by walking forward after that.
+    const int launch_tiles = (int)(a.total_tiles - a.tile_first);
+    const int share = (launch_tiles + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int step = G == CTA ? (int)gridDim.x : 1;            // to the CTA's next tile
+    const int tile_begin = (int)min(a.tile_first + (int64_t)blockIdx.x * (G == CTA ? 1 : share), a.total_tiles);
+    const int tile_end = G == CTA ? (int)a.total_tiles : (int)min((int64_t)tile_begin + share, a.total_tiles);
+    int tensor = (a.num_tensors > 1 && tile_begin < tile_end ? find_tensor(a.tile_start, a.num_tensors, tile_begin) : 0) - 1;
     int t_lo = 0, t_hi = 0, full_tiles = 0;      // the tensor's tiles [t_lo, t_hi); its first full_tiles are full
-    int64_t n = 0, jb0 = 0;
+    int64_t jb0 = 0;
     char* pbase = nullptr;
     const char* gbase = nullptr;
     bool skip = false;
     Ahead ah;
     int par = 0;
-    for (int tile = (int)a.tile_first + blockIdx.x; tile < total_tiles; tile += stride) {
+    for (int tile = tile_begin; tile < tile_end; tile += step) {
         if (tile >= t_hi) {
             do {
                 ++tensor;
                 t_hi = (int)__ldg(a.tile_start + tensor + 1);
             } while (tile >= t_hi);
             t_lo = (int)__ldg(a.tile_start + tensor);
-            n = __ldg(a.numel + tensor);
+            const int64_t n = __ldg(a.numel + tensor);
             jb0 = __ldg(a.block_start + tensor);
             pbase = (char*)(a.param_list ? a.param_list[tensor] : a.param_single);
             gbase = (const char*)(a.grad_list ? a.grad_list[tensor] : a.grad_single);
@@ -975,10 +984,11 @@ __global__ void __launch_bounds__(CTA, (BM == 8 || BV == 8) ? 3 : 4) solo_step_f
         if (a.only_partial && tin < full_tiles) continue;
         const int64_t jb_tile = jb0 + (int64_t)tin * (CTA / G);
         if (tin < full_tiles)
-            fast_tile<BM, BV, G, true, PBF, PLAIN>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, ah,
-                                       tin + stride < full_tiles && tile + stride < total_tiles, stride);
+            fast_tile<BM, BV, G, true, PBF, PLAIN>(a, s, s_y, s_mid, pbase, gbase, 0, tin, jb_tile, tensor, par, ah,
+                                       tin + step < full_tiles && tile + step < tile_end, step);
         else
-            fast_tile<BM, BV, G, false, PBF, PLAIN>(a, s, s_y, s_mid, pbase, gbase, n, tin, jb_tile, tensor, par, ah, false, 0);
+            fast_tile<BM, BV, G, false, PBF, PLAIN>(a, s, s_y, s_mid, pbase, gbase, __ldg(a.numel + tensor), tin, jb_tile,
+                                                    tensor, par, ah, false, 0);
         par ^= 1;
     }
     // every copy that was issued has been waited for by the thread that issued it, unless that
