@@ -223,9 +223,9 @@ int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
                              s->tiles_total < ((int64_t)1 << 31) - ((int64_t)1 << 20);   // 32-bit tile arithmetic with headroom
     const bool plain = !a.l2 && !a.belief && a.fixed_alpha == 0.0f && a.round_v;
     solo::StepKernel k16 = nullptr;
-    // worth its second launch and its 128-thread CTAs on large tensors only: measured faster on the
-    // 7B-shaped set and on one 268M-element tensor, slower on sets of small tensors
-    const bool large = s->tiles_total >= (int64_t)4096 * s->num_tensors;
+    // worth its second launch only when there is work for many tiles per CTA (measured faster on the
+    // 7B-shaped, the GPT-125M-shaped and the ragged set; a 1 Mi-element tensor is launch-bound)
+    const bool large = s->tiles_total >= 8192;
     if (streamlined && ((policy == 0 && large) || policy == 3) && s->block == 128 && !a.param_bf16 && plain &&
         a.k_full == 13)
         k16 = solo::fast16_kernel(s->bits_m, s->bits_v);
@@ -575,7 +575,6 @@ int solo_multi_step_host(const solo_host_list_t* list, const solo_hyper_t* hyper
         a.grad_list = (const void* const*)hp->d_grad_list[slot];
         a.tile_first = first;
         a.total_tiles = last;
-        a.tensor_first = tensor_first;
         rc = launch_step(s, a, st);
         if (rc) break;
         if (list->param_out_host) {

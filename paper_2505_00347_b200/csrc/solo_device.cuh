@@ -40,7 +40,6 @@ struct StepArgs {
     int32_t num_tensors;
     int64_t total_tiles;               // the launch covers tiles [tile_first, total_tiles)
     int64_t tile_first;
-    int32_t tensor_first;              // tensor that holds tile_first
     int32_t only_partial;              // streamlined kernel: skip full tiles of aligned tensors (another launch did them)
     // state
     uint8_t* codes_m;

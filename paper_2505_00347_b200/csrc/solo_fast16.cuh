@@ -427,9 +427,13 @@ __global__ void __launch_bounds__(CTA16, 6) solo_step_fast16_kernel(const StepAr
     }
     __syncthreads();
 
-    // the tile walk of solo_step_fast_kernel; tiles that are not full are skipped here
-    const int total_tiles = (int)a.total_tiles, stride = (int)gridDim.x;
-    int tensor = a.tensor_first - 1;
+    // the tile walk of solo_step_fast_kernel (a contiguous share of the tiles per CTA); tiles that are
+    // not full are skipped here
+    const int launch_tiles = (int)(a.total_tiles - a.tile_first);
+    const int share = (launch_tiles + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int tile_begin = (int)min(a.tile_first + (int64_t)blockIdx.x * share, a.total_tiles);
+    const int tile_end = (int)min((int64_t)tile_begin + share, a.total_tiles);
+    int tensor = (a.num_tensors > 1 && tile_begin < tile_end ? find_tensor(a.tile_start, a.num_tensors, tile_begin) : 0) - 1;
     int t_lo = 0, t_hi = 0, full_tiles = 0;
     int64_t jb0 = 0;
     char* pbase = nullptr;
@@ -437,7 +441,7 @@ __global__ void __launch_bounds__(CTA16, 6) solo_step_fast16_kernel(const StepAr
     bool skip = false;
     Ahead ah;
     int par = 0;
-    for (int tile = (int)a.tile_first + blockIdx.x; tile < total_tiles; tile += stride) {
+    for (int tile = tile_begin; tile < tile_end; ++tile) {
         if (tile >= t_hi) {
             do {
                 ++tensor;
@@ -455,7 +459,7 @@ __global__ void __launch_bounds__(CTA16, 6) solo_step_fast16_kernel(const StepAr
         const int tin = tile - t_lo;
         if (skip || tin >= full_tiles) continue;
         fast16_tile<BM, BV>(a, s, s_y, s_mid, pbase, gbase, tin, jb0 + (int64_t)tin * 16, tensor, par, ah,
-                    tin + stride < full_tiles && tile + stride < total_tiles, stride);
+                    tin + 1 < full_tiles && tile + 1 < tile_end, 1);
         par ^= 1;
     }
     if (tid == 0 && ah.failed && ah.fill > 0) {
