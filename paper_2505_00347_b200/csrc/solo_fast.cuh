@@ -981,7 +981,10 @@ __global__ void __launch_bounds__(CTA, (BM == 8 || BV == 8) ? 3 : 4) solo_step_f
         }
         if (skip) continue;
         const int tin = tile - t_lo;
-        if (a.only_partial && tin < full_tiles) continue;
+        if (a.only_partial && tin < full_tiles) {                 // another launch did the full tiles
+            if (step == 1) tile = t_lo + full_tiles - 1;          // on to the tensor's first tile that is not full
+            continue;
+        }
         const int64_t jb_tile = jb0 + (int64_t)tin * (CTA / G);
         if (tin < full_tiles)
             fast_tile<BM, BV, G, true, PBF, PLAIN>(a, s, s_y, s_mid, pbase, gbase, 0, tin, jb_tile, tensor, par, ah,
