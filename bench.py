@@ -239,7 +239,7 @@ def run_ours(args, rank, world):
         "config": {"workload": f"{w.name}: {len(w.sizes)} tensors, {n} params, m {w.bits_m}-bit / v {w.bits_v}-bit, "
                                f"block {w.block}, {'bf16' if args.param_bf16 else 'fp32'} params"
                                f"{' (stochastic rounding)' if args.param_bf16 == 2 else ''}, bf16 grads, "
-                               "one solo_multi_step launch per step"
+                               "one solo_multi_step call per step"
                                + (f", fixed base {args.fixed_alpha}" if args.fixed_alpha else "")
                                + (f", baseline v codebook {args.v_codebook}" if args.v_codebook else ""),
                    "l2": "working set (params+grads+state) far larger than the 126 MB L2; no flush needed"
