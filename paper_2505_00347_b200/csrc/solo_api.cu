@@ -226,9 +226,8 @@ int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
     // worth its second launch only when there is work for many tiles per CTA (measured faster on the
     // 7B-shaped, the GPT-125M-shaped and the ragged set; a 1 Mi-element tensor is launch-bound)
     const bool large = s->tiles_total >= 8192;
-    if (streamlined && ((policy == 0 && large) || policy == 3) && s->block == 128 && !a.param_bf16 && plain &&
-        a.k_full == 13)
-        k16 = solo::fast16_kernel(s->bits_m, s->bits_v);
+    if (streamlined && ((policy == 0 && large) || policy == 3) && s->block == 128 && plain && a.k_full == 13)
+        k16 = solo::fast16_kernel(s->bits_m, s->bits_v, a.param_bf16 != 0);
     if (k16) {
         // blocks of 128, plain step: full tiles by the sixteen-per-thread kernel, whatever it leaves
         // (tails, tensors that are not 16-byte aligned) by the streamlined kernel

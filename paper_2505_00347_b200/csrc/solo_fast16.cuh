@@ -1,6 +1,6 @@
 // Sixteen elements per thread: the streamlined step for the paper's default block size and
 // plain step (2/3/4-bit states, of which 2-bit first moments are instantiated; blocks of 128,
-// fp32 parameters; no L2 term in the gradient, no AdaBelief, base from the p = 0.1 quantile, xi
+// fp32 or bf16 parameters; no L2 term in the gradient, no AdaBelief, base from the p = 0.1 quantile, xi
 // drawn).
 //
 // Same arithmetic, element for element, as solo_step_fast_kernel (solo_fast.cuh); what changes
@@ -35,7 +35,7 @@ struct Fast16Shared {
     static constexpr int N3 = (BM == 3 ? 1 : 0) + (BV == 3 ? 1 : 0);
     alignas(16) uint32_t cout[N3 > 0 ? N3 : 1][4][48];
     struct Stage {
-        float4 p[TILE / 4];              // 2048 parameters
+        float4 p[TILE / 4];              // 2048 parameters (bf16: the first half)
         uint4 g[TILE / 8];               // 2048 bf16 gradients
         uint32_t cm[64 * BM + 4];        // packed codes of the tile: 256 * bits bytes
         uint32_t cv[64 * BV + 4];
@@ -140,15 +140,15 @@ __device__ __forceinline__ uint32_t pop_round16(uint32_t& head, int& off, const 
 // Bulk copies of one full tile's inputs into stage `fill & 1` (one thread).  With blocks of 128
 // the tile's codes start on 16-byte boundaries (16 * bits bytes per block); the per-block scalars
 // are copied from the boundary at or below the first.
-template <int BM, int BV>
+template <int BM, int BV, bool PBF>
 __device__ __forceinline__ void issue_tile_copy16(const StepArgs& a, Fast16Shared<BM, BV>& s, uint32_t fill,
                                                   const char* pt, const char* gt, int64_t jb_tile) {
     typename Fast16Shared<BM, BV>::Stage& st = s.stage[fill & 1u];
     const uint32_t bar = smem_u32(&s.mbar[fill & 1u]);
     const uint32_t bytes_s = (16u + ((jb_tile & 3) ? 4u : 0u)) * 4u;
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar),
-                 "r"((uint32_t)(TILE * 4 + TILE * 2 + 256 * BM + 256 * BV) + 3u * bytes_s) : "memory");
-    bulk_copy(st.p, pt, TILE * 4, bar);
+                 "r"((uint32_t)(TILE * (PBF ? 2 : 4) + TILE * 2 + 256 * BM + 256 * BV) + 3u * bytes_s) : "memory");
+    bulk_copy(st.p, pt, TILE * (PBF ? 2 : 4), bar);
     bulk_copy(st.g, gt, TILE * 2, bar);
     bulk_copy(st.cm, a.codes_m + jb_tile * (16 * BM), 256 * BM, bar);
     bulk_copy(st.cv, a.codes_v + jb_tile * (16 * BV), 256 * BV, bar);
@@ -159,7 +159,7 @@ __device__ __forceinline__ void issue_tile_copy16(const StepArgs& a, Fast16Share
 }
 
 // One full tile.  Arguments as for fast_tile.
-template <int BM, int BV>
+template <int BM, int BV, bool PBF>
 __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, BV>& s, const float* s_y, const float* s_mid,
                                             char* pbase, const char* gbase, const int tin, const int64_t jb_tile,
                                             const int tensor, const int par, Ahead& ah, const bool next_full,
@@ -171,14 +171,15 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     const uint32_t vflip = hi ? 0xFFFFFFFFu : 0u;                 // x domain <-> v domain
 
     const int64_t tile_elem0 = (int64_t)tin * TILE;
-    char* const pt = pbase + tile_elem0 * 4;
+    constexpr int PSZ = PBF ? 2 : 4;                              // bytes per parameter
+    char* const pt = pbase + tile_elem0 * PSZ;
     const char* const gt = gbase + tile_elem0 * 2;
 
     // ---- inputs from the stage (see fast_tile for the protocol) ----
     if (tid == 0) {
-        if (!ah.staged) issue_tile_copy16<BM, BV>(a, s, ah.fill, pt, gt, jb_tile);
+        if (!ah.staged) issue_tile_copy16<BM, BV, PBF>(a, s, ah.fill, pt, gt, jb_tile);
         if (next_full)
-            issue_tile_copy16<BM, BV>(a, s, ah.fill + 1u, pt + (int64_t)next_dtin * (TILE * 4),
+            issue_tile_copy16<BM, BV, PBF>(a, s, ah.fill + 1u, pt + (int64_t)next_dtin * (TILE * PSZ),
                               gt + (int64_t)next_dtin * (TILE * 2), jb_tile + (int64_t)next_dtin * NG);
     }
     const uint32_t mine = ah.fill;
@@ -200,10 +201,23 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
             g[8 * h + 2 * i + 1] = __uint_as_float(gg[i] & 0xffff0000u);
         }
     }
+    if constexpr (PBF) {
 #pragma unroll
-    for (int h = 0; h < 4; ++h) {
-        const float4 pv = st.p[4 * tid + h];
-        p[4 * h] = pv.x; p[4 * h + 1] = pv.y; p[4 * h + 2] = pv.z; p[4 * h + 3] = pv.w;
+        for (int h = 0; h < 2; ++h) {
+            const uint4 pw = reinterpret_cast<const uint4*>(st.p)[2 * tid + h];
+            const uint32_t pp[4] = {pw.x, pw.y, pw.z, pw.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                p[8 * h + 2 * i] = __uint_as_float(pp[i] << 16);
+                p[8 * h + 2 * i + 1] = __uint_as_float(pp[i] & 0xffff0000u);
+            }
+        }
+    } else {
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+            const float4 pv = st.p[4 * tid + h];
+            p[4 * h] = pv.x; p[4 * h + 1] = pv.y; p[4 * h + 2] = pv.z; p[4 * h + 3] = pv.w;
+        }
     }
     uint32_t cm[2], cv[2];                                        // eight codes per word
     load_codes16<BM>(st.cm, tid, cm);
@@ -247,8 +261,35 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     }
     uint32_t mx_m = __float_as_uint(mx_m_f);
 
-    // Adam(W) update of element i, stored after every fourth
+    // Adam(W) update of element i; fp32 parameters are stored after every fourth.  bf16 parameters:
+    // IEEE square root and division (see solo_fast.cuh), stored after every eighth, rounded to
+    // nearest even or with the element's Philox draw (purpose 2, one block per eight elements)
+    const uint64_t ctr = ((uint64_t)(uint32_t)tin * (TILE / 8)) + 2u * (uint32_t)tid;   // element index / 8
     auto update = [&](int i) {
+        if constexpr (PBF) {
+            const float den = __fmaf_rn(__fsqrt_rn(vh[i]), a.inv_sqrt_bc2, a.eps);
+            p[i] = __fmaf_rn(-a.step_size, __fdiv_rn(mh[i], den), p[i] * a.decay);
+            if ((i & 7) == 7) {
+                const int b = i - 7;
+                uint32_t pp[4];
+                if (a.param_sr) {
+                    uint32_t wp[4];
+                    const uint64_t c = ctr + (uint64_t)(i >> 3);
+                    philox_rk((uint32_t)c, (uint32_t)(c >> 32), a.step32, (uint32_t)tensor * 4u + 2u, a.rk, wp);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        pp[j] = bf16_sr(p[b + 2 * j], wp[j] & 0xFFFFu) | (bf16_sr(p[b + 2 * j + 1], wp[j] >> 16) << 16);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const __nv_bfloat162 h2 = __floats2bfloat162_rn(p[b + 2 * j], p[b + 2 * j + 1]);
+                        pp[j] = *reinterpret_cast<const uint32_t*>(&h2);
+                    }
+                }
+                __stcs(reinterpret_cast<uint4*>(pt) + 2 * tid + (i >> 3), make_uint4(pp[0], pp[1], pp[2], pp[3]));
+            }
+            return;
+        }
         const float den = __fmaf_rn(sqrt_approx(vh[i]), a.inv_sqrt_bc2, a.eps);
         const float rc = rcp_approx(den);
         const float q0 = mh[i] * rc;
@@ -289,7 +330,6 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     if (gl == 0) s.xin[par][grp] = make_uint4(mx_m, mx_v, x_p, 0u);
     bar_sync16(1);
     uint32_t w[8];
-    const uint64_t ctr = ((uint64_t)(uint32_t)tin * (TILE / 8)) + 2u * (uint32_t)tid;   // element index / 8
     auto draw = [&]() {
         uint32_t wa[4], wb[4];
         philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, (uint32_t)tensor * 4u, a.rk, wa);
@@ -408,8 +448,8 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     store_codes16<BV>(a.codes_v + jb_tile * (16 * BV), s.cout[BM == 3 ? 1 : 0][warp], tid, ov);
 }
 
-template <int BM, int BV>
-__global__ void __launch_bounds__(CTA16, 6) solo_step_fast16_kernel(const StepArgs a) {
+template <int BM, int BV, bool PBF>
+__global__ void __launch_bounds__(CTA16, PBF ? 5 : 6) solo_step_fast16_kernel(const StepArgs a) {
     constexpr int KM = 1 << BM;
     extern __shared__ __align__(16) unsigned char fast16_smem[];
     Fast16Shared<BM, BV>& s = *reinterpret_cast<Fast16Shared<BM, BV>*>(fast16_smem);
@@ -458,7 +498,7 @@ __global__ void __launch_bounds__(CTA16, 6) solo_step_fast16_kernel(const StepAr
         }
         const int tin = tile - t_lo;
         if (skip || tin >= full_tiles) continue;
-        fast16_tile<BM, BV>(a, s, s_y, s_mid, pbase, gbase, tin, jb0 + (int64_t)tin * 16, tensor, par, ah,
+        fast16_tile<BM, BV, PBF>(a, s, s_y, s_mid, pbase, gbase, tin, jb0 + (int64_t)tin * 16, tensor, par, ah,
                     tin + 1 < full_tiles && tile + 1 < tile_end, 1);
         par ^= 1;
     }
