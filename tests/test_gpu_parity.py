@@ -286,12 +286,16 @@ def test_nan_and_inf_gradients_do_not_hang():
     (8, 3, 2048, dict(round_m=1), 2048 * 2),
     (3, 3, 256, dict(v_codebook=2), 2048 * 5),
     (2, 3, 128, dict(), 0),
+    (2, 3, 128, dict(policy=3), 2048 * 3),
+    (2, 4, 128, dict(policy=3, param_dtype=1, param_round=1), 2048 * 2),
 ])
 def test_host_buffer_entry_point(bits_m, bits_v, block, extra, chunk):
     """solo_multi_step_host (gradients from host memory, parameters copied back, chunked over three
     streams) against solo_multi_step on the same inputs: identical state and parameters, chunk
     boundaries inside tensors, more chunks than staging slots, tiny tensors, two steps."""
     from paper_2505_00347_b200 import binding as B
+    extra = dict(extra)
+    policy = extra.pop("policy", 0)            # 3: the sixteen-per-thread kernel on the chunks' tile ranges
     sizes = (2048 * 7 + 300, 5, 2048 * 2, 129, 2048 * 4 + 1, 2047)
     w = synth.workload(2, sizes=sizes)
     dtype = torch.bfloat16 if extra.get("param_dtype") == 1 else torch.float32
@@ -306,8 +310,12 @@ def test_host_buffer_entry_point(bits_m, bits_v, block, extra, chunk):
         grads = [synth.make_grad(w, i, t) for i in range(len(sizes))]
         B.solo_multi_step(B.TensorSet(p_dev, [g.cuda() for g in grads], st_dev), h, t)
         pinned = [g.pin_memory() for g in grads]
-        B.solo_multi_step_host(p_hst, pinned, out if t == 2 else None, st_hst, h, t, chunk_elems=chunk)
-        torch.cuda.synchronize()
+        B.set_kernel_policy(policy)
+        try:
+            B.solo_multi_step_host(p_hst, pinned, out if t == 2 else None, st_hst, h, t, chunk_elems=chunk)
+            torch.cuda.synchronize()
+        finally:
+            B.set_kernel_policy(0)
         assert st_hst.status() == 0
         assert torch.equal(st_dev.export(), st_hst.export()), t
         for a, b in zip(p_dev, p_hst):
