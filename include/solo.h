@@ -235,7 +235,7 @@ int solo_state_import(solo_state_t* state, const void* host_src, size_t bytes, v
  * Reads the state's device status word into *status_out (0 = no problem seen).
  *   bit 0  a solo_multi_step descriptor's numel disagreed with the state; the affected
  *          tensors were skipped
- *   bit 1  the streamlined kernel gave up waiting for an asynchronous copy of its inputs
+ *   bit 1  a kernel that stages its inputs gave up waiting for an asynchronous copy of them
  *          (a bounded wait, so the kernel always ends); the results of that step are undefined
  * Synchronizes the device.
  */

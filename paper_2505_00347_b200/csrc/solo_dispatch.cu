@@ -54,25 +54,6 @@ int kernel_occupancy(StepKernel k, size_t dyn_smem, int threads) {
     return n;
 }
 
-int step_kernel_occupancy(int bits_m, int bits_v, bool cta_group) {
-    static std::mutex mu;
-    static int cache[4][4][2];
-    const int bm = bits_index(bits_m), bv = bits_index(bits_v);
-    if (bm < 0 || bv < 0) return 0;
-    std::lock_guard<std::mutex> lk(mu);
-    int& c = cache[bm][bv][cta_group ? 1 : 0];
-    if (c == 0) {
-        StepKernel k = step_kernel(bits_m, bits_v, cta_group);
-        int n = 0;
-        if (!k || cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k, CTA, 0) != cudaSuccess || n <= 0) {
-            cudaGetLastError();
-            return 0;
-        }
-        c = n;
-    }
-    return c;
-}
-
 cudaError_t launch_dequant(int bits, const DequantArgs& a, unsigned grid, cudaStream_t stream) {
     switch (bits) {
         case 2: solo_dequant_kernel<2><<<grid, CTA, 0, stream>>>(a); break;

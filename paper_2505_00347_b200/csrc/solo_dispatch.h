@@ -54,8 +54,6 @@ int kernel_occupancy(StepKernel k, size_t dyn_smem, int threads = CTA);
 // Exhaustive comparison of the hardware lg2 approximation with log2_sp (tests).
 cudaError_t launch_fast_log_check(uint32_t lo, uint32_t hi, float* out_max_excess, cudaStream_t stream);
 float fast_log_abs_bound();
-// Resident CTAs per SM of that kernel (cached), 0 on error.
-int step_kernel_occupancy(int bits_m, int bits_v, bool cta_group);
 
 cudaError_t launch_dequant(int bits, const DequantArgs& a, unsigned grid, cudaStream_t stream);
 
