@@ -38,8 +38,8 @@ StepKernel fast_kernel_bm3(int bv_index, int block, bool param_bf16, bool plain)
 StepKernel fast_kernel_bm4(int bv_index, int block, bool param_bf16, bool plain);
 StepKernel fast_kernel_bm8(int bv_index, int block, bool param_bf16, bool plain);
 StepKernel fast_kernel(int bits_m, int bits_v, int block, bool param_bf16, bool plain);
-// Sixteen elements per thread: 2-bit first moment, 2/3/4-bit second moment, block 128, fp32 or
-// bf16 parameters, the plain step with p-quantile rank 13; full tiles of aligned tensors only (the rest is left to a launch of the
+// Sixteen elements per thread: 2/3/4-bit states (not 4-bit / 4-bit), block 128, fp32 or bf16
+// parameters, the plain step with p-quantile rank 13; full tiles of aligned tensors only (the rest is left to a launch of the
 // streamlined kernel with StepArgs::only_partial).  Launched with CTA16 = 128 threads.  Null / 0
 // for other widths.
 constexpr int CTA16 = 128;         // threads per CTA of that kernel

@@ -1,6 +1,5 @@
 // Sixteen elements per thread: the streamlined step for the paper's default block size and
-// plain step (2/3/4-bit states, of which 2-bit first moments are instantiated; blocks of 128,
-// fp32 or bf16 parameters; no L2 term in the gradient, no AdaBelief, base from the p = 0.1 quantile, xi
+// plain step (2/3/4-bit states, blocks of 128, fp32 or bf16 parameters; no L2 term in the gradient, no AdaBelief, base from the p = 0.1 quantile, xi
 // drawn).
 //
 // Same arithmetic, element for element, as solo_step_fast_kernel (solo_fast.cuh); what changes
@@ -28,12 +27,15 @@ struct Fast16Shared {
     // Twelve rounds of popping read rows 0..11 at most.
     uint32_t sort[12][CTA16];
     float tab[16][(1 << BV) + (1 << BM)]; // per block: K_v second-moment levels, then K_m first-moment levels
-    uint4 xin[2][16];                    // per block: bits of Delta_m', Delta_v', x_p
-    float4 xout[2][16];                  // per block: 1/Delta_m', 1/Delta_v', 1/log2(alpha'), rounding limit
-    uint32_t xflag[2][16];
+    // Exchange with the first warp.  One copy is enough: xin is written before the tile's first
+    // barrier and read between its two barriers, xout and xflag are written between the barriers and
+    // read after the second, and nobody writes either again before passing those barriers.
+    uint4 xin[16];                       // per block: bits of Delta_m', Delta_v', x_p
+    float4 xout[16];                     // per block: 1/Delta_m', 1/Delta_v', 1/log2(alpha'), rounding limit
+    uint32_t xflag[16];
     // per 3-bit moment and warp: the packed codes of the warp's 512 elements, for 128-bit stores
     static constexpr int N3 = (BM == 3 ? 1 : 0) + (BV == 3 ? 1 : 0);
-    alignas(16) uint32_t cout[N3 > 0 ? N3 : 1][4][48];
+    alignas(16) uint32_t cout[N3 > 0 ? N3 : 1][N3 > 0 ? 4 : 1][N3 > 0 ? 48 : 4];   // (a token array without 3-bit codes)
     struct Stage {
         float4 p[TILE / 4];              // 2048 parameters (bf16: the first half)
         uint4 g[TILE / 8];               // 2048 bf16 gradients
@@ -162,7 +164,7 @@ __device__ __forceinline__ void issue_tile_copy16(const StepArgs& a, Fast16Share
 template <int BM, int BV, bool PBF>
 __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, BV>& s, const float* s_y, const float* s_mid,
                                             char* pbase, const char* gbase, const int tin, const int64_t jb_tile,
-                                            const int tensor, const int par, Ahead& ah, const bool next_full,
+                                            const int tensor, Ahead& ah, const bool next_full,
                                             const int next_dtin) {
     constexpr int KM = 1 << BM, KV = 1 << BV, G = 8, NG = 16;     // 8 lanes per block, 16 blocks per tile
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -327,7 +329,7 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     }
 
     // ---- per-block scalars by the first warp; the others draw xi meanwhile ----
-    if (gl == 0) s.xin[par][grp] = make_uint4(mx_m, mx_v, x_p, 0u);
+    if (gl == 0) s.xin[grp] = make_uint4(mx_m, mx_v, x_p, 0u);
     bar_sync16(1);
     uint32_t w[8];
     auto draw = [&]() {
@@ -340,7 +342,7 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     if (warp != 0) {
         draw();
     } else if (tid < NG) {
-        const uint4 in = s.xin[par][tid];
+        const uint4 in = s.xin[tid];
         const float dm_new = __uint_as_float(in.x), dv_new = __uint_as_float(in.y);
         const bool zero_m = dm_new < TINY, zero_v = dv_new < TINY;
         const float inv_dm = 1.0f / dm_new;
@@ -350,8 +352,8 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
         const float al_new = exp2_sp(lam);
         const float inv_lambda = 1.0f / log2_sp(al_new);
         const float guard = __fmaf_rn(fabsf(inv_lambda), LG2_ABS, LG2_REL * (float)(KV + 1));
-        s.xout[par][tid] = make_float4(inv_dm, inv_dv, inv_lambda, 0.5f - guard);
-        s.xflag[par][tid] = (zero_m ? 1u : 0u) | (zero_v ? 2u : 0u);
+        s.xout[tid] = make_float4(inv_dm, inv_dv, inv_lambda, 0.5f - guard);
+        s.xflag[tid] = (zero_m ? 1u : 0u) | (zero_v ? 2u : 0u);
         const int64_t j = jb_tile + tid;
         a.scale_m[j] = zero_m ? 0.0f : dm_new;
         a.scale_v[j] = zero_v ? 0.0f : dv_new;
@@ -362,8 +364,8 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     float dr[EPT16];
 #pragma unroll
     for (int i = 0; i < 8; ++i) halves_to_float(w[i], dr[2 * i], dr[2 * i + 1]);
-    const float4 sc = s.xout[par][grp];
-    const uint32_t zf = s.xflag[par][grp];
+    const float4 sc = s.xout[grp];
+    const uint32_t zf = s.xflag[grp];
 
     // ---- first moment: nearest level (Eq. 1), see fast_tile ----
     uint32_t om[2] = {0u, 0u};                                    // eight codes per word
@@ -444,8 +446,8 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     if (zf & 2u) { ov[0] = 0; ov[1] = 0; }
 
     // ---- store the codes ----
-    store_codes16<BM>(a.codes_m + jb_tile * (16 * BM), s.cout[0][warp], tid, om);
-    store_codes16<BV>(a.codes_v + jb_tile * (16 * BV), s.cout[BM == 3 ? 1 : 0][warp], tid, ov);
+    store_codes16<BM>(a.codes_m + jb_tile * (16 * BM), s.cout[0][BM == 3 ? warp : 0], tid, om);
+    store_codes16<BV>(a.codes_v + jb_tile * (16 * BV), s.cout[(BM == 3 && BV == 3) ? 1 : 0][BV == 3 ? warp : 0], tid, ov);
 }
 
 template <int BM, int BV, bool PBF>
@@ -480,7 +482,6 @@ __global__ void __launch_bounds__(CTA16, PBF ? 5 : 6) solo_step_fast16_kernel(co
     const char* gbase = nullptr;
     bool skip = false;
     Ahead ah;
-    int par = 0;
     for (int tile = tile_begin; tile < tile_end; ++tile) {
         if (tile >= t_hi) {
             do {
@@ -498,9 +499,8 @@ __global__ void __launch_bounds__(CTA16, PBF ? 5 : 6) solo_step_fast16_kernel(co
         }
         const int tin = tile - t_lo;
         if (skip || tin >= full_tiles) continue;
-        fast16_tile<BM, BV, PBF>(a, s, s_y, s_mid, pbase, gbase, tin, jb0 + (int64_t)tin * 16, tensor, par, ah,
+        fast16_tile<BM, BV, PBF>(a, s, s_y, s_mid, pbase, gbase, tin, jb0 + (int64_t)tin * 16, tensor, ah,
                     tin + 1 < full_tiles && tile + 1 < tile_end, 1);
-        par ^= 1;
     }
     if (tid == 0 && ah.failed && ah.fill > 0) {
         const uint32_t last = ah.fill - 1u;

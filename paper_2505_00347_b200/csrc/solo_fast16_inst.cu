@@ -1,28 +1,37 @@
-// The sixteen-elements-per-thread kernels: 2-bit first moment, 2/3/4-bit second moment, block 128,
-// fp32 or bf16 parameters, plain step.  (With wider first moments the nearest-level search over
-// sixteen elements costs more than the shared per-thread work saves: measured slower than the
-// eight-per-thread kernel, so those widths are not instantiated.)
+// The sixteen-elements-per-thread kernels: 2/3/4-bit states except 4-bit / 4-bit (measured slower
+// than the eight-per-thread kernel: 223 vs 236 Gparams/s), block 128, fp32 or bf16 parameters, plain
+// step.
 #include "solo_dispatch.h"
 #include "solo_fast16.cuh"
 
 namespace solo {
 
+#define SOLO_K16(BM, BV) (param_bf16 ? solo_step_fast16_kernel<BM, BV, true> : solo_step_fast16_kernel<BM, BV, false>)
+
 StepKernel fast16_kernel(int bits_m, int bits_v, bool param_bf16) {
-    if (bits_m != 2) return nullptr;
-    switch (bits_v) {
-        case 2: return param_bf16 ? solo_step_fast16_kernel<2, 2, true> : solo_step_fast16_kernel<2, 2, false>;
-        case 3: return param_bf16 ? solo_step_fast16_kernel<2, 3, true> : solo_step_fast16_kernel<2, 3, false>;
-        case 4: return param_bf16 ? solo_step_fast16_kernel<2, 4, true> : solo_step_fast16_kernel<2, 4, false>;
+    switch (bits_m * 10 + bits_v) {
+        case 22: return SOLO_K16(2, 2);
+        case 23: return SOLO_K16(2, 3);
+        case 24: return SOLO_K16(2, 4);
+        case 32: return SOLO_K16(3, 2);
+        case 33: return SOLO_K16(3, 3);
+        case 34: return SOLO_K16(3, 4);
+        case 42: return SOLO_K16(4, 2);
+        case 43: return SOLO_K16(4, 3);
         default: return nullptr;
     }
 }
 
 size_t fast16_kernel_smem(int bits_m, int bits_v) {
-    if (bits_m != 2) return 0;
-    switch (bits_v) {
-        case 2: return sizeof(Fast16Shared<2, 2>);
-        case 3: return sizeof(Fast16Shared<2, 3>);
-        case 4: return sizeof(Fast16Shared<2, 4>);
+    switch (bits_m * 10 + bits_v) {
+        case 22: return sizeof(Fast16Shared<2, 2>);
+        case 23: return sizeof(Fast16Shared<2, 3>);
+        case 24: return sizeof(Fast16Shared<2, 4>);
+        case 32: return sizeof(Fast16Shared<3, 2>);
+        case 33: return sizeof(Fast16Shared<3, 3>);
+        case 34: return sizeof(Fast16Shared<3, 4>);
+        case 42: return sizeof(Fast16Shared<4, 2>);
+        case 43: return sizeof(Fast16Shared<4, 3>);
         default: return 0;
     }
 }

@@ -80,9 +80,9 @@ def test_bits_and_blocks_random_state(bits_m, bits_v, block):
     params, gf = _inputs(w)
     st0 = synth.make_state(sizes, bits_m, bits_v, block, seed=bits_m * 100 + bits_v * 10 + block)
     hk = dict(lr=1e-3, beta1=0.8, beta2=0.999, weight_decay=0.01, seed=5)
-    # block 128 with a 2-bit first moment: policy 3 is the sixteen-per-thread kernel plus the
-    # streamlined kernel for the tails (policy 0 picks it for large tensors only)
-    policies = (0, 3, 1) if block == 128 and bits_m == 2 and bits_v <= 4 else (0, 1)
+    # block 128 with widths up to 4 bits: policy 3 is the sixteen-per-thread kernel plus the
+    # streamlined kernel for the tails (policy 0 picks it for large sets only)
+    policies = (0, 3, 1) if block == 128 and max(bits_m, bits_v) <= 4 else (0, 1)
     rep = run_lockstep(sizes, bits_m, bits_v, block, hk, 2, gf, params, state0=st0, policies=policies)
     assert rep.exempt_m + rep.exempt_v <= 3 * len(policies)
 
@@ -166,7 +166,7 @@ def test_bf16_parameters_every_kernel(bits_m, bits_v, block, param_round):
               param_round=param_round)
     st0 = synth.make_state(sizes, bits_m, bits_v, block, seed=block + bits_m)
     # (2, 3, 128): policy 3 adds the sixteen-per-thread kernel (policy 0 uses it for large sets only)
-    policies = (0, 3, 1) if (bits_m, block) == (2, 128) else (0, 1)
+    policies = (0, 3, 1) if block == 128 and max(bits_m, bits_v) <= 4 else (0, 1)
     run_lockstep(sizes, bits_m, bits_v, block, hk, 2, gf, params, state0=st0, policies=policies)
     run_lockstep(sizes, bits_m, bits_v, block, hk, 3, gf, params, policies=policies)
 
@@ -191,7 +191,7 @@ def test_stochastic_bf16_rounding_is_unbiased_on_the_device():
         st.destroy()
 
 
-@pytest.mark.parametrize("bits_m,bits_v", [(2, 3), (2, 2), (2, 4)])
+@pytest.mark.parametrize("bits_m,bits_v", [(2, 3), (2, 2), (2, 4), (3, 3), (4, 2), (4, 4), (3, 4), (4, 3), (3, 2)])
 def test_block_128_plain_step_all_three_kernels(bits_m, bits_v):
     """Block 128, plain step: the sixteen-per-thread kernel (policy 3: full tiles there, the rest in
     the streamlined kernel), the streamlined kernel alone (2) and the general kernel (1) against
