@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 # (dram__bytes_read.sum + dram__bytes_write.sum over the parameters of the captured launch, taken on
 # the first three tensors of the 7B-shaped set and scaled by the element count; see profiles/).
 # Valid for the 2-bit / 3-bit, block 128 streamlined kernel only; None for anything else.
-NCU_TRAFFIC_BYTES_PER_PARAM = 11.10
+NCU_TRAFFIC_BYTES_PER_PARAM = 11.11
 
 
 def algorithmic_bytes_per_param(bits_m: int, bits_v: int, block: int, param_bytes: int = 4) -> float:
