@@ -28,8 +28,8 @@
 // two halves of a warp are reduced by one minimum and one maximum over a transformed
 // value: all quantities reduced here are non-negative binary32 bit patterns (bit 31
 // clear), so complementing the upper half's values moves them above every lower-half
-// value and reverses their order.  For G = 8 the same is done for each pair of groups, the
-// other pair's lanes contributing a neutral value.
+// value and reverses their order.  For G = 8 (four groups per warp) three shuffle-and-compare
+// steps over the untransformed values serve all groups at once.
 #pragma once
 
 #include <type_traits>
@@ -179,34 +179,30 @@ __device__ __forceinline__ void philox_rk(uint32_t c0, uint32_t c1, uint32_t c2,
 }
 
 // ---------------------------------------------------------------------------
-// Group collectives on 31-bit values, full-mask instructions only.
-// `hi`: the lane belongs to the odd group of its pair of groups (G = 16: the upper half of the
-// warp; G = 8: lanes 8..15 and 24..31).  NEUTRAL neither lowers a minimum over the even group's
-// values (bit 31 clear) nor raises a maximum over the odd group's (bit 31 set).
+// Group collectives on 31-bit values.
+// `hi` (G = 16 only): the lane belongs to the upper half of the warp, the odd group of the pair.
 // ---------------------------------------------------------------------------
-constexpr uint32_t NEUTRAL = 0x7FFFFFFFu;
 
 // min over the even group and max over the odd group of `u`, for the calling lane's pair; returns
 // the one that belongs to the lane's own group
 template <int G>
 __device__ __forceinline__ uint32_t seg_pick(uint32_t u, bool hi) {
-    if constexpr (G == 16) {
-        const uint32_t lo = __reduce_min_sync(0xffffffffu, u);
-        const uint32_t up = __reduce_max_sync(0xffffffffu, u);
-        return hi ? up : lo;
-    } else {
-        static_assert(G == 8, "group of 8, 16 or 32 lanes");
-        const bool pair1 = (threadIdx.x & 16) != 0;
-        const uint32_t ua = pair1 ? NEUTRAL : u, ub = pair1 ? u : NEUTRAL;
-        const uint32_t a_lo = __reduce_min_sync(0xffffffffu, ua), a_up = __reduce_max_sync(0xffffffffu, ua);
-        const uint32_t b_lo = __reduce_min_sync(0xffffffffu, ub), b_up = __reduce_max_sync(0xffffffffu, ub);
-        return pair1 ? (hi ? b_up : b_lo) : (hi ? a_up : a_lo);
-    }
+    static_assert(G == 16, "two groups of sixteen lanes");
+    const uint32_t lo = __reduce_min_sync(0xffffffffu, u);
+    const uint32_t up = __reduce_max_sync(0xffffffffu, u);
+    return hi ? up : lo;
 }
 template <int G>
 __device__ __forceinline__ uint32_t seg_max31(uint32_t x, bool hi) {
     if constexpr (G == 32) {
         return __reduce_max_sync(0xffffffffu, x);
+    } else if constexpr (G == 8) {
+        // four groups per warp: three shuffle-and-compare steps serve them all and were measured
+        // faster than four reductions plus selects (the groups of eight use no transformed domain:
+        // `hi` is false for them)
+#pragma unroll
+        for (int d = 1; d < 8; d <<= 1) x = max(x, __shfl_xor_sync(0xffffffffu, x, d));
+        return x;
     } else {
         // even group: complement of the low 31 bits (order reversed, bit 31 clear); odd group:
         // bit 31 set.  min = even group's maximum, max = odd group's maximum.
@@ -220,6 +216,10 @@ template <int G>
 __device__ __forceinline__ uint32_t seg_min_v(uint32_t v, bool hi) {
     if constexpr (G == 32) {
         return __reduce_min_sync(0xffffffffu, v);
+    } else if constexpr (G == 8) {
+#pragma unroll
+        for (int d = 1; d < 8; d <<= 1) v = min(v, __shfl_xor_sync(0xffffffffu, v, d));
+        return v;
     } else {
         return seg_pick<G>(v, hi);
     }
@@ -500,7 +500,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
     const bool round_v = PLAIN || a.round_v;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gl = tid & (G - 1), grp = tid / G;
-    const bool hi = G < 32 && (lane & G) != 0;                  // odd group of its pair
+    const bool hi = G == 16 && (lane & G) != 0;                 // odd group of its pair (groups of 16 only)
     const uint32_t vflip = hi ? 0xFFFFFFFFu : 0u;               // x domain <-> v domain
 
     // validity (all true in a full tile)
@@ -935,7 +935,7 @@ __global__ void __launch_bounds__(CTA, (BM == 8 || BV == 8) ? 3 : 4) solo_step_f
         s_y[i] = a.tables[i];
         if (i < KM - 1) s_mid[i] = a.tables[KM + i];
     }
-    for (int r = 7; r < 16; ++r) s.sort[r][tid] = (G < 32 && (tid & G)) ? ~KEY_MAX : KEY_MAX;   // sentinels, v domain
+    for (int r = 7; r < 16; ++r) s.sort[r][tid] = (G == 16 && (tid & G)) ? ~KEY_MAX : KEY_MAX;   // sentinels, v domain
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s.mbar[0])) : "memory");
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s.mbar[1])) : "memory");
