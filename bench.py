@@ -244,7 +244,8 @@ def run_ours(args, rank, world):
                                + (f", baseline v codebook {args.v_codebook}" if args.v_codebook else ""),
                    "l2": "working set (params+grads+state) far larger than the 126 MB L2; no flush needed"
                          if n * abytes > 1e9 else "working set fits L2: launch-bound point, not a bandwidth point",
-                   "bytes_per_param": round(abytes, 4)},
+                   "bytes_per_param": round(abytes, 4),
+                   "kernel_launches_per_step": round(launches / args.steps, 2)},
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
                      "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind} copy bandwidth",
                      "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
