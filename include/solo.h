@@ -82,13 +82,13 @@ typedef struct {
     int32_t round_m;       /* 0: nearest level (Eq. 1); 1: stochastic rounding (Eq. 5) */
     int32_t round_v;       /* 1: xi ~ U(-1/2,1/2) in Eq. 6; 0: xi = 0 (deterministic) */
     int32_t param_dtype;   /* 0: fp32 parameters; 1: bf16 parameters */
-    int32_t belief;        /* 0: Adam(W); 1: AdaBelief (Sec. 5.2): the unsigned EMA tracks
+    int32_t belief;        /* 0: Adam(W); 1: AdaBelief (Sec. 4.2): the unsigned EMA tracks
                               (g - m^)^2 and eps is added to it at every step */
     int32_t param_round;   /* bf16 parameters: 0 round to nearest even; 1 stochastic rounding with
                               the element's Philox draw (purpose 2).  No counterpart in the paper,
-                              whose 16-bit baseline is plain BF16 (Sec. 5, "Baselines") */
+                              whose 16-bit baseline is plain BF16 (Sec. 4, "Baselines") */
     int32_t v_codebook;    /* quantizer of the unsigned state: SOLO_V_LOG (Eq. 6, the paper's), or
-                              one of the baselines of Sec. 5 (block-wise absmax scaling, nearest
+                              one of the baselines of Sec. 4 (block-wise absmax scaling, nearest
                               level of a fixed codebook, Eq. 1): SOLO_V_DE, SOLO_V_LINEAR,
                               SOLO_V_LINEAR_NOZERO.  A state must be stepped and dequantized
                               with the selector it was written with */
@@ -129,7 +129,7 @@ int solo_state_create_multi(const int64_t* numel_host, int num_tensors, int bits
 int solo_state_destroy(solo_state_t* state);
 
 /*
- * Memory accounting of Sec. 5.2 ("Block size") / Table 2: bytes of state for one
+ * Memory accounting of Sec. 4.2 ("Block size") / Table 2: bytes of state for one
  * tensor = codes of both moments (whole slots) + 12 bytes per block.  Host only.
  */
 int solo_state_bytes(int64_t numel, int bits_m, int bits_v, int block, size_t* out);

@@ -21,8 +21,11 @@
 // Proposition 3.5 decay statistics, Theorem 3.6 (unbiased SR, variance bound),
 // brute-force nearest-level search, Philox known answers, textbook AdamW,
 // memory accounting of Table 2, the stochastic bf16 rounding over all 2^16
-// draws, the baseline second-moment codebooks by exhaustive search and the
-// swamping of Corollary 3.2 through the whole step.  Unpinned (paper silent; internal consistency
+// draws, the baseline second-moment codebooks by exhaustive search, the
+// swamping of Corollary 3.2 through the whole step, the decode of the previous
+// packed state (Eq. 2) redone in binary64 from the bytes with the Appendix A
+// levels typed out, and every Eq. 5 code of the step against the element's own
+// draw.  Unpinned (paper silent; internal consistency
 // only): the rank convention of the p-quantile, the clamp constants of the
 // base, the 3-bit layout, the +1/-1 orientation of the signed DE codebook.
 //
@@ -289,7 +292,7 @@ inline uint16_t float_to_bf16(float x) {         // round to nearest, ties to ev
 // bits).  A value already representable is returned unchanged; the largest
 // finite magnitudes can round to infinity; infinities and NaN are truncated
 // (NaN kept quiet).  Not from the paper: its 16-bit baseline is plain BF16
-// (Sec. 5, "Baselines"); this is the usual companion of bf16 parameters without
+// (Sec. 4, "Baselines"); this is the usual companion of bf16 parameters without
 // a binary32 master copy.
 inline uint16_t float_to_bf16_sr(float x, uint32_t d) {
     uint32_t u = f2u(x);
@@ -329,7 +332,7 @@ struct so_hyper {
     int32_t belief;       // 0: Adam(W); 1: AdaBelief (second moment tracks (g - m^)^2 + eps)
     int32_t param_round;  // bf16 parameters: 0 round to nearest even, 1 stochastic (Philox purpose 2)
     int32_t v_codebook;   // second moment: 0 logarithmic, Eq. 6 (SOLO); 1 unsigned DE, 2 linear,
-                          // 3 linear without zero -- the baselines of Sec. 5, nearest rounding (Eq. 1)
+                          // 3 linear without zero -- the baselines of Sec. 4, nearest rounding (Eq. 1)
     uint64_t seed;
 };
 
@@ -360,7 +363,7 @@ void so_set_code(uint8_t* blk, int e, int b, int v) { set_code(blk, e, b, v); }
 
 // Bytes of optimizer state for `numel` elements: packed codes of both moments
 // (a full slot for every block, tail included) plus three binary32 words per
-// block (Delta_m, Delta_v, alpha).  Sec. 5.2 "Block size": one binary32 scale
+// block (Delta_m, Delta_v, alpha).  Sec. 4.2 "Block size": one binary32 scale
 // costs 1/4 bit per element at block 128, SOLO's buffered base doubles that
 // for the second moment.
 int so_state_bytes(int64_t numel, int bits_m, int bits_v, int block, uint64_t* out) {
@@ -445,7 +448,7 @@ static void step_blocks(void* param, const uint16_t* grad, int64_t n, int64_t el
             float v_t = v32 ? v32[i]
                       : v_kind >= 0 ? yv[get_code(cv, e, bits_v)] * dv
                                     : pow_sm(al, get_code(cv, e, bits_v)) * dv;
-            // Eq. 3.  AdaBelief (Sec. 5.2, "AdaBelief"; Zhuang et al. 2020): the unsigned EMA's
+            // Eq. 3.  AdaBelief (Sec. 4.2, "AdaBelief"; Zhuang et al. 2020): the unsigned EMA's
             // signal is (g - m^)^2 instead of g^2 and eps is added to the state at every step
             float m_h = std::fmaf(b1, m_t, omb1 * g);
             float sig = h->belief ? g - m_h : g;
@@ -511,7 +514,7 @@ static void step_blocks(void* param, const uint16_t* grad, int64_t n, int64_t el
             alpha[j] = 0.5f;
         } else if (v_kind >= 0) {
             // baseline: block-wise absmax scaling and the nearest level of a fixed codebook
-            // (Eq. 1; Sec. 5, "Baselines"); the base is not used and keeps its initial value
+            // (Eq. 1; Sec. 4, "Baselines"); the base is not used and keeps its initial value
             scale_v[j] = dv_new;
             alpha[j] = 0.5f;
             const float inv = 1.0f / dv_new;

@@ -141,7 +141,7 @@ def test_hyper_parameter_modes(hk):
 @pytest.mark.parametrize("sel", [1, 2, 3])
 @pytest.mark.parametrize("bits_v,block", [(2, 64), (3, 128), (4, 2048), (8, 256)])
 def test_baseline_second_moment_codebooks(sel, bits_v, block):
-    """Sec. 5 baselines for the unsigned state (unsigned DE, linear, linear without zero;
+    """Sec. 4 baselines for the unsigned state (unsigned DE, linear, linear without zero;
     Appendix A) at every width, from a random packed state and from zero, ragged sizes."""
     sizes = (block * 5 + 3, 1, 2048 * 2 + 9, block - 1)
     w = synth.workload(4, sizes=sizes)                            # zero blocks and zero elements

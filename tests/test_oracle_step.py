@@ -326,7 +326,7 @@ def test_bf16_parameters_stochastic_rounding():
 @pytest.mark.parametrize("sel,kind", [(1, "DE_UNSIGNED"), (2, "LINEAR_UNSIGNED"), (3, "LINEAR_NOZERO")])
 @pytest.mark.parametrize("bits_v", [2, 4])
 def test_baseline_second_moment_codebooks(sel, kind, bits_v):
-    """v_codebook != 0 (Sec. 5, "Baselines"): block-wise absmax scaling, codes are the nearest
+    """v_codebook != 0 (Sec. 4, "Baselines"): block-wise absmax scaling, codes are the nearest
     level by exhaustive search, dequantization is level times scale, the base is not touched."""
     n, block = 128 * 4 + 40, 128
     p, _, _ = rand_inputs(n, 21)
