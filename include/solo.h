@@ -149,8 +149,11 @@ int solo_step(void* param_dev, const void* grad_dev, solo_state_t* state,
               const solo_hyper_t* hyper, int64_t step, void* stream);
 
 /*
- * The same step over every tensor of the list in ONE kernel launch, ragged block
- * tails included.  Tensor t uses Philox stream t.  Asynchronous on `stream`.
+ * The same step over every tensor of the list, ragged block tails included, in one kernel
+ * launch -- or in two when the kernel with sixteen elements per thread is selected (see
+ * solo_set_kernel_policy: large sets at block 128; it takes the full 2048-element tiles and a
+ * second, short launch the tiles that are not full; policy 2 keeps every set to one launch).
+ * Tensor t uses Philox stream t.  Asynchronous on `stream`.
  */
 int solo_multi_step(const solo_tensor_list_t* list, const solo_hyper_t* hyper, int64_t step,
                     void* stream);
@@ -232,12 +235,15 @@ int solo_state_export(const solo_state_t* state, void* host_dst, size_t bytes, v
 int solo_state_import(solo_state_t* state, const void* host_src, size_t bytes, void* stream);
 
 /*
- * Reads the state's device status word into *status_out (0 = no problem seen).
+ * Reads the state's device status word into *status_out (0 = no problem seen).  The word is
+ * sticky: bits stay set until the state is destroyed.
  *   bit 0  a solo_multi_step descriptor's numel disagreed with the state; the affected
  *          tensors were skipped
  *   bit 1  a kernel that stages its inputs gave up waiting for an asynchronous copy of them
- *          (a bounded wait, so the kernel always ends); the results of that step are undefined
- * Synchronizes the device.
+ *          (a bounded wait, so the kernel always ends).  The warps that gave up stored nothing
+ *          for the tiles concerned: those parameters and state blocks keep their old values,
+ *          i.e. the step is incomplete
+ * Synchronizes the device.  (No counterpart in the paper: error reporting of this library.)
  */
 int solo_state_status(solo_state_t* state, int* status_out);
 
@@ -332,13 +338,36 @@ typedef struct {
  * The fixed array is shared by every call on a device and is rewritten by each call, in
  * stream order: calls whose GPU work can overlap (different streams without ordering between
  * them) race on it and must be serialised by the caller.  Its address is looked up on the
- * first call on each device; make that first call outside any stream capture.  No
- * cudaMalloc, cudaFree or other allocating routine is called.  Asynchronous on `stream`
- * except for the copy of the offsets from host memory, which is staged before the call returns.
+ * first call on each device.  The call copies its tables from its own stack frame, so it must
+ * not be made while `stream` is capturing: that is refused with SOLO_EINVAL before anything is
+ * queued.  No cudaMalloc, cudaFree or other allocating routine is called.  Asynchronous on
+ * `stream` except for the copy of the offsets from host memory, which is staged before the call
+ * returns.  solo_static_status reads the call's status word.
  */
 int solo_multi_step_static(int32_t num_tensors, void* const* param_dev, const void* const* grad_dev,
                            const int64_t* numel_host, const solo_raw_state_t* st,
                            const solo_hyper_t* hyper, int64_t step, void* stream);
+
+/*
+ * The status word of solo_multi_step_static's last call on the current device (same bits as
+ * solo_state_status; every solo_multi_step_static call clears it before its kernels run).
+ * Copies the word from the fixed array to HOST *status_out on `stream` and waits for that
+ * stream; allocates nothing.  Call it on the stream the step was issued on, or after that
+ * stream's work has completed.  (No counterpart in the paper.)
+ */
+int solo_static_status(int* status_out, void* stream);
+
+/*
+ * Test hook for the bounded wait of the kernels that stage their inputs with asynchronous
+ * copies.  The next step launched by this process announces 16 bytes more than it copies for
+ * the inputs of tile number `tile` (tiles of 2048 elements, counted over the tensor list), so the
+ * wait for that tile's inputs runs out after its fixed number of polls: the waiting warps set
+ * status bit 1, store nothing for that tile and the tiles their CTA processes after it, and the
+ * kernel returns.  Nothing faults and nothing spins without limit.  One-shot and process-wide;
+ * tiles that are not staged (not full, or in the general kernel) ignore it.  (No counterpart
+ * in the paper.)
+ */
+int solo_debug_stall_copy(int64_t tile);
 
 /* Number of kernel launches issued by this library in the calling process so far. */
 int64_t solo_launch_count(void);

@@ -116,6 +116,10 @@ def lib() -> C.CDLL:
     L.solo_state_export_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
     L.solo_state_export.argtypes = [vp, vp, C.c_size_t, vp]
     L.solo_state_import.argtypes = [vp, vp, C.c_size_t, vp]
+    L.solo_static_status.argtypes = [C.POINTER(C.c_int), vp]
+    L.solo_static_status.restype = C.c_int
+    L.solo_debug_stall_copy.argtypes = [i64]
+    L.solo_debug_stall_copy.restype = C.c_int
     L.solo_launch_count.argtypes = []
     L.solo_launch_count.restype = C.c_int64
     L.solo_strerror.argtypes = [i32]
@@ -388,6 +392,20 @@ def debug_check_fast_log(lo_bits: int, hi_bits: int) -> tuple[float, float]:
     _check(lib().solo_debug_check_fast_log(lo_bits, hi_bits, C.byref(ex), C.byref(ab)),
            "solo_debug_check_fast_log")
     return ex.value, ab.value
+
+
+def static_status() -> int:
+    """Status word of the last solo_multi_step_static call on the current device (waits for the
+    current stream)."""
+    out = C.c_int(-1)
+    _check(lib().solo_static_status(C.byref(out), _stream()), "solo_static_status")
+    return out.value
+
+
+def debug_stall_copy(tile: int) -> None:
+    """Test hook: the next step over-announces the input copy of tile `tile`, so the bounded wait
+    for it runs out."""
+    _check(lib().solo_debug_stall_copy(int(tile)), "solo_debug_stall_copy")
 
 
 def launch_count() -> int:

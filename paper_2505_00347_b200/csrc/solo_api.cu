@@ -54,6 +54,7 @@ struct HostPipe {
 namespace {
 
 std::atomic<int64_t> g_launches{0};
+std::atomic<int64_t> g_stall_tile_p1{0};   // test hook: 1 + tile whose input copy the next step over-announces; 0: none
 std::atomic<int> g_policy{0};          // 0: fastest kernel that applies; 1: general kernel only; 2: no sixteen-per-thread
                                        // kernel; 3: sixteen-per-thread kernel wherever it exists
 
@@ -217,6 +218,7 @@ int launch_kernel(solo::StepKernel k, const StepArgs& a, int device, int threads
 }
 
 int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
+    a.debug_stall_tile_p1 = g_stall_tile_p1.exchange(0, std::memory_order_relaxed);
     const bool cta_group = s->block == 2048;
     const int policy = g_policy.load(std::memory_order_relaxed);
     const bool streamlined = policy != 1 && !a.round_m && !a.tables_v && a.eps >= 1e-12f &&
@@ -231,7 +233,7 @@ int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
     if (k16) {
         // blocks of 128, plain step: full tiles by the sixteen-per-thread kernel, whatever it leaves
         // (tails, tensors that are not 16-byte aligned) by the streamlined kernel
-        int rc = launch_kernel(k16, a, s->device, solo::CTA16, solo::fast16_kernel_smem(s->bits_m, s->bits_v), stream);
+        int rc = launch_kernel(k16, a, s->device, solo::CTA16, solo::fast16_kernel_smem(s->bits_m, s->bits_v, a.param_bf16 != 0), stream);
         if (rc) return rc;
         const bool all_full = !a.param_list && s->num_tensors == 1 && s->numel[0] % solo::TILE == 0;
         if (all_full) return SOLO_OK;
@@ -615,8 +617,12 @@ int solo_multi_step_static(int32_t num_tensors, void* const* param_dev, const vo
     rc = static_scratch(device, &scratch);
     if (rc) return rc;
     cudaStream_t stream = (cudaStream_t)stream_;
+    // the tables below are copied from this call's stack: a captured copy would read a dead frame at replay
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) { cudaGetLastError(); return SOLO_ECUDA; }
+    if (cap != cudaStreamCaptureStatusNone) return SOLO_EINVAL;
 
-    // geometry and codebook tables, built in fixed-size host arrays (no heap, no device allocation)
+    // geometry and codebook tables, built in fixed-size host arrays (no device allocation)
     const int T = num_tensors, block = st->block;
     int64_t geom[3 * STATIC_MAX_T + 2];
     int64_t* numel = geom;
@@ -685,6 +691,28 @@ int solo_multi_step_static(int32_t num_tensors, void* const* param_dev, const vo
     a.grad_list = grad_dev;
     a.numel_check = nullptr;
     return launch_step(&tmp, a, stream);
+}
+
+int solo_static_status(int* status_out, void* stream_) {
+    if (!status_out) return SOLO_EINVAL;
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) { cudaGetLastError(); return SOLO_ECUDA; }
+    unsigned char* scratch = nullptr;
+    int rc = static_scratch(device, &scratch);
+    if (rc) return rc;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    if (cudaMemcpyAsync(status_out, scratch + STATIC_STATUS_OFF, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess) {
+        cudaGetLastError();
+        return SOLO_ECUDA;
+    }
+    return SOLO_OK;
+}
+
+int solo_debug_stall_copy(int64_t tile) {
+    if (tile < 0) return SOLO_EINVAL;
+    g_stall_tile_p1.store(tile + 1, std::memory_order_relaxed);
+    return SOLO_OK;
 }
 
 int solo_dequant(const solo_state_t* s, int which, float* out_dev, void* stream) {

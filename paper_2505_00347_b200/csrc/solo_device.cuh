@@ -41,6 +41,8 @@ struct StepArgs {
     int64_t total_tiles;               // the launch covers tiles [tile_first, total_tiles)
     int64_t tile_first;
     int32_t only_partial;              // streamlined kernel: skip full tiles of aligned tensors (another launch did them)
+    int64_t debug_stall_tile_p1;       // test hook of the staged kernels: 1 + the number of the tile whose input copy
+                                       // announces 16 bytes more than it brings (the wait for it runs out); 0: none
     // state
     uint8_t* codes_m;
     uint8_t* codes_v;

@@ -44,7 +44,7 @@ StepKernel fast_kernel(int bits_m, int bits_v, int block, bool param_bf16, bool 
 // for other widths.
 constexpr int CTA16 = 128;         // threads per CTA of that kernel
 StepKernel fast16_kernel(int bits_m, int bits_v, bool param_bf16);
-size_t fast16_kernel_smem(int bits_m, int bits_v);
+size_t fast16_kernel_smem(int bits_m, int bits_v, bool param_bf16);
 // Dynamic shared memory the streamlined kernel for these widths is launched with.
 size_t fast_kernel_smem(int bits_m, int bits_v);
 // Resident CTAs per SM of a step kernel launched with `dyn_smem` bytes of dynamic shared memory

@@ -76,15 +76,17 @@ using FastShared = FastSharedT<(BM == 8 ? 2 : 1), (BV == 8 ? 2 : 1)>;
 struct Ahead {
     uint32_t fill = 0;        // number of the next bulk copy to wait for (uniform over the CTA)
     bool staged = false;      // that copy has already been issued (uniform)
-    bool failed = false;      // this thread once waited in vain for a copy
+    bool failed = false;      // this thread once waited in vain for a copy: it polls once per tile from then on
+                              // and its warp stores nothing
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 // Waits until the phase with the given parity of an mbarrier has completed.  Bounded: gives up
-// (returns false) after 2^14 timed-out polls instead of spinning for ever.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (int it = 0; it < (1 << 14); ++it) {
+// (returns false) after `polls` timed-out polls (2^14 unless told otherwise) instead of spinning for ever.
+constexpr int MBAR_POLLS = 1 << 14;
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int polls = MBAR_POLLS) {
+    for (int it = 0; it < polls; ++it) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
@@ -112,6 +114,14 @@ __device__ __forceinline__ float rcp_approx(float x) {
     float y;
     asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+
+// max(acc, |x|) that returns NaN when x is NaN: a NaN among the block's values makes the block's
+// scale NaN, as the maximum over bit patterns of the general kernel does.
+__device__ __forceinline__ float max_abs_nan(float acc, float x) {
+    float r;
+    asm("{\n\t.reg .f32 t;\n\tabs.f32 t, %2;\n\tmax.NaN.f32 %0, %1, t;\n\t}" : "=f"(r) : "f"(acc), "f"(x));
+    return r;
 }
 
 // The two 16-bit halves of a word as binary32 (one conversion each, no shift or mask).
@@ -249,9 +259,10 @@ __device__ __forceinline__ uint32_t warp_load_codes(const uint8_t* warp_base, in
 // first block is odd) and scalars are copied from the 16-byte boundary at or below them, with 16
 // bytes more when they do not start on it; readers add the offset.  The scalar arrays are
 // allocated in multiples of 16 bytes, so the copy never leaves them.
+// `extra_tx`: bytes announced on top of what is copied (test hook: the wait for this tile then runs out).
 template <int BM, int BV, int G, bool PBF>
 __device__ __forceinline__ void issue_tile_copy(const StepArgs& a, FastShared<BM, BV>& s, uint32_t fill, const char* pt,
-                                                const char* gt, int64_t jb_tile) {
+                                                const char* gt, int64_t jb_tile, uint32_t extra_tx) {
     constexpr int NG = CTA / G;
     constexpr uint32_t PBYTES = TILE * (PBF ? 2 : 4);
     typename FastShared<BM, BV>::Stage& st = s.stage[fill & 1u];
@@ -262,7 +273,7 @@ __device__ __forceinline__ void issue_tile_copy(const StepArgs& a, FastShared<BM
     // single block's scalar (NG = 1) lies within the 16 bytes that start at that boundary
     const uint32_t bytes_s = NG >= 4 ? (NG + ((jb_tile & 3) ? 4u : 0u)) * 4u : 16u;
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar),
-                 "r"((uint32_t)(PBYTES + TILE * 2) + bytes_m + bytes_v + 3u * bytes_s) : "memory");
+                 "r"((uint32_t)(PBYTES + TILE * 2) + bytes_m + bytes_v + 3u * bytes_s + extra_tx) : "memory");
     bulk_copy(st.p, pt, PBYTES, bar);
     bulk_copy(st.g, gt, TILE * 2, bar);
     bulk_copy(st.cm, a.codes_m + (bm0 & ~(int64_t)15), bytes_m, bar);
@@ -283,16 +294,16 @@ __device__ __forceinline__ uint32_t warp_codes_finish(uint32_t w, int lane) {
     return __funnelshift_r(lo, hi, o) & 0xFFFFFFu;
 }
 template <int BITS>
-__device__ __forceinline__ void warp_store_codes(uint8_t* warp_base, int lane, uint32_t c) {
+__device__ __forceinline__ void warp_store_codes(uint8_t* warp_base, int lane, uint32_t c, bool keep) {
     if constexpr (BITS == 2) {
-        __stcs(reinterpret_cast<unsigned short*>(warp_base) + lane, (unsigned short)c);
+        if (keep) __stcs(reinterpret_cast<unsigned short*>(warp_base) + lane, (unsigned short)c);
     } else if constexpr (BITS == 4) {
-        __stcs(reinterpret_cast<unsigned int*>(warp_base) + lane, c);
+        if (keep) __stcs(reinterpret_cast<unsigned int*>(warp_base) + lane, c);
     } else {
         const int a = (4 * lane) / 3, o = 32 * lane - 24 * a;        // o in {0, 8, 16} for lane < 24
         const uint32_t lo = __shfl_sync(0xffffffffu, c, a & 31);
         const uint32_t hi = __shfl_sync(0xffffffffu, c, (a + 1) & 31);
-        if (lane < 24)
+        if (lane < 24 && keep)
             __stcs(reinterpret_cast<unsigned int*>(warp_base) + lane, (lo >> (o & 31)) | (hi << ((24 - o) & 31)));
     }
 }
@@ -489,7 +500,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
                                           const float* s_mid, char* pbase, const char* gbase,
                                           const int64_t n, const int tin, const int64_t jb_tile,
                                           const int tensor, const int par, Ahead& ah, const bool next_full,
-                                          const int next_dtin) {
+                                          const int next_dtin, const int64_t tile_no) {
     constexpr int KM = 1 << BM, KV = 1 << BV;
     constexpr int NG = CTA / G, B = G * EPT;
     constexpr int PSZ = PBF ? 2 : 4;                            // bytes per parameter
@@ -530,18 +541,20 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
         // refilled all threads have finished reading it: they read at the start of a tile and
         // pass that tile's barriers before any thread starts the next one.
         if (tid == 0) {
-            if (!ah.staged) issue_tile_copy<BM, BV, G, PBF>(a, s, ah.fill, pt, gt, jb_tile);
+            if (!ah.staged)
+                issue_tile_copy<BM, BV, G, PBF>(a, s, ah.fill, pt, gt, jb_tile, tile_no + 1 == a.debug_stall_tile_p1 ? 16u : 0u);
             if (next_full)
                 issue_tile_copy<BM, BV, G, PBF>(a, s, ah.fill + 1u, pt + (int64_t)next_dtin * (TILE * PSZ),
-                                           gt + (int64_t)next_dtin * (TILE * 2), jb_tile + (int64_t)next_dtin * NG);
+                                           gt + (int64_t)next_dtin * (TILE * 2), jb_tile + (int64_t)next_dtin * NG,
+                                           tile_no + next_dtin + 1 == a.debug_stall_tile_p1 ? 16u : 0u);
         }
         const uint32_t mine = ah.fill;
         ah.fill += 1u;
         ah.staged = next_full;
-        if (!mbar_wait(smem_u32(&s.mbar[mine & 1u]), (mine >> 1) & 1u)) {
-            // the copy was never seen to arrive: flag it; what the stage holds is used as it is
-            // (the step's results are then undefined, solo_state_status reports bit 1)
-            atomicOr(a.status, 2);
+        if (!mbar_wait(smem_u32(&s.mbar[mine & 1u]), (mine >> 1) & 1u, ah.failed ? 1 : MBAR_POLLS)) {
+            // the copy was never seen to arrive: flag it (solo_state_status reports bit 1); what the
+            // stage holds is worked on as it is, but nothing derived from it is stored (see `keep`)
+            if (!ah.failed) atomicOr(a.status, 2);
             ah.failed = true;
         }
         const typename FastShared<BM, BV>::Stage& st = s.stage[mine & 1u];
@@ -602,6 +615,14 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
         }
     }
 
+    // A warp in which any lane gave up waiting for its inputs stores nothing for this tile: parameters
+    // and state keep their old values.  Blocks of 2048 span the CTA, which then decides as a whole.
+    bool keep = true;
+    if (FULL) {
+        if constexpr (G == CTA) keep = !__syncthreads_or(ah.failed ? 1 : 0);
+        else keep = !__any_sync(0xffffffffu, ah.failed);
+    }
+
     // ---- per-block level tables: alpha^k Delta_v and y_k Delta_m (Eq. 2) ----
     // 8-bit second moments: the table holds the product of the first four factors of the
     // square-and-multiply chain (alpha^(q & 15)); the other four are multiplied on per element.
@@ -639,7 +660,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
     // ---- Eq. 2, Eq. 3, Adam(W) ----
     float mh[EPT], vh[EPT];
     uint32_t mx_v = 0;
-    float mx_m_f = 0.0f;                                         // max |m^| (a NaN element is passed over)
+    float mx_m_f = 0.0f;                                         // max |m^|, NaN if any is
     const char* const tab_v = reinterpret_cast<const char*>(tab);
     const char* const tab_m = reinterpret_cast<const char*>(tab + KVT);
     const CodeOffsets<BM> om4(cm, cm_hi);
@@ -669,7 +690,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
             vh[i] = __fmaf_rn(a.beta2, vt, a.omb2 * (gi * gi));
         }
         const bool valid = FULL || i < nv;
-        mx_m_f = fmaxf(mx_m_f, valid ? fabsf(mh[i]) : 0.0f);
+        mx_m_f = max_abs_nan(mx_m_f, valid ? mh[i] : 0.0f);
         mx_v = max(mx_v, valid ? __float_as_uint(vh[i]) : 0u);
     }
     };
@@ -702,7 +723,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
                             pp[j] = *reinterpret_cast<const uint32_t*>(&h);
                         }
                     }
-                    __stcs(reinterpret_cast<uint4*>(pt) + tid, make_uint4(pp[0], pp[1], pp[2], pp[3]));
+                    if (keep) __stcs(reinterpret_cast<uint4*>(pt) + tid, make_uint4(pp[0], pp[1], pp[2], pp[3]));
                 }
             } else if (i < nv) {
                 reinterpret_cast<uint16_t*>(pt)[tid * EPT + i] =
@@ -717,8 +738,8 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
         const float q1 = __fmaf_rn(__fmaf_rn(-den, q0, mh[i]), rc, q0);
         p[i] = __fmaf_rn(-a.step_size, q1, p[i] * a.decay);
         if (FULL) {
-            if (i == 3) __stcs(reinterpret_cast<float4*>(pt) + 2 * tid, make_float4(p[0], p[1], p[2], p[3]));
-            if (i == 7) __stcs(reinterpret_cast<float4*>(pt) + 2 * tid + 1, make_float4(p[4], p[5], p[6], p[7]));
+            if (i == 3 && keep) __stcs(reinterpret_cast<float4*>(pt) + 2 * tid, make_float4(p[0], p[1], p[2], p[3]));
+            if (i == 7 && keep) __stcs(reinterpret_cast<float4*>(pt) + 2 * tid + 1, make_float4(p[4], p[5], p[6], p[7]));
         } else {
             if (i < nv) reinterpret_cast<float*>(pt)[tid * EPT + i] = p[i];
         }
@@ -779,7 +800,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
     }
 
     // ---- per-block scalars, once per block, by the first warp; the others draw xi meanwhile ----
-    if (gl == 0) s.xin[par][grp] = make_uint4(mx_m, mx_v, x_p, 0u);
+    if (gl == 0) s.xin[par][grp] = make_uint4(mx_m, mx_v, x_p, keep ? 0u : 1u);   // .w: the block's warp stores nothing
     bar_sync(1);
     uint32_t w[4] = {0u, 0u, 0u, 0u};
     if (warp != 0) {
@@ -798,7 +819,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
         s.xout[par][tid] = make_float4(inv_dm, inv_dv, inv_lambda, 0.5f - guard);
         s.xflag[par][tid] = (zero_m ? 1u : 0u) | (zero_v ? 2u : 0u);
         const bool blk_exists = FULL || (int64_t)tid * B < rem_tile;
-        if (blk_exists) {
+        if (blk_exists && in.w == 0u) {
             const int64_t j = jb_tile + tid;
             a.scale_m[j] = zero_m ? 0.0f : dm_new;
             a.scale_v[j] = zero_v ? 0.0f : dv_new;
@@ -913,10 +934,10 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
 
     // ---- store the codes ----
     if (FULL) {
-        if constexpr (BM == 8) __stcs(reinterpret_cast<uint2*>(wcm) + lane, make_uint2(om, om_hi));
-        else warp_store_codes<BM>(wcm, lane, om);
-        if constexpr (BV == 8) __stcs(reinterpret_cast<uint2*>(wcv) + lane, make_uint2(ov, ov_hi));
-        else warp_store_codes<BV>(wcv, lane, ov);
+        if constexpr (BM == 8) { if (keep) __stcs(reinterpret_cast<uint2*>(wcm) + lane, make_uint2(om, om_hi)); }
+        else warp_store_codes<BM>(wcm, lane, om, keep);
+        if constexpr (BV == 8) { if (keep) __stcs(reinterpret_cast<uint2*>(wcv) + lane, make_uint2(ov, ov_hi)); }
+        else warp_store_codes<BV>(wcv, lane, ov, keep);
     } else if (have_block) {
         store_codes<BM>(wcm + lane * BM, ((uint64_t)om_hi << 32) | om);
         store_codes<BV>(wcv + lane * BV, ((uint64_t)ov_hi << 32) | ov);
@@ -988,15 +1009,15 @@ __global__ void __launch_bounds__(CTA, (BM == 8 || BV == 8) ? 3 : 4) solo_step_f
         const int64_t jb_tile = jb0 + (int64_t)tin * (CTA / G);
         if (tin < full_tiles)
             fast_tile<BM, BV, G, true, PBF, PLAIN>(a, s, s_y, s_mid, pbase, gbase, 0, tin, jb_tile, tensor, par, ah,
-                                       tin + step < full_tiles && tile + step < tile_end, step);
+                                       tin + step < full_tiles && tile + step < tile_end, step, tile);
         else
             fast_tile<BM, BV, G, false, PBF, PLAIN>(a, s, s_y, s_mid, pbase, gbase, __ldg(a.numel + tensor), tin, jb_tile,
-                                                    tensor, par, ah, false, 0);
+                                                    tensor, par, ah, false, 0, tile);
         par ^= 1;
     }
-    // every copy that was issued has been waited for by the thread that issued it, unless that
-    // thread gave up once: then it waits (bounded) once more for its last copy before the CTA exits
-    if (tid == 0 && ah.failed && ah.fill > 0) {
+    // A thread that gave up on a copy waits once more, again bounded, for the last one that was issued,
+    // so that no copy is still writing to a stage when the CTA's shared memory is released.
+    if (ah.failed && ah.fill > 0) {
         const uint32_t last = ah.fill - 1u;
         mbar_wait(smem_u32(&s.mbar[last & 1u]), (last >> 1) & 1u);
     }

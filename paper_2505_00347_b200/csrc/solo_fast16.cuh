@@ -9,6 +9,21 @@
 // addressing, the level tables, the exchange with the first warp, the rounds of the selection)
 // is spent once per sixteen elements instead of once per eight.
 //
+// Resources are cut for seven resident CTAs per SM (28 warps): at most 72 registers per thread
+// and one input stage of 13.6 KB (21.5 KB of shared memory in all).  The stage is read only
+// before the tile's first CTA barrier, so the copies of the CTA's next tile are issued right after
+// that barrier and land while the tile's second half (per-block scalars, random draws,
+// quantization) runs.  Parameters stay in the stage until the update of their four elements needs
+// them.
+//
+// Shared-memory banks: a thread's sixteen parameters are 64 consecutive bytes of the staged tile, so
+// the eight lanes that one 128-bit shared-memory access serves hit only two groups of four banks (a
+// four-way conflict; gradients, 32 bytes per thread: two-way).  Lanes 4..7 of every group of eight
+// therefore take the two halves of their sixteen elements in the other order (`sw`): their accesses
+// fall on the other banks, which halves the conflicts of the parameters and removes those of the
+// gradients.  Everything that is tied to an element's position (its codes, its Philox draw, where
+// its parameter is stored) follows the swap; nothing else depends on the order.
+//
 // This kernel processes full tiles of 16-byte aligned tensors only; every other tile is left to
 // a second launch of solo_step_fast_kernel with StepArgs::only_partial set.
 #pragma once
@@ -21,30 +36,36 @@ namespace solo {
 constexpr int EPT16 = 16;               // elements per thread
 static_assert(CTA16 * EPT16 == TILE, "same tile as the other kernels");
 
-template <int BM, int BV>
+#ifndef SOLO_F16_CTAS
+#define SOLO_F16_CTAS 7                 // resident CTAs per SM the fp32 kernel is compiled for
+#endif
+
+template <int BM, int BV, bool PBF>
 struct Fast16Shared {
     // Sorted keys of the threads, one column per thread: row j holds the (j+2)-th smallest key.
     // Twelve rounds of popping read rows 0..11 at most.
     uint32_t sort[12][CTA16];
-    float tab[16][(1 << BV) + (1 << BM)]; // per block: K_v second-moment levels, then K_m first-moment levels
+    // per block: K_v second-moment levels alpha^k Delta_v and K_m first-moment levels y_k Delta_m.
+    // Two arrays, so that the four blocks of a warp occupy distinct banks (up to eight levels).
+    float tab_v[16][1 << BV];
+    float tab_m[16][1 << BM];
     // Exchange with the first warp.  One copy is enough: xin is written before the tile's first
-    // barrier and read between its two barriers, xout and xflag are written between the barriers and
-    // read after the second, and nobody writes either again before passing those barriers.
-    uint4 xin[16];                       // per block: bits of Delta_m', Delta_v', x_p
-    float4 xout[16];                     // per block: 1/Delta_m', 1/Delta_v', 1/log2(alpha'), rounding limit
-    uint32_t xflag[16];
+    // barrier and read between its two barriers, xout is written between the barriers and read
+    // after the second, and nobody writes either again before passing those barriers.
+    uint4 xin[16];                       // per block: bits of Delta_m', Delta_v', x_p; .w != 0: the block's warp skips the tile
+    float4 xout[16];                     // per block: vanishing Delta_v' (1 or 0), 1/Delta_v', 1/log2(alpha'), rounding limit
     // per 3-bit moment and warp: the packed codes of the warp's 512 elements, for 128-bit stores
     static constexpr int N3 = (BM == 3 ? 1 : 0) + (BV == 3 ? 1 : 0);
     alignas(16) uint32_t cout[N3 > 0 ? N3 : 1][N3 > 0 ? 4 : 1][N3 > 0 ? 48 : 4];   // (a token array without 3-bit codes)
     struct Stage {
-        float4 p[TILE / 4];              // 2048 parameters (bf16: the first half)
-        uint4 g[TILE / 8];               // 2048 bf16 gradients
+        alignas(16) unsigned char p[TILE * (PBF ? 2 : 4)];   // 2048 parameters
+        alignas(16) unsigned char g[TILE * 2];                // 2048 bf16 gradients
         uint32_t cm[64 * BM + 4];        // packed codes of the tile: 256 * bits bytes
         uint32_t cv[64 * BV + 4];
         float sc[3][16 + 4];             // Delta_m, Delta_v, alpha of the 16 blocks, from a 16-byte boundary
     };
-    alignas(16) Stage stage[2];
-    alignas(8) unsigned long long mbar[2];
+    alignas(16) Stage stage;
+    alignas(8) unsigned long long mbar;
 };
 
 __device__ __forceinline__ void bar_sync16(int id) {
@@ -64,22 +85,24 @@ struct CodeOffsets16x2 {
 };
 
 // The thread's sixteen BITS-bit codes as two words of eight codes each, from the tile's staged
-// code words (thread t owns bytes [2 * BITS * t, 2 * BITS * (t + 1)) of them).
+// code words (thread t owns bytes [2 * BITS * t, 2 * BITS * (t + 1)) of them).  sw = 1: the two
+// words are exchanged (h[0] then holds elements 8..15).
 template <int BITS>
-__device__ __forceinline__ void load_codes16(const uint32_t* st, int tid, uint32_t (&h)[2]) {
+__device__ __forceinline__ void load_codes16(const uint32_t* st, int tid, uint32_t sw, uint32_t (&h)[2]) {
     if constexpr (BITS == 2) {
-        const uint32_t c = st[tid];
+        const uint32_t c = __funnelshift_r(st[tid], st[tid], 16u * sw);
         h[0] = c & 0xFFFFu; h[1] = c >> 16;
     } else if constexpr (BITS == 4) {
         const uint2 c = reinterpret_cast<const uint2*>(st)[tid];
-        h[0] = c.x; h[1] = c.y;
+        h[0] = sw ? c.y : c.x; h[1] = sw ? c.x : c.y;
     } else {
         static_assert(BITS == 3, "2, 3 or 4 bits");
         const int cw = (6 * tid) >> 2, cs = ((6 * tid) & 3) * 8;  // 48 bits from byte 6 * tid; cs is 0 or 16
         const uint32_t w0 = st[cw], w1 = st[cw + 1];
         const uint32_t c32 = __funnelshift_r(w0, w1, cs);         // bits 0..31
         const uint32_t c16 = (w1 >> cs) & 0xFFFFu;                // bits 32..47
-        h[0] = c32 & 0xFFFFFFu; h[1] = (c32 >> 24) | (c16 << 8);
+        const uint32_t lo = c32 & 0xFFFFFFu, hi = (c32 >> 24) | (c16 << 8);
+        h[0] = sw ? hi : lo; h[1] = sw ? lo : hi;
     }
 }
 // The reverse, to the tile's codes in global memory (`tile_codes`: their first byte).  3-bit codes
@@ -154,17 +177,20 @@ __device__ __forceinline__ uint32_t pop_round16(uint32_t& head, int& off, const 
     return tgt;
 }
 
-// Bulk copies of one full tile's inputs into stage `fill & 1` (one thread).  With blocks of 128
-// the tile's codes start on 16-byte boundaries (16 * bits bytes per block); the per-block scalars
-// are copied from the boundary at or below the first.
+// Bulk copies of one full tile's inputs into the stage (one thread; a bulk copy is a warp-wide
+// instruction, so copies issued by many lanes would be serialised lane by lane).  With blocks of 128
+// the tile's codes start on 16-byte boundaries (16 * bits bytes per block); the per-block scalars are
+// copied from the boundary at or below the first.
+// `extra_tx`: bytes announced on top of what is copied (test hook: the wait for this tile then runs out).
 template <int BM, int BV, bool PBF>
-__device__ __forceinline__ void issue_tile_copy16(const StepArgs& a, Fast16Shared<BM, BV>& s, uint32_t fill,
-                                                  const char* pt, const char* gt, int64_t jb_tile) {
-    typename Fast16Shared<BM, BV>::Stage& st = s.stage[fill & 1u];
-    const uint32_t bar = smem_u32(&s.mbar[fill & 1u]);
+__device__ __forceinline__ void issue_tile_copy16(const StepArgs& a, Fast16Shared<BM, BV, PBF>& s, const char* pt,
+                                                  const char* gt, int64_t jb_tile, uint32_t extra_tx) {
+    typename Fast16Shared<BM, BV, PBF>::Stage& st = s.stage;
+    const uint32_t bar = smem_u32(&s.mbar);
     const uint32_t bytes_s = (16u + ((jb_tile & 3) ? 4u : 0u)) * 4u;
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar),
-                 "r"((uint32_t)(TILE * (PBF ? 2 : 4) + TILE * 2 + 256 * BM + 256 * BV) + 3u * bytes_s) : "memory");
+                 "r"((uint32_t)(TILE * (PBF ? 2 : 4) + TILE * 2 + 256 * BM + 256 * BV) + 3u * bytes_s + extra_tx)
+                 : "memory");
     bulk_copy(st.p, pt, TILE * (PBF ? 2 : 4), bar);
     bulk_copy(st.g, gt, TILE * 2, bar);
     bulk_copy(st.cm, a.codes_m + jb_tile * (16 * BM), 256 * BM, bar);
@@ -175,216 +201,213 @@ __device__ __forceinline__ void issue_tile_copy16(const StepArgs& a, Fast16Share
     bulk_copy(st.sc[2], a.alpha + j0, bytes_s, bar);
 }
 
-// One full tile.  Arguments as for fast_tile.
-template <int BM, int BV, bool PBF>
-__device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, BV>& s, const float* s_y, const float* s_mid,
+// What a CTA carries from one full tile to the next.
+struct Ahead16 {
+    uint32_t fill = 0;        // number of the next copy to wait for (uniform over the CTA); its parity is the phase
+    bool staged = false;      // that copy has already been issued (uniform)
+    bool failed = false;      // this thread once waited in vain for a copy: it waits no longer and stores nothing
+};
+
+// Per-block scalars of the tile's sixteen blocks (one block per calling thread, tid = 0..15), from
+// what the blocks' lanes left in xin: stores Delta_m', Delta_v', alpha' of the blocks whose warp did not
+// skip the tile and leaves what Eq. 6 needs in xout.
+template <int KV, class Shared>
+__device__ __forceinline__ void block_scalars16(const StepArgs& a, Shared& s, const int64_t jb_tile, const int tid) {
+    const uint4 in = s.xin[tid];
+    const float dm_new = __uint_as_float(in.x), dv_new = __uint_as_float(in.y);
+    const bool zero_m = dm_new < TINY, zero_v = dv_new < TINY;
+    const float inv_dv = 1.0f / dv_new;
+    const float rho = fminf(fmaxf(__uint_as_float(in.z) * inv_dv, RHO_MIN), RHO_MAX);
+    const float lam = log2_sp(rho) * (1.0f / (float)(KV - 1));
+    const float al_new = exp2_sp(lam);
+    const float inv_lambda = 1.0f / log2_sp(al_new);
+    const float guard = __fmaf_rn(fabsf(inv_lambda), LG2_ABS, LG2_REL * (float)(KV + 1));
+    s.xout[tid] = make_float4(zero_v ? 1.0f : 0.0f, inv_dv, inv_lambda, 0.5f - guard);
+    if (in.w == 0u) {
+        const int64_t j = jb_tile + tid;
+        a.scale_m[j] = zero_m ? 0.0f : dm_new;
+        a.scale_v[j] = zero_v ? 0.0f : dv_new;
+        a.alpha[j] = zero_v ? 0.5f : al_new;
+    }
+}
+
+// One full tile.  DECAY: the parameter is multiplied by 1 - lr * wd (false: that factor is 1).
+//
+// Order of the work, chosen so that at most the two moments and the sort keys (48 registers) are
+// live at once: (A) inputs, Eq. 2-3; (B) the parameter update, parameters read from the stage four
+// at a time; (C) the first moment's scale and codes (each thread divides for itself: the scale is
+// known to all eight lanes after the maximum); (D) the sort and the selection rounds, with the Philox
+// rounds of the thread's two blocks of draws issued between them (they depend on nothing); (E) the
+// exchange with the first warp, the second moment's codes, the stores.
+template <int BM, int BV, bool PBF, bool DECAY>
+__device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, BV, PBF>& s, const float* s_y, const float* s_mid,
                                             char* pbase, const char* gbase, const int tin, const int64_t jb_tile,
-                                            const int tensor, Ahead& ah, const bool next_full,
-                                            const int next_dtin) {
+                                            const int tensor, Ahead16& ah, const bool next_full, const int64_t tile_no) {
     constexpr int KM = 1 << BM, KV = 1 << BV, G = 8, NG = 16;     // 8 lanes per block, 16 blocks per tile
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gl = tid & (G - 1), grp = tid >> 3;
+    const uint32_t sw = ((uint32_t)tid >> 2) & 1u;               // 1: this thread takes elements 8..15 first (see the top of the file)
 
     const int64_t tile_elem0 = (int64_t)tin * TILE;
     constexpr int PSZ = PBF ? 2 : 4;                              // bytes per parameter
     char* const pt = pbase + tile_elem0 * PSZ;
     const char* const gt = gbase + tile_elem0 * 2;
 
-    // ---- inputs from the stage (see fast_tile for the protocol) ----
-    if (tid == 0) {
-        if (!ah.staged) issue_tile_copy16<BM, BV, PBF>(a, s, ah.fill, pt, gt, jb_tile);
-        if (next_full)
-            issue_tile_copy16<BM, BV, PBF>(a, s, ah.fill + 1u, pt + (int64_t)next_dtin * (TILE * PSZ),
-                              gt + (int64_t)next_dtin * (TILE * 2), jb_tile + (int64_t)next_dtin * NG);
-    }
+    // ---- (A) inputs from the stage ----
+    // Copy number f completes phase f of the stage's mbarrier (parity f & 1).  The copy for this tile
+    // was issued after the first barrier of the tile before it (ah.staged), or is issued now (the
+    // CTA's first full tile, or the first after a tensor change or a tile that was not full): every
+    // thread has passed both barriers of the last tile that used the stage, so nobody reads it still.
+    if (!ah.staged && tid == 0)
+        issue_tile_copy16<BM, BV, PBF>(a, s, pt, gt, jb_tile, tile_no + 1 == a.debug_stall_tile_p1 ? 16u : 0u);
     const uint32_t mine = ah.fill;
     ah.fill += 1u;
     ah.staged = next_full;
-    if (!mbar_wait(smem_u32(&s.mbar[mine & 1u]), (mine >> 1) & 1u)) {
-        atomicOr(a.status, 2);
+    if (!mbar_wait(smem_u32(&s.mbar), mine & 1u, ah.failed ? 1 : MBAR_POLLS)) {
+        if (!ah.failed) atomicOr(a.status, 2);
         ah.failed = true;
     }
-    const typename Fast16Shared<BM, BV>::Stage& st = s.stage[mine & 1u];
-    float p[EPT16], g[EPT16];
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        const uint4 gw = st.g[2 * tid + h];
-        const uint32_t gg[4] = {gw.x, gw.y, gw.z, gw.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            g[8 * h + 2 * i] = __uint_as_float(gg[i] << 16);
-            g[8 * h + 2 * i + 1] = __uint_as_float(gg[i] & 0xffff0000u);
-        }
+    // A warp in which any lane gave up leaves the tile alone: it stores nothing, flags its four blocks
+    // for the first warp (which stores the per-block scalars), and only keeps the CTA's barriers, the
+    // copy-ahead and, if it is the first warp, the other warps' scalars going.
+    if (__any_sync(0xffffffffu, ah.failed)) {
+        if (gl == 0) s.xin[grp] = make_uint4(0u, 0u, 0u, 1u);
+        bar_sync16(1);
+        if (next_full && tid == 32)
+            issue_tile_copy16<BM, BV, PBF>(a, s, pt + TILE * PSZ, gt + TILE * 2, jb_tile + NG,
+                                           tile_no + 2 == a.debug_stall_tile_p1 ? 16u : 0u);
+        if (tid < NG) block_scalars16<KV>(a, s, jb_tile, tid);
+        bar_sync16(2);
+        return;
     }
-    if constexpr (PBF) {
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const uint4 pw = reinterpret_cast<const uint4*>(st.p)[2 * tid + h];
-            const uint32_t pp[4] = {pw.x, pw.y, pw.z, pw.w};
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                p[8 * h + 2 * i] = __uint_as_float(pp[i] << 16);
-                p[8 * h + 2 * i + 1] = __uint_as_float(pp[i] & 0xffff0000u);
-            }
-        }
-    } else {
-#pragma unroll
-        for (int h = 0; h < 4; ++h) {
-            const float4 pv = st.p[4 * tid + h];
-            p[4 * h] = pv.x; p[4 * h + 1] = pv.y; p[4 * h + 2] = pv.z; p[4 * h + 3] = pv.w;
-        }
-    }
-    uint32_t cm[2], cv[2];                                        // eight codes per word
-    load_codes16<BM>(st.cm, tid, cm);
-    load_codes16<BV>(st.cv, tid, cv);
-    const int so = (int)(jb_tile & 3) + grp;
-    const float dm = st.sc[0][so], dv = st.sc[1][so], al = st.sc[2][so];
 
-    // ---- per-block level tables (Eq. 2), built by the block's eight lanes ----
-    float* const tab = s.tab[grp];
-    {
-        float a2[BV];
-        a2[0] = al;
-#pragma unroll
-        for (int i = 1; i < BV; ++i) a2[i] = a2[i - 1] * a2[i - 1];
-#pragma unroll
-        for (int r0 = 0; r0 < KV; r0 += G) tab[r0 + gl] = pow_sm<BV>(a2, (uint32_t)(r0 + gl)) * dv;
-#pragma unroll
-        for (int r0 = 0; r0 < KM; r0 += G)
-            if (r0 + gl < KM) tab[KV + r0 + gl] = s_y[r0 + gl] * dm;
-    }
-    __syncwarp();
-
-    // ---- Eq. 2, Eq. 3 ----
+    const typename Fast16Shared<BM, BV, PBF>::Stage& st = s.stage;
     float mh[EPT16], vh[EPT16];
     uint32_t mx_v = 0;
     float mx_m_f = 0.0f;
-    const char* const tab_v = reinterpret_cast<const char*>(tab);
-    const char* const tab_m = reinterpret_cast<const char*>(tab + KV);
-    const CodeOffsets16x2 om16(cm[0] | (cm[1] << 16));            // used for 2-bit codes only
-    const CodeOffsets<BM> om4a(cm[0], 0u), om4b(cm[1], 0u);
-    const CodeOffsets<BV> ov4a(cv[0], 0u), ov4b(cv[1], 0u);
-#pragma unroll
-    for (int i = 0; i < EPT16; ++i) {
-        const float mt = *reinterpret_cast<const float*>(tab_m + (BM == 2 ? om16(i) : i < 8 ? om4a(i) : om4b(i - 8)));
-        const float vt = *reinterpret_cast<const float*>(tab_v + (i < 8 ? ov4a(i) : ov4b(i - 8)));
-        const float gi = g[i];
-        mh[i] = __fmaf_rn(a.beta1, mt, a.omb1 * gi);
-        vh[i] = __fmaf_rn(a.beta2, vt, a.omb2 * (gi * gi));
-        mx_m_f = fmaxf(mx_m_f, fabsf(mh[i]));
-        mx_v = max(mx_v, __float_as_uint(vh[i]));
-    }
-    uint32_t mx_m = __float_as_uint(mx_m_f);
-
-    // Adam(W) update of element i; fp32 parameters are stored after every fourth.  bf16 parameters:
-    // IEEE square root and division (see solo_fast.cuh), stored after every eighth, rounded to
-    // nearest even or with the element's Philox draw (purpose 2, one block per eight elements)
-    const uint64_t ctr = ((uint64_t)(uint32_t)tin * (TILE / 8)) + 2u * (uint32_t)tid;   // element index / 8
-    auto update = [&](int i) {
-        if constexpr (PBF) {
-            const float den = __fmaf_rn(__fsqrt_rn(vh[i]), a.inv_sqrt_bc2, a.eps);
-            p[i] = __fmaf_rn(-a.step_size, __fdiv_rn(mh[i], den), p[i] * a.decay);
-            if ((i & 7) == 7) {
-                const int b = i - 7;
-                uint32_t pp[4];
-                if (a.param_sr) {
-                    uint32_t wp[4];
-                    const uint64_t c = ctr + (uint64_t)(i >> 3);
-                    philox_rk((uint32_t)c, (uint32_t)(c >> 32), a.step32, (uint32_t)tensor * 4u + 2u, a.rk, wp);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        pp[j] = bf16_sr(p[b + 2 * j], wp[j] & 0xFFFFu) | (bf16_sr(p[b + 2 * j + 1], wp[j] >> 16) << 16);
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const __nv_bfloat162 h2 = __floats2bfloat162_rn(p[b + 2 * j], p[b + 2 * j + 1]);
-                        pp[j] = *reinterpret_cast<const uint32_t*>(&h2);
-                    }
-                }
-                __stcs(reinterpret_cast<uint4*>(pt) + 2 * tid + (i >> 3), make_uint4(pp[0], pp[1], pp[2], pp[3]));
-            }
-            return;
-        }
-        const float den = __fmaf_rn(sqrt_approx(vh[i]), a.inv_sqrt_bc2, a.eps);
-        const float rc = rcp_approx(den);
-        const float q0 = mh[i] * rc;
-        const float q1 = __fmaf_rn(__fmaf_rn(-den, q0, mh[i]), rc, q0);
-        p[i] = __fmaf_rn(-a.step_size, q1, p[i] * a.decay);
-        if ((i & 3) == 3)
-            __stcs(reinterpret_cast<float4*>(pt) + 4 * tid + (i >> 2), make_float4(p[i - 3], p[i - 2], p[i - 1], p[i]));
-    };
-    auto update2 = [&](int r) { update(2 * r); update(2 * r + 1); };
-
-    // ---- block scales and the p-quantile (k = 13 of 128) ----
-    mx_m = group8_max(mx_m);
-    mx_v = group8_max(mx_v);
-    uint32_t x_p;
     {
-        uint32_t key[EPT16];
+        uint32_t cm[2], cv[2];                                    // eight codes per word
+        load_codes16<BM>(st.cm, tid, sw, cm);
+        load_codes16<BV>(st.cv, tid, sw, cv);
+        const int so = (int)(jb_tile & 3) + grp;
+        const float dm = st.sc[0][so], dv = st.sc[1][so], al = st.sc[2][so];
+
+        // per-block level tables (Eq. 2), built by the block's eight lanes
+        float* const tab_vf = s.tab_v[grp];
+        float* const tab_mf = s.tab_m[grp];
+        {
+            float a2[BV];
+            a2[0] = al;
 #pragma unroll
-        for (int i = 0; i < EPT16; ++i) key[i] = __float_as_uint(vh[i]);
-        sort16_low13(key);
-        uint32_t* const col = &s.sort[0][tid];
+            for (int i = 1; i < BV; ++i) a2[i] = a2[i - 1] * a2[i - 1];
 #pragma unroll
-        for (int j = 1; j <= 12; ++j) col[(j - 1) * CTA16] = key[j];
-        // twelve rounds pop the twelve smallest keys of the block, the thirteenth minimum is x_p;
-        // the parameter updates are issued between the rounds
-        const uint32_t self = 1u << lane;
-        const uint32_t le = (self | (self - 1u)) & (0xFFu << (lane & ~(G - 1)));
-        uint32_t head = key[0];
-        int off = 0;
+            for (int r0 = 0; r0 < KV; r0 += G)
+                if (r0 + gl < KV) tab_vf[r0 + gl] = pow_sm<BV>(a2, (uint32_t)(r0 + gl)) * dv;
 #pragma unroll
-        for (int r = 0; r < 12; ++r) {
-            pop_round16<false>(head, off, col, le, self);
-            if (r < 8) update2(r);
+            for (int r0 = 0; r0 < KM; r0 += G)
+                if (r0 + gl < KM) tab_mf[r0 + gl] = s_y[r0 + gl] * dm;
         }
-        x_p = pop_round16<true>(head, off, col, le, self);
+        __syncwarp();
+
+        // Eq. 2, Eq. 3
+        const char* const tab_v = reinterpret_cast<const char*>(tab_vf);
+        const char* const tab_m = reinterpret_cast<const char*>(tab_mf);
+        const CodeOffsets16x2 om16(cm[0] | (cm[1] << 16));        // used for 2-bit codes only
+        const CodeOffsets<BM> om4a(cm[0], 0u), om4b(cm[1], 0u);
+        const CodeOffsets<BV> ov4a(cv[0], 0u), ov4b(cv[1], 0u);
+        const unsigned char* const sgb = st.g + 32 * tid;
+        const uint4* const sg[2] = {reinterpret_cast<const uint4*>(sgb + 16u * sw),
+                                    reinterpret_cast<const uint4*>(sgb + 16u - 16u * sw)};
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint4 gw = *sg[h];
+            const uint32_t gg[4] = {gw.x, gw.y, gw.z, gw.w};
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int i = 8 * h + k;
+                const float gi = __uint_as_float((k & 1) ? (gg[k >> 1] & 0xffff0000u) : (gg[k >> 1] << 16));
+                const float mt = *reinterpret_cast<const float*>(tab_m + (BM == 2 ? om16(i) : i < 8 ? om4a(i) : om4b(i - 8)));
+                const float vt = *reinterpret_cast<const float*>(tab_v + (i < 8 ? ov4a(i) : ov4b(i - 8)));
+                mh[i] = __fmaf_rn(a.beta1, mt, a.omb1 * gi);
+                vh[i] = __fmaf_rn(a.beta2, vt, a.omb2 * (gi * gi));
+                mx_m_f = max_abs_nan(mx_m_f, mh[i]);
+                mx_v = max(mx_v, __float_as_uint(vh[i]));
+            }
+        }
     }
 
-    // ---- per-block scalars by the first warp; the others draw xi meanwhile ----
-    if (gl == 0) s.xin[grp] = make_uint4(mx_m, mx_v, x_p, 0u);
-    bar_sync16(1);
-    uint32_t w[8];
-    auto draw = [&]() {
-        uint32_t wa[4], wb[4];
-        philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, (uint32_t)tensor * 4u, a.rk, wa);
-        philox_rk((uint32_t)(ctr + 1), (uint32_t)((ctr + 1) >> 32), a.step32, (uint32_t)tensor * 4u, a.rk, wb);
+    // ---- (B) Adam(W) update, four (fp32) or eight (bf16) elements at a time ----
+    // bf16 parameters: IEEE square root and division (see solo_fast.cuh), rounded to nearest even or
+    // with the element's Philox draw (purpose 2, one block per eight elements)
+    const uint32_t ctr_lo = (uint32_t)tin * (TILE / 8) + 2u * (uint32_t)tid;   // element index / 8: even, below 2^32
+    if constexpr (!PBF) {
+        // the thread's first eight elements (in its own order) at `sp[0]`, the others at `sp[1]`
+        const unsigned char* const spb = st.p + 64 * tid;
+        char* const gpb = pt + 64 * tid;
+        const float4* const sp[2] = {reinterpret_cast<const float4*>(spb + 32u * sw),
+                                     reinterpret_cast<const float4*>(spb + 32u - 32u * sw)};
+        float4* const gp[2] = {reinterpret_cast<float4*>(gpb + 32u * sw), reinterpret_cast<float4*>(gpb + 32u - 32u * sw)};
 #pragma unroll
-        for (int i = 0; i < 4; ++i) { w[i] = wa[i]; w[4 + i] = wb[i]; }
-    };
-    if (warp != 0) {
-        draw();
-    } else if (tid < NG) {
-        const uint4 in = s.xin[tid];
-        const float dm_new = __uint_as_float(in.x), dv_new = __uint_as_float(in.y);
-        const bool zero_m = dm_new < TINY, zero_v = dv_new < TINY;
-        const float inv_dm = 1.0f / dm_new;
-        const float inv_dv = 1.0f / dv_new;
-        const float rho = fminf(fmaxf(__uint_as_float(in.z) * inv_dv, RHO_MIN), RHO_MAX);
-        const float lam = log2_sp(rho) * (1.0f / (float)(KV - 1));
-        const float al_new = exp2_sp(lam);
-        const float inv_lambda = 1.0f / log2_sp(al_new);
-        const float guard = __fmaf_rn(fabsf(inv_lambda), LG2_ABS, LG2_REL * (float)(KV + 1));
-        s.xout[tid] = make_float4(inv_dm, inv_dv, inv_lambda, 0.5f - guard);
-        s.xflag[tid] = (zero_m ? 1u : 0u) | (zero_v ? 2u : 0u);
-        const int64_t j = jb_tile + tid;
-        a.scale_m[j] = zero_m ? 0.0f : dm_new;
-        a.scale_v[j] = zero_v ? 0.0f : dv_new;
-        a.alpha[j] = zero_v ? 0.5f : al_new;
+        for (int q = 0; q < 4; ++q) {
+            const float4 pv = sp[q >> 1][q & 1];
+            float p[4] = {pv.x, pv.y, pv.z, pv.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int i = 4 * q + k;
+                const float den = __fmaf_rn(sqrt_approx(vh[i]), a.inv_sqrt_bc2, a.eps);
+                const float rc = rcp_approx(den);
+                const float q0 = mh[i] * rc;
+                const float q1 = __fmaf_rn(__fmaf_rn(-den, q0, mh[i]), rc, q0);
+                p[k] = __fmaf_rn(-a.step_size, q1, DECAY ? p[k] * a.decay : p[k]);
+            }
+            __stcs(gp[q >> 1] + (q & 1), make_float4(p[0], p[1], p[2], p[3]));
+        }
+    } else {
+        const uint4* const sp = reinterpret_cast<const uint4*>(st.p) + 2 * tid;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t he = (uint32_t)h ^ sw;
+            const uint4 pw = sp[he];
+            const uint32_t pin[4] = {pw.x, pw.y, pw.z, pw.w};
+            float p[8];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                p[2 * k] = __uint_as_float(pin[k] << 16);
+                p[2 * k + 1] = __uint_as_float(pin[k] & 0xffff0000u);
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int i = 8 * h + k;
+                const float den = __fmaf_rn(__fsqrt_rn(vh[i]), a.inv_sqrt_bc2, a.eps);
+                p[k] = __fmaf_rn(-a.step_size, __fdiv_rn(mh[i], den), DECAY ? p[k] * a.decay : p[k]);
+            }
+            uint32_t pp[4];
+            if (a.param_sr) {
+                uint32_t wp[4];
+                philox_rk(ctr_lo + he, 0u, a.step32, (uint32_t)tensor * 4u + 2u, a.rk, wp);
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    pp[k] = bf16_sr(p[2 * k], wp[k] & 0xFFFFu) | (bf16_sr(p[2 * k + 1], wp[k] >> 16) << 16);
+            } else {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const __nv_bfloat162 h2 = __floats2bfloat162_rn(p[2 * k], p[2 * k + 1]);
+                    pp[k] = *reinterpret_cast<const uint32_t*>(&h2);
+                }
+            }
+            __stcs(reinterpret_cast<uint4*>(pt) + 2 * tid + he, make_uint4(pp[0], pp[1], pp[2], pp[3]));
+        }
     }
-    bar_sync16(2);
-    if (warp == 0) draw();
-    float dr[EPT16];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) halves_to_float(w[i], dr[2 * i], dr[2 * i + 1]);
-    const float4 sc = s.xout[grp];
-    const uint32_t zf = s.xflag[grp];
 
-    // ---- first moment: nearest level (Eq. 1), see fast_tile ----
+    // ---- (C) first moment: block scale, nearest level (Eq. 1), see fast_tile ----
+    const uint32_t mx_m = group8_max(__float_as_uint(mx_m_f));
     uint32_t om[2] = {0u, 0u};                                    // eight codes per word
     {
-        const float inv = sc.x;
+        const float dm_new = __uint_as_float(mx_m);
+        const float inv = 1.0f / dm_new;
         if constexpr (BM == 2) {
+            // code = number of midpoints below r, each comparison as the saturation of
+            // (r - mid) * 2^100 on the FMA pipe (exactly 0 or 1, see fast_tile)
             constexpr float BIG = 0x1p100f;
             const float n0 = -s_mid[0] * BIG, n1 = -s_mid[1] * BIG, n2 = -s_mid[2] * BIG;
             float omf[2] = {0.0f, 0.0f};
@@ -404,14 +427,71 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
                 const float r = mh[i] * inv;
                 uint32_t q = 0;
 #pragma unroll
-                for (int st = KM / 2; st >= 1; st >>= 1)
-                    if (r > s_mid[q + st - 1]) q += st;
+                for (int st2 = KM / 2; st2 >= 1; st2 >>= 1)
+                    if (r > s_mid[q + st2 - 1]) q += st2;
                 om[i >> 3] = (om[i >> 3] << BM) + q;
             }
         }
+        if (dm_new < TINY) { om[0] = 0; om[1] = 0; }             // vanishing block: all codes 0
     }
 
-    // ---- second moment: Eq. 6, see fast_tile ----
+    // ---- (D) second moment: block scale and the p-quantile (k = 13 of 128); the draws of Eq. 6 ----
+    mx_v = group8_max(mx_v);
+    uint32_t x_p;
+    uint32_t w[8];                                                // 16 halfwords: the draws of the 16 elements
+    {
+        // Philox4x32-10 on the counters of the thread's two groups of eight elements,
+        // (ctr_lo, 0, step, 4 * tensor) and (ctr_lo + 1, ...), in the thread's order; one round of both per call
+        uint32_t ca[4] = {ctr_lo + sw, 0u, a.step32, (uint32_t)tensor * 4u};
+        uint32_t cb[4] = {ctr_lo + (sw ^ 1u), 0u, a.step32, (uint32_t)tensor * 4u};
+        auto philox_round = [&](int r) {
+#pragma unroll
+            for (int b = 0; b < 2; ++b) {
+                uint32_t(&c)[4] = b ? cb : ca;
+                const uint64_t p0 = (uint64_t)0xD2511F53u * c[0];
+                const uint64_t p1 = (uint64_t)0xCD9E8D57u * c[2];
+                const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c[1] ^ a.rk[2 * r];
+                const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c[3] ^ a.rk[2 * r + 1];
+                c[1] = (uint32_t)p1;
+                c[3] = (uint32_t)p0;
+                c[0] = n0;
+                c[2] = n2;
+            }
+        };
+        uint32_t key[EPT16];
+#pragma unroll
+        for (int i = 0; i < EPT16; ++i) key[i] = __float_as_uint(vh[i]);
+        sort16_low13(key);
+        uint32_t* const col = &s.sort[0][tid];
+#pragma unroll
+        for (int j = 1; j <= 12; ++j) col[(j - 1) * CTA16] = key[j];
+        // twelve rounds pop the twelve smallest keys of the block, the thirteenth minimum is x_p
+        const uint32_t self = 1u << lane;
+        const uint32_t le = (self | (self - 1u)) & (0xFFu << (lane & ~(G - 1)));
+        uint32_t head = key[0];
+        int off = 0;
+#pragma unroll
+        for (int r = 0; r < 12; ++r) {
+            pop_round16<false>(head, off, col, le, self);
+            if (r < 10) philox_round(r);
+        }
+        x_p = pop_round16<true>(head, off, col, le, self);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { w[i] = ca[i]; w[4 + i] = cb[i]; }
+    }
+
+    // ---- (E) per-block scalars by the first warp; the next tile's copies start meanwhile ----
+    if (gl == 0) s.xin[grp] = make_uint4(mx_m, mx_v, x_p, 0u);
+    bar_sync16(1);
+    // every thread has read what it needs from the stage
+    if (next_full && tid == 32)
+        issue_tile_copy16<BM, BV, PBF>(a, s, pt + TILE * PSZ, gt + TILE * 2, jb_tile + NG,
+                                       tile_no + 2 == a.debug_stall_tile_p1 ? 16u : 0u);
+    if (tid < NG) block_scalars16<KV>(a, s, jb_tile, tid);
+    bar_sync16(2);
+    const float4 sc = s.xout[grp];
+
+    // second moment: Eq. 6, see fast_tile
     uint32_t ov[2];
     {
         const float inv = sc.y, il = sc.z, lim = sc.w;
@@ -424,12 +504,18 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
         float worst = 0.0f;
         uint32_t acc[2] = {0u, 0u};
 #pragma unroll
-        for (int i = EPT16 - 1; i >= 0; --i) {
-            const float r = vh[i] * inv;
-            const float ts = __saturatef(__fmaf_rn(lg2_approx(r), ils, __fmaf_rn(dr[i], xs1, xs0)));
-            const float u = __fmaf_rn(ts, KM1, MAGIC);
-            worst = fmaxf(worst, fabsf(__fmaf_rn(ts, KM1, MAGIC - u)));
-            acc[i >> 3] = acc[i >> 3] * (1u << BV) + __float_as_uint(u);
+        for (int j = EPT16 / 2 - 1; j >= 0; --j) {
+            float d[2];                                           // the 16-bit draws of elements 2j, 2j + 1 as binary32
+            halves_to_float(w[j], d[0], d[1]);
+#pragma unroll
+            for (int e = 1; e >= 0; --e) {
+                const int i = 2 * j + e;
+                const float r = vh[i] * inv;
+                const float ts = __saturatef(__fmaf_rn(lg2_approx(r), ils, __fmaf_rn(d[e], xs1, xs0)));
+                const float u = __fmaf_rn(ts, KM1, MAGIC);
+                worst = fmaxf(worst, fabsf(__fmaf_rn(ts, KM1, MAGIC - u)));
+                acc[i >> 3] = acc[i >> 3] * (1u << BV) + __float_as_uint(u);
+            }
         }
         uint32_t magic_sum = 0;
 #pragma unroll
@@ -443,31 +529,38 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
             ov[0] = 0;
             ov[1] = 0;
 #pragma unroll
-            for (int i = EPT16 - 1; i >= 0; --i) {
-                const float r = vh[i] * inv;
-                uint32_t q = KV - 1;
-                if (!(r < TINY)) {
-                    float t = __fmaf_rn(log2_sp(r), il, __fmaf_rn(dr[i], x1, x0));
-                    t = fminf(fmaxf(t, 0.0f), KM1);
-                    q = (uint32_t)__float2int_rn(t);
+            for (int j = EPT16 / 2 - 1; j >= 0; --j) {
+                float d[2];
+                halves_to_float(w[j], d[0], d[1]);
+#pragma unroll
+                for (int e = 1; e >= 0; --e) {
+                    const int i = 2 * j + e;
+                    const float r = vh[i] * inv;
+                    uint32_t q = KV - 1;
+                    if (!(r < TINY)) {
+                        float t = __fmaf_rn(log2_sp(r), il, __fmaf_rn(d[e], x1, x0));
+                        t = fminf(fmaxf(t, 0.0f), KM1);
+                        q = (uint32_t)__float2int_rn(t);
+                    }
+                    ov[i >> 3] = (ov[i >> 3] << BV) + q;
                 }
-                ov[i >> 3] = (ov[i >> 3] << BV) + q;
             }
         }
+        if (sc.x != 0.0f) { ov[0] = 0; ov[1] = 0; }              // vanishing block: all codes 0
     }
-    if (zf & 1u) { om[0] = 0; om[1] = 0; }
-    if (zf & 2u) { ov[0] = 0; ov[1] = 0; }
 
     // ---- store the codes ----
-    store_codes16<BM>(a.codes_m + jb_tile * (16 * BM), s.cout[0][BM == 3 ? warp : 0], tid, om);
-    store_codes16<BV>(a.codes_v + jb_tile * (16 * BV), s.cout[(BM == 3 && BV == 3) ? 1 : 0][BV == 3 ? warp : 0], tid, ov);
+    const uint32_t om_e[2] = {sw ? om[1] : om[0], sw ? om[0] : om[1]};      // back to element order
+    const uint32_t ov_e[2] = {sw ? ov[1] : ov[0], sw ? ov[0] : ov[1]};
+    store_codes16<BM>(a.codes_m + jb_tile * (16 * BM), s.cout[0][BM == 3 ? warp : 0], tid, om_e);
+    store_codes16<BV>(a.codes_v + jb_tile * (16 * BV), s.cout[(BM == 3 && BV == 3) ? 1 : 0][BV == 3 ? warp : 0], tid, ov_e);
 }
 
 template <int BM, int BV, bool PBF>
-__global__ void __launch_bounds__(CTA16, PBF ? 5 : 6) solo_step_fast16_kernel(const StepArgs a) {
+__global__ void __launch_bounds__(CTA16, (PBF || BM != 2) ? 6 : SOLO_F16_CTAS) solo_step_fast16_kernel(const StepArgs a) {
     constexpr int KM = 1 << BM;
     extern __shared__ __align__(16) unsigned char fast16_smem[];
-    Fast16Shared<BM, BV>& s = *reinterpret_cast<Fast16Shared<BM, BV>*>(fast16_smem);
+    Fast16Shared<BM, BV, PBF>& s = *reinterpret_cast<Fast16Shared<BM, BV, PBF>*>(fast16_smem);
     __shared__ float s_y[KM];
     __shared__ float s_mid[KM];
     const int tid = threadIdx.x;
@@ -476,8 +569,7 @@ __global__ void __launch_bounds__(CTA16, PBF ? 5 : 6) solo_step_fast16_kernel(co
         if (tid < KM - 1) s_mid[tid] = a.tables[KM + tid];
     }
     if (tid == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s.mbar[0])) : "memory");
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s.mbar[1])) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s.mbar)) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -494,7 +586,8 @@ __global__ void __launch_bounds__(CTA16, PBF ? 5 : 6) solo_step_fast16_kernel(co
     char* pbase = nullptr;
     const char* gbase = nullptr;
     bool skip = false;
-    Ahead ah;
+    Ahead16 ah;
+    const bool decay = a.decay != 1.0f;
     for (int tile = tile_begin; tile < tile_end; ++tile) {
         if (tile >= t_hi) {
             do {
@@ -512,13 +605,15 @@ __global__ void __launch_bounds__(CTA16, PBF ? 5 : 6) solo_step_fast16_kernel(co
         }
         const int tin = tile - t_lo;
         if (skip || tin >= full_tiles) continue;
-        fast16_tile<BM, BV, PBF>(a, s, s_y, s_mid, pbase, gbase, tin, jb0 + (int64_t)tin * 16, tensor, ah,
-                    tin + 1 < full_tiles && tile + 1 < tile_end, 1);
+        const bool next_full = tin + 1 < full_tiles && tile + 1 < tile_end;
+        if (decay)
+            fast16_tile<BM, BV, PBF, true>(a, s, s_y, s_mid, pbase, gbase, tin, jb0 + (int64_t)tin * 16, tensor, ah, next_full, tile);
+        else
+            fast16_tile<BM, BV, PBF, false>(a, s, s_y, s_mid, pbase, gbase, tin, jb0 + (int64_t)tin * 16, tensor, ah, next_full, tile);
     }
-    if (tid == 0 && ah.failed && ah.fill > 0) {
-        const uint32_t last = ah.fill - 1u;
-        mbar_wait(smem_u32(&s.mbar[last & 1u]), (last >> 1) & 1u);
-    }
+    // A thread that gave up on a copy waits once more, again bounded, for the last one that was issued,
+    // so that no copy is still writing to the stage when the CTA's shared memory is released.
+    if (ah.failed && ah.fill > 0) mbar_wait(smem_u32(&s.mbar), (ah.fill - 1u) & 1u);
 }
 
 }  // namespace solo

@@ -22,16 +22,16 @@ StepKernel fast16_kernel(int bits_m, int bits_v, bool param_bf16) {
     }
 }
 
-size_t fast16_kernel_smem(int bits_m, int bits_v) {
+size_t fast16_kernel_smem(int bits_m, int bits_v, bool param_bf16) {
     switch (bits_m * 10 + bits_v) {
-        case 22: return sizeof(Fast16Shared<2, 2>);
-        case 23: return sizeof(Fast16Shared<2, 3>);
-        case 24: return sizeof(Fast16Shared<2, 4>);
-        case 32: return sizeof(Fast16Shared<3, 2>);
-        case 33: return sizeof(Fast16Shared<3, 3>);
-        case 34: return sizeof(Fast16Shared<3, 4>);
-        case 42: return sizeof(Fast16Shared<4, 2>);
-        case 43: return sizeof(Fast16Shared<4, 3>);
+        case 22: return param_bf16 ? sizeof(Fast16Shared<2, 2, true>) : sizeof(Fast16Shared<2, 2, false>);
+        case 23: return param_bf16 ? sizeof(Fast16Shared<2, 3, true>) : sizeof(Fast16Shared<2, 3, false>);
+        case 24: return param_bf16 ? sizeof(Fast16Shared<2, 4, true>) : sizeof(Fast16Shared<2, 4, false>);
+        case 32: return param_bf16 ? sizeof(Fast16Shared<3, 2, true>) : sizeof(Fast16Shared<3, 2, false>);
+        case 33: return param_bf16 ? sizeof(Fast16Shared<3, 3, true>) : sizeof(Fast16Shared<3, 3, false>);
+        case 34: return param_bf16 ? sizeof(Fast16Shared<3, 4, true>) : sizeof(Fast16Shared<3, 4, false>);
+        case 42: return param_bf16 ? sizeof(Fast16Shared<4, 2, true>) : sizeof(Fast16Shared<4, 2, false>);
+        case 43: return param_bf16 ? sizeof(Fast16Shared<4, 3, true>) : sizeof(Fast16Shared<4, 3, false>);
         default: return 0;
     }
 }
