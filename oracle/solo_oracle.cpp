@@ -122,7 +122,11 @@ int build_codebook(int kind, int bits, float* levels) {
 
 // log2(x) for normal x > 0.  x = 2^e * m with m in [sqrt(1/2), sqrt(2));
 // log2(m) = f * P(f), f = m - 1, P of degree 8 evaluated by Horner with fma.
+// A NaN is returned as it is (the bit operations below would turn it into a
+// number that depends on its sign and payload): in Eq. 6 the clamp then takes the
+// unordered value to code 0, whatever produced the NaN.
 float log2_sp(float x) {
+    if (x != x) return x;
     static const float c[9] = {
         0x1.715476p+0f, -0x1.71547p-1f, 0x1.ec73d6p-2f, -0x1.715c4ep-2f, 0x1.26d384p-2f,
         -0x1.e95be6p-3f, 0x1.b9c91ap-3f, -0x1.a87d0ep-3f, 0x1.01b6dep-3f};

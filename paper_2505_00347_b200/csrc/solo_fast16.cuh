@@ -36,6 +36,9 @@ namespace solo {
 constexpr int EPT16 = 16;               // elements per thread
 static_assert(CTA16 * EPT16 == TILE, "same tile as the other kernels");
 
+#ifndef SOLO_F16_MIX
+#define SOLO_F16_MIX 1                  // 1: the first moment's codes are computed between the exchanges of the sort
+#endif
 #ifndef SOLO_F16_CTAS
 #define SOLO_F16_CTAS 7                 // resident CTAs per SM the fp32 kernel is compiled for
 #endif
@@ -147,6 +150,16 @@ __device__ __forceinline__ void sort16_low13(uint32_t (&k)[EPT16]) {
 #undef SOLO_CS
 }
 
+// The same network as a list, for callers that issue other work between its exchanges.
+__device__ constexpr unsigned char SORT16_PAIRS[62][2] = {
+    {0, 1}, {2, 3}, {0, 2}, {1, 3}, {1, 2}, {4, 5}, {6, 7}, {4, 6}, {5, 7}, {5, 6},
+    {0, 4}, {2, 6}, {2, 4}, {1, 5}, {3, 7}, {3, 5}, {1, 2}, {3, 4}, {5, 6},
+    {8, 9}, {10, 11}, {8, 10}, {9, 11}, {9, 10}, {12, 13}, {14, 15}, {12, 14}, {13, 15}, {13, 14},
+    {8, 12}, {10, 14}, {10, 12}, {9, 13}, {11, 15}, {11, 13}, {9, 10}, {11, 12}, {13, 14},
+    {0, 8}, {4, 12}, {4, 8}, {2, 10}, {6, 14}, {6, 10}, {2, 4}, {6, 8}, {10, 12},
+    {1, 9}, {5, 13}, {5, 9}, {3, 11}, {7, 15}, {7, 11}, {3, 5}, {7, 9}, {11, 13},
+    {1, 2}, {3, 4}, {5, 6}, {7, 8}, {9, 10}, {11, 12}};
+
 // Minimum / maximum over the calling lane's group of eight lanes.  Three shuffle-and-compare steps
 // serve the warp's four groups at once; measured faster here than the full-mask reductions over a
 // transformed value that solo_fast.cuh uses for its groups of sixteen (four REDUX plus selects for
@@ -216,11 +229,11 @@ __device__ __forceinline__ void block_scalars16(const StepArgs& a, Shared& s, co
     const uint4 in = s.xin[tid];
     const float dm_new = __uint_as_float(in.x), dv_new = __uint_as_float(in.y);
     const bool zero_m = dm_new < TINY, zero_v = dv_new < TINY;
-    const float inv_dv = 1.0f / dv_new;
+    const float inv_dv = __frcp_rn(dv_new);
     const float rho = fminf(fmaxf(__uint_as_float(in.z) * inv_dv, RHO_MIN), RHO_MAX);
     const float lam = log2_sp(rho) * (1.0f / (float)(KV - 1));
     const float al_new = exp2_sp(lam);
-    const float inv_lambda = 1.0f / log2_sp(al_new);
+    const float inv_lambda = __frcp_rn(log2_sp(al_new));
     const float guard = __fmaf_rn(fabsf(inv_lambda), LG2_ABS, LG2_REL * (float)(KV + 1));
     s.xout[tid] = make_float4(zero_v ? 1.0f : 0.0f, inv_dv, inv_lambda, 0.5f - guard);
     if (in.w == 0u) {
@@ -402,37 +415,39 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     // ---- (C) first moment: block scale, nearest level (Eq. 1), see fast_tile ----
     const uint32_t mx_m = group8_max(__float_as_uint(mx_m_f));
     uint32_t om[2] = {0u, 0u};                                    // eight codes per word
-    {
-        const float dm_new = __uint_as_float(mx_m);
-        const float inv = 1.0f / dm_new;
+    const float dm_new = __uint_as_float(mx_m);
+    const float inv_m = __frcp_rn(dm_new);
+    // BM == 2: code = number of midpoints below r, each comparison as the saturation of
+    // (r - mid) * 2^100 on the FMA pipe (exactly 0 or 1, see fast_tile), accumulated in binary32
+    constexpr float BIG = 0x1p100f;
+    const float n0 = -s_mid[0] * BIG, n1 = -s_mid[1] * BIG, n2 = -s_mid[BM == 2 ? 2 : 1] * BIG;
+    float omf[2] = {0.0f, 0.0f};
+    auto quant_m = [&](int i) {                                   // call with i = 15, 14, ..., 0
+        const float r = mh[i] * inv_m;
         if constexpr (BM == 2) {
-            // code = number of midpoints below r, each comparison as the saturation of
-            // (r - mid) * 2^100 on the FMA pipe (exactly 0 or 1, see fast_tile)
-            constexpr float BIG = 0x1p100f;
-            const float n0 = -s_mid[0] * BIG, n1 = -s_mid[1] * BIG, n2 = -s_mid[2] * BIG;
-            float omf[2] = {0.0f, 0.0f};
+            float& acc = omf[i >> 3];
+            acc = __fmaf_rn(acc, 4.0f, __saturatef(__fmaf_rn(r, BIG, n0)));
+            acc += __saturatef(__fmaf_rn(r, BIG, n1));
+            acc += __saturatef(__fmaf_rn(r, BIG, n2));
+        } else {
+            uint32_t q = 0;
 #pragma unroll
-            for (int i = EPT16 - 1; i >= 0; --i) {
-                const float r = mh[i] * inv;
-                float& acc = omf[i >> 3];
-                acc = __fmaf_rn(acc, 4.0f, __saturatef(__fmaf_rn(r, BIG, n0)));
-                acc += __saturatef(__fmaf_rn(r, BIG, n1));
-                acc += __saturatef(__fmaf_rn(r, BIG, n2));
-            }
+            for (int st2 = KM / 2; st2 >= 1; st2 >>= 1)
+                if (r > s_mid[q + st2 - 1]) q += st2;
+            om[i >> 3] = (om[i >> 3] << BM) + q;
+        }
+    };
+    auto quant_m_done = [&]() {
+        if constexpr (BM == 2) {
             om[0] = (uint32_t)omf[0];
             om[1] = (uint32_t)omf[1];
-        } else {
-#pragma unroll
-            for (int i = EPT16 - 1; i >= 0; --i) {
-                const float r = mh[i] * inv;
-                uint32_t q = 0;
-#pragma unroll
-                for (int st2 = KM / 2; st2 >= 1; st2 >>= 1)
-                    if (r > s_mid[q + st2 - 1]) q += st2;
-                om[i >> 3] = (om[i >> 3] << BM) + q;
-            }
         }
         if (dm_new < TINY) { om[0] = 0; om[1] = 0; }             // vanishing block: all codes 0
+    };
+    if constexpr (!SOLO_F16_MIX) {
+#pragma unroll
+        for (int i = EPT16 - 1; i >= 0; --i) quant_m(i);
+        quant_m_done();
     }
 
     // ---- (D) second moment: block scale and the p-quantile (k = 13 of 128); the draws of Eq. 6 ----
@@ -461,7 +476,16 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
         uint32_t key[EPT16];
 #pragma unroll
         for (int i = 0; i < EPT16; ++i) key[i] = __float_as_uint(vh[i]);
-        sort16_low13(key);
+        if constexpr (SOLO_F16_MIX) {
+#pragma unroll
+            for (int k = 0; k < 62; ++k) {
+                cswap(key[SORT16_PAIRS[k][0]], key[SORT16_PAIRS[k][1]]);
+                if ((k & 3) == 3 || k == 61) quant_m(15 - (k >> 2));
+            }
+            quant_m_done();
+        } else {
+            sort16_low13(key);
+        }
         uint32_t* const col = &s.sort[0][tid];
 #pragma unroll
         for (int j = 1; j <= 12; ++j) col[(j - 1) * CTA16] = key[j];

@@ -261,23 +261,97 @@ def test_ragged_zero_blocks_and_zero_elements():
         assert rep.exempt_m + rep.exempt_v <= 3
 
 
-def test_nan_and_inf_gradients_do_not_hang():
-    sizes = (128 * 4,)
+@pytest.mark.parametrize("bits_m,bits_v,block", [(2, 3, 128), (4, 4, 128), (3, 2, 64), (2, 2, 2048), (8, 4, 256)])
+def test_nan_and_inf_gradients_follow_one_rule(bits_m, bits_v, block):
+    """The paper says nothing about non-finite gradients; the rule here is that they propagate: a
+    NaN in a block makes that block's scale NaN and its codes 0, an infinity makes the scale
+    infinite, the element's parameter becomes NaN, and nothing outside the block changes.  Every
+    kernel (sixteen-per-thread where it exists, streamlined, general) must reproduce the oracle's
+    state bit for bit (NaN equal to NaN) and leave the other blocks' parameters finite."""
+    sizes = (2048 * 3 + 300, 700)
     w = synth.workload(1, sizes=sizes)
     params, _ = _inputs(w)
-    g = synth.make_grad(w, 0, 1)
-    g[5] = float("nan")
-    g[200] = float("inf")
+
+    def gf(t):
+        gs = [synth.make_grad(w, i, t) for i in range(2)]
+        gs[0][5] = float("nan")                 # full tile, first block
+        gs[0][2048 + 200] = float("inf")        # full tile, another block
+        gs[0][2048 + 700] = float("-inf")
+        gs[0][2048 * 3 + 17] = float("nan")     # tail tile
+        gs[1][650] = float("inf")
+        if t == 2:
+            gs[0][4096:4096 + 128] = float("nan")   # a whole block of NaN
+        return gs
+
+    policies = (3, 2, 1) if block == 128 and max(bits_m, bits_v) <= 4 else (0, 1)
+    run_lockstep(sizes, bits_m, bits_v, block, dict(seed=9, weight_decay=0.0), 3, gf, params, policies=policies)
+    # and on its own state for three steps: no hang, status clean, untouched blocks finite
     from paper_2505_00347_b200 import binding as B
-    st = B.State(sizes[0], 4, 4, 128)
-    p = params[0].cuda()
-    for t in (1, 2):
-        B.solo_step(p, g.cuda(), st, B.hyper(), t)
+    st = B.State(list(sizes), bits_m, bits_v, block)
+    ps = [p.cuda() for p in params]
+    for t in (1, 2, 3):
+        B.solo_multi_step(B.TensorSet(ps, [g.cuda() for g in gf(t)], st), B.hyper(), t)
     torch.cuda.synchronize()
-    out = p.cpu()
-    assert torch.isfinite(out[256:]).all()          # untouched blocks stay finite
     assert st.status() == 0
+    for i in range(2):                          # blocks that never saw a non-finite gradient stay finite
+        bad = torch.zeros(sizes[i], dtype=torch.bool)
+        for t in (1, 2, 3):
+            bad |= ~torch.isfinite(gf(t)[i].float())
+        nb = -(-sizes[i] // block)
+        pad = torch.zeros(nb * block, dtype=torch.bool)
+        pad[: sizes[i]] = bad
+        clean = ~pad.view(nb, block).any(dim=1).repeat_interleave(block)[: sizes[i]]
+        assert clean.any() or block == 2048
+        assert torch.isfinite(ps[i].cpu()[clean]).all()
     st.destroy()
+
+
+def test_bounded_wait_runs_out_and_nothing_is_stored():
+    """A copy of a tile's inputs that announces more bytes than it brings never completes its
+    barrier phase: the kernel's bounded wait gives up, status bit 1 is set, the warps concerned store
+    nothing (that tile's parameters and state keep their old values), every other tile is stepped
+    as usual and the kernel returns.  Both kernels that stage their inputs."""
+    from paper_2505_00347_b200 import binding as B
+    tiles = 24
+    sizes = (2048 * tiles,)
+    w = synth.workload(3, sizes=sizes)
+    p0 = synth.make_param(w, 0)
+    g = synth.make_grad(w, 0, 1).cuda()
+    st0 = synth.make_state(sizes, 2, 3, 128, seed=31)
+    h = B.hyper(lr=1e-3, beta1=0.5, weight_decay=0.0, seed=4)
+    for policy, stalled in ((3, 7), (2, 11)):
+        B.set_kernel_policy(policy)
+        try:
+            ref, hit = B.State(sizes[0], 2, 3, 128), B.State(sizes[0], 2, 3, 128)
+            for s_ in (ref, hit):
+                for k, v in st0.items():
+                    s_.raw_set(k, v)
+            p_ref, p_hit = p0.clone().cuda(), p0.clone().cuda()
+            B.solo_step(p_ref, g, ref, h, 1)
+            B.debug_stall_copy(stalled)
+            B.solo_step(p_hit, g, hit, h, 1)
+            torch.cuda.synchronize()
+            assert ref.status() == 0 and hit.status() == 2
+            lo, hi = stalled * 2048, (stalled + 1) * 2048
+            same = torch.ones(sizes[0], dtype=torch.bool)
+            same[lo:hi] = False
+            assert torch.equal(p_hit.cpu()[same], p_ref.cpu()[same])
+            assert torch.equal(p_hit.cpu()[lo:hi], p0[lo:hi])                  # untouched
+            for key, per_tile in (("codes_m", 512), ("codes_v", 768), ("scale_m", 16), ("scale_v", 16), ("alpha", 16)):
+                got, want, old = hit.raw_get(key), ref.raw_get(key), st0[key]
+                a, b = stalled * per_tile, (stalled + 1) * per_tile
+                assert torch.equal(got[:a], want[:a]) and torch.equal(got[b:], want[b:]), key
+                assert torch.equal(got[a:b], old[a:b]), key
+            # the hook is one-shot: the next step is an ordinary one (the status word is sticky)
+            B.solo_step(p_hit, g, hit, h, 2)
+            B.solo_step(p_ref, g, ref, h, 2)
+            torch.cuda.synchronize()
+            assert torch.equal(p_hit.cpu()[same], p_ref.cpu()[same])
+            assert hit.status() == 2
+            ref.destroy()
+            hit.destroy()
+        finally:
+            B.set_kernel_policy(0)
 
 
 @pytest.mark.parametrize("bits_m,bits_v,block,extra,chunk", [

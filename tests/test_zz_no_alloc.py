@@ -61,8 +61,16 @@ def _run_pair(B, sizes, bits_m, bits_v, block, steps, seed, state0=None, **hyper
     for t in range(1, steps + 1):
         grads = [synth.make_grad(w, i, t).cuda() for i in range(len(sizes))]
         B.solo_multi_step(B.TensorSet(p_lib, grads, lib_state), h, t)
-        B.solo_multi_step_static(p_sta, grads, list(sizes), bufs, bits_m, bits_v, block, h, t)
+        # the pointer arrays are made with torch before the measurement: what is measured is the library call
+        pp = torch.tensor([p.data_ptr() for p in p_sta], dtype=torch.int64, device="cuda")
+        gp = torch.tensor([g.data_ptr() for g in grads], dtype=torch.int64, device="cuda")
         torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
+        B.solo_multi_step_static(p_sta, grads, list(sizes), bufs, bits_m, bits_v, block, h, t,
+                                 param_ptrs=pp, grad_ptrs=gp)
+        assert B.static_status() == 0                     # waits for the stream; no mismatch, no copy given up on
+        if t > 1:     # (the very first call on a device may load the library's kernels and looks the fixed array up)
+            assert torch.cuda.mem_get_info()[0] == free_before   # free device memory did not move: nothing was allocated
         for key in ("codes_m", "codes_v", "scale_m", "scale_v", "alpha"):
             got = bufs[key].cpu().numpy().view(np.uint8)
             want = lib_state.raw_get(key).numpy().view(np.uint8)
@@ -84,6 +92,33 @@ def test_static_entry_point_matches_library_state_twice():
     _run_pair(B, sizes, 8, 4, 2048, steps=2, seed=8, state0=st0, round_m=1)
     # third: a baseline codebook for the second moment (its table also lives in the fixed array)
     _run_pair(B, (2048 + 9, 640), 4, 4, 128, steps=2, seed=9, v_codebook=3)
+
+
+def test_static_entry_point_refuses_a_capturing_stream():
+    """The call copies its tables from its own stack frame; recorded into a graph those copies would
+    read a dead frame at replay, so a capturing stream is refused before anything is queued."""
+    from paper_2505_00347_b200 import binding as B
+    sizes = [2048 + 5]
+    ps = [torch.zeros(sizes[0], device="cuda")]
+    gs = [torch.zeros(sizes[0], device="cuda", dtype=torch.bfloat16)]
+    bufs = _fresh_buffers(sizes, 2, 3, 128)
+    pp = torch.tensor([ps[0].data_ptr()], dtype=torch.int64, device="cuda")
+    gp = torch.tensor([gs[0].data_ptr()], dtype=torch.int64, device="cuda")
+    B.solo_multi_step_static(ps, gs, sizes, bufs, 2, 3, 128, B.hyper(), 1, param_ptrs=pp, grad_ptrs=gp)   # looks the array up
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        graph.capture_begin()
+        try:
+            with pytest.raises(B.SoloError) as e:
+                B.solo_multi_step_static(ps, gs, sizes, bufs, 2, 3, 128, B.hyper(), 2, param_ptrs=pp, grad_ptrs=gp)
+            assert e.value.status == B.SOLO_EINVAL
+        finally:
+            graph.capture_end()
+    torch.cuda.synchronize()
+    B.solo_multi_step_static(ps, gs, sizes, bufs, 2, 3, 128, B.hyper(), 2, param_ptrs=pp, grad_ptrs=gp)   # still usable
+    assert B.static_status() == 0
 
 
 def test_static_entry_point_rejects_what_it_cannot_hold():
