@@ -88,10 +88,13 @@ class Report:
         self.exempt_m = 0
         self.exempt_v = 0
         self.max_param_rel = 0.0
+        self.allowance_elems = 0      # parameters outside 1e-6 / 1e-9 that pass only through update_tol
+        self.allowance_excess = 0.0   # their largest distance beyond the 1e-6 / 1e-9 bound
 
     def __repr__(self):
         return (f"elements={self.elements} exempt_m={self.exempt_m} exempt_v={self.exempt_v} "
-                f"max_param_err={self.max_param_rel:.3g}")
+                f"max_param_err={self.max_param_rel:.3g} beyond_plain_bar={self.allowance_elems} "
+                f"(largest excess {self.allowance_excess:.3g})")
 
 
 def close(a: np.ndarray, b: np.ndarray) -> np.ndarray:
@@ -138,7 +141,7 @@ def flags_to_blocks(flags_list, sizes, block) -> np.ndarray:
 
 
 def run_lockstep(sizes, bits_m, bits_v, block, hyper_kw, steps, grads_fn, params0, state0=None,
-                 multi=None, free_run=False, nthreads=8, policies=(0, 1), update_tol=3e-7):
+                 multi=None, free_run=False, nthreads=8, policies=(0, 1), update_tol=0.0):
     """Runs `steps` steps on both sides.
 
     lock-step (free_run=False): before every step the library's state and parameters are set to
@@ -147,9 +150,11 @@ def run_lockstep(sizes, bits_m, bits_v, block, hyper_kw, steps, grads_fn, params
     grads_fn(step) -> list of CPU bf16 tensors; params0: list of CPU tensors (fp32 or bf16).
     policies: kernel-selection policies of the library to run (0 streamlined where it applies,
     1 general kernel); each is compared with the one oracle run.
-    update_tol: extra parameter tolerance as a fraction of |p_new - p_old| (the streamlined
-    kernel computes the update term to a few ulp, not with IEEE division and square root);
-    pass 0 to hold the parameters to the plain 1e-6 relative / 1e-9 absolute bar.
+    update_tol: extra parameter tolerance as a fraction of |p_new - p_old|.  The default 0 holds the
+    parameters to the plain 1e-6 relative / 1e-9 absolute bar.  The two faster kernels compute the
+    update term with an approximate square root and a refined approximate reciprocal (a few 1e-7 of
+    the term, not bit for bit); tests whose learning rate or random state makes that term large
+    pass 3e-7 here, and the report counts how many elements needed it and by how much.
     """
     from paper_2505_00347_b200 import binding as B
     sizes = [int(n) for n in sizes]
@@ -205,7 +210,14 @@ def run_lockstep(sizes, bits_m, bits_v, block, hyper_kw, steps, grads_fn, params
                 ok |= np.abs(gp.astype(np.float64) - wp) <= RTOL * np.abs(wp) + ATOL * steps
             if update_tol and prev is not None:
                 upd = np.abs(wp.astype(np.float64) - prev[i].astype(np.float64))
-                ok |= np.abs(gp.astype(np.float64) - wp) <= RTOL * np.abs(wp) + ATOL + update_tol * upd
+                err = np.abs(gp.astype(np.float64) - wp)
+                allowed = err <= RTOL * np.abs(wp) + ATOL + update_tol * upd
+                only = allowed & ~ok
+                if only.any():
+                    rep.allowance_elems += int(only.sum())
+                    rep.allowance_excess = max(rep.allowance_excess,
+                                               float((err - RTOL * np.abs(wp) - ATOL)[only].max()))
+                ok |= allowed
             assert ok.all(), (f"{where} tensor {i} params", int((~ok).sum()), gp[~ok][:4], wp[~ok][:4])
             if bf16p and not free_run:
                 # both kernels compute the update of bf16 parameters with IEEE division and square root: the

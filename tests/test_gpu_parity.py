@@ -11,6 +11,11 @@ from parity import run_lockstep
 
 pytestmark = pytest.mark.gpu
 
+# Extra parameter tolerance, as a fraction of the update |p_new - p_old|, for runs that start from a
+# random packed state or use a learning rate of 0.1 (see parity.run_lockstep); everything else is held
+# to the plain 1e-6 relative / 1e-9 absolute bar.
+RANDOM_STATE_TOL = 3e-7
+
 
 def _inputs(w, device="cpu"):
     params = [synth.make_param(w, i) for i in range(len(w.sizes))]
@@ -33,15 +38,13 @@ def test_gpt125m_set_free_run_100_steps():
     """GPT-style 125M set (148 tensors, 124,439,808 parameters, 3-bit / 3-bit, block 128): the
     library runs 100 steps on its own state, the oracle likewise; the packed state is compared bit
     for bit at steps 10, 50 and 100 (any difference would compound, so equality at 100 covers every
-    step), the parameters within the per-step tolerance accumulated over the steps."""
+    step), the parameters within the plain per-step tolerance accumulated over the steps."""
     from paper_2505_00347_b200 import binding as B
     w = synth.workload(2)
     T = len(w.sizes)
     dev = torch.device("cuda")
     gparams = [synth.make_param(w, i, device=dev) for i in range(T)]
     oparams = [p.cpu().numpy().copy() for p in gparams]
-    prev = [p.clone() for p in gparams]
-    path = [torch.zeros_like(p) for p in gparams]                # sum over the steps of |update|
     gstate = B.State(list(w.sizes), 3, 3, 128)
     ostates = [oracle.State(n, 3, 3, 128) for n in w.sizes]
     kw = dict(lr=w.lr, beta1=w.beta1, beta2=w.beta2, weight_decay=w.weight_decay, seed=2024)
@@ -51,8 +54,6 @@ def test_gpt125m_set_free_run_100_steps():
         grads = [synth.make_grad(w, i, t, device=dev) for i in range(T)]
         B.solo_multi_step(B.TensorSet(gparams, grads, gstate), hg, t)
         for i in range(T):
-            path[i] += (gparams[i] - prev[i]).abs()
-            prev[i].copy_(gparams[i])
             oracle.step(oparams[i], synth.bf16_bits(grads[i]), ostates[i], ho, t, tensor=i, nthreads=threads)
         if t in (10, 50, 100):
             torch.cuda.synchronize()
@@ -64,8 +65,8 @@ def test_gpt125m_set_free_run_100_steps():
             for i in range(T):
                 gp = gparams[i].cpu().numpy().astype(np.float64)
                 wp = oparams[i].astype(np.float64)
-                # per step: 1e-6 relative / 1e-9 absolute plus 3e-7 of the update term
-                tol = parity.RTOL * np.abs(wp) + parity.ATOL * t + 3e-7 * path[i].cpu().numpy().astype(np.float64)
+                # the plain bar, 1e-6 relative / 1e-9 absolute per step, accumulated over the steps
+                tol = parity.RTOL * np.abs(wp) + parity.ATOL * t
                 assert np.all(np.abs(gp - wp) <= tol), (t, i, float(np.max(np.abs(gp - wp) - tol)))
     gstate.destroy()
 
@@ -83,8 +84,13 @@ def test_bits_and_blocks_random_state(bits_m, bits_v, block):
     # block 128 with widths up to 4 bits: policy 3 is the sixteen-per-thread kernel plus the
     # streamlined kernel for the tails (policy 0 picks it for large sets only)
     policies = (0, 3, 1) if block == 128 and max(bits_m, bits_v) <= 4 else (0, 1)
-    rep = run_lockstep(sizes, bits_m, bits_v, block, hk, 2, gf, params, state0=st0, policies=policies)
+    # a random packed state pairs huge first moments with tiny second moments: update terms far above
+    # the parameters themselves, where the faster kernels' quotient (a few 1e-7 of the term) shows
+    rep = run_lockstep(sizes, bits_m, bits_v, block, hk, 2, gf, params, state0=st0, policies=policies,
+                       update_tol=RANDOM_STATE_TOL)
+    print(rep)
     assert rep.exempt_m + rep.exempt_v <= 3 * len(policies)
+    assert rep.allowance_elems <= 1e-3 * rep.elements
 
 
 @pytest.mark.parametrize("bits_m,bits_v,block", [(2, 3, 128), (3, 2, 64), (4, 4, 256), (2, 2, 2048), (8, 4, 64),
@@ -102,7 +108,7 @@ def test_mode_flags_at_other_widths(bits_m, bits_v, block, hk):
     base = dict(lr=1e-3, beta1=0.6, beta2=0.999, weight_decay=0.01, seed=13)
     base.update(hk)
     st0 = synth.make_state(sizes, bits_m, bits_v, block, seed=19)
-    run_lockstep(sizes, bits_m, bits_v, block, base, 2, gf, params, state0=st0)
+    print(run_lockstep(sizes, bits_m, bits_v, block, base, 2, gf, params, state0=st0, update_tol=RANDOM_STATE_TOL))
 
 
 @pytest.mark.parametrize("hk", [
@@ -134,8 +140,11 @@ def test_hyper_parameter_modes(hk):
     base = dict(lr=1e-3, beta1=0.8, beta2=0.999, weight_decay=0.01, seed=3)
     base.update(hk)
     st0 = synth.make_state(sizes, 4, 3, 128, seed=17)
-    run_lockstep(sizes, 4, 3, 128, base, 3, gf, params, state0=st0)
-    run_lockstep(sizes, 4, 3, 128, base, 3, gf, params)
+    print(run_lockstep(sizes, 4, 3, 128, base, 3, gf, params, state0=st0, update_tol=RANDOM_STATE_TOL))
+    # from the zero state the plain bar holds, except at a learning rate of 0.1 (updates of the
+    # parameters' own size)
+    print(run_lockstep(sizes, 4, 3, 128, base, 3, gf, params,
+                       update_tol=RANDOM_STATE_TOL if base["lr"] > 1e-2 else 0.0))
 
 
 @pytest.mark.parametrize("sel", [1, 2, 3])
@@ -202,7 +211,8 @@ def test_block_128_plain_step_all_three_kernels(bits_m, bits_v):
     params, gf = _inputs(w)
     hk = dict(lr=2e-5, beta1=0.5, beta2=0.999, weight_decay=0.0, seed=1234)
     st0 = synth.make_state(sizes, bits_m, bits_v, 128, seed=5)
-    run_lockstep(sizes, bits_m, bits_v, 128, hk, 3, gf, params, state0=st0, policies=(3, 2, 1))
+    print(run_lockstep(sizes, bits_m, bits_v, 128, hk, 3, gf, params, state0=st0, policies=(3, 2, 1),
+                       update_tol=RANDOM_STATE_TOL))
     run_lockstep(sizes, bits_m, bits_v, 128, hk, 4, gf, params, policies=(3, 2, 1))
     w1 = synth.workload(1, sizes=(2048 * 6,))
     p1, g1 = _inputs(w1)
@@ -554,7 +564,7 @@ def _full_size_sampled(cfg: int, random_per_tensor: int, need_bytes: float, over
         B._cuda_memcpy(out.data_ptr(), ptrs[key] + off, nbytes, 2)
         return out.numpy().view(dtype)
 
-    worst = 0.0
+    worst, beyond, excess, checked = 0.0, 0, -1.0, 0
     for (t, j), b in zip(sample, before):
         n = b["p"].size
         ost = oracle.State(n, bm, bv, block)
@@ -573,18 +583,97 @@ def _full_size_sampled(cfg: int, random_per_tensor: int, need_bytes: float, over
         gp = params[t][j * block: j * block + n].cpu().numpy()
         err = np.abs(gp.astype(np.float64) - p)
         # random states pair huge first moments with tiny second moments: allow the streamlined
-        # kernel's 3e-7 of the update term on top of the 1e-6 / 1e-9 bar
-        tol = parity.RTOL * np.abs(p) + parity.ATOL + 3e-7 * np.abs(p - b["p"].astype(np.float64))
+        # kernel's 3e-7 of the update term on top of the 1e-6 / 1e-9 bar, and count who needs it
+        plain = parity.RTOL * np.abs(p) + parity.ATOL
+        tol = plain + 3e-7 * np.abs(p - b["p"].astype(np.float64))
         assert np.all(err <= tol), (t, j, float(err.max()))
+        beyond += int((err > plain).sum())
+        excess = max(excess, float((err - plain).max()))
+        checked += n
         worst = max(worst, float(err.max()))
     print(f"workload {cfg}: {len(sample)} blocks of {len(w.sizes)} tensors checked, "
-          f"largest parameter difference {worst:.3g}")
+          f"largest parameter difference {worst:.3g}; {beyond} of {checked} parameters beyond the plain "
+          f"1e-6 / 1e-9 bar (largest excess {max(excess, 0.0):.3g}), all within 3e-7 of their update")
     gstate.destroy()
 
 
 def test_full_size_7b_set_sampled_blocks():
     """LLaMA-7B-shaped set, 6.74 B parameters, 2-bit / 3-bit, block 128 (the headline workload)."""
     _full_size_sampled(3, 12, 60e9)
+
+
+def test_full_size_7b_set_ten_steps_from_zero_plain_bar():
+    """The headline workload on realistic values: from the zero state, ten steps with fresh gradients,
+    the library running on its own state.  Sampled blocks (first, last and four random ones per tensor)
+    are stepped by the oracle alongside; their packed state must be identical at steps 1, 5 and 10 and
+    their parameters within the plain bar, 1e-6 relative / 1e-9 absolute per step, with no allowance
+    for the approximate division."""
+    from paper_2505_00347_b200 import binding as B
+    free, _ = torch.cuda.mem_get_info()
+    if free < 62e9:
+        pytest.skip("needs about 62 GB of free device memory")
+    w = synth.workload(3)
+    bm, bv, block = w.bits_m, w.bits_v, w.block
+    dev = torch.device("cuda")
+    T = len(w.sizes)
+    params = [synth.make_param(w, i, device=dev) for i in range(T)]
+    gstate = B.State(list(w.sizes), bm, bv, block)
+    rng = np.random.default_rng(77)
+    nblk = [-(-n // block) for n in w.sizes]
+    bstart = np.concatenate([[0], np.cumsum(nblk)])
+    picks = [sorted({0, nb - 1} | set(int(x) for x in rng.integers(0, nb, size=4 if nb > 2 else 0))) for nb in nblk]
+    idx = []                                                   # per tensor: element indices of its sampled blocks
+    for t in range(T):
+        e = np.concatenate([np.arange(j * block, min(w.sizes[t], (j + 1) * block)) for j in picks[t]])
+        idx.append(torch.from_numpy(e).to(dev))
+    osts, ops = [], []
+    for t in range(T):
+        for j in picks[t]:
+            n = min(w.sizes[t], (j + 1) * block) - j * block
+            osts.append(oracle.State(n, bm, bv, block))
+            ops.append(params[t][j * block: j * block + n].cpu().numpy().copy())
+    kw = dict(lr=w.lr, beta1=w.beta1, beta2=w.beta2, weight_decay=w.weight_decay, seed=1234)
+    ho, hg = parity.hyper_pair(**kw)
+    ptrs = {k: gstate.raw_ptr(k)[0] for k in parity.KEYS}
+    sm, sv = block * bm // 8, block * bv // 8
+
+    def fetch(key, off, nbytes, dtype):
+        out = torch.empty(nbytes, dtype=torch.uint8)
+        B._cuda_memcpy(out.data_ptr(), ptrs[key] + off, nbytes, 2)
+        return out.numpy().view(dtype)
+
+    worst = 0.0
+    for step in range(1, 11):
+        grads = [synth.make_grad(w, i, step, device=dev) for i in range(T)]
+        gs = [synth.bf16_bits(grads[t][idx[t]]) for t in range(T)]
+        B.solo_multi_step(B.TensorSet(params, grads, gstate), hg, step)
+        torch.cuda.synchronize()
+        del grads
+        k = 0
+        for t in range(T):
+            pos = 0
+            for j in picks[t]:
+                n = osts[k].numel
+                oracle.step(ops[k], gs[t][pos:pos + n], osts[k], ho, step, tensor=t, elem_offset=j * block)
+                pos += n
+                k += 1
+        if step in (1, 5, 10):
+            assert gstate.status() == 0
+            k = 0
+            for t in range(T):
+                for j in picks[t]:
+                    jb, ost = int(bstart[t]) + j, osts[k]
+                    assert np.array_equal(fetch("codes_m", jb * sm, sm, np.uint8), ost.codes_m), (step, t, j)
+                    assert np.array_equal(fetch("codes_v", jb * sv, sv, np.uint8), ost.codes_v), (step, t, j)
+                    for key in ("scale_m", "scale_v", "alpha"):
+                        assert np.array_equal(fetch(key, jb * 4, 4, np.uint32), getattr(ost, key).view(np.uint32)), (step, t, j, key)
+                    gp = params[t][j * block: j * block + ost.numel].cpu().numpy().astype(np.float64)
+                    err = np.abs(gp - ops[k])
+                    assert np.all(err <= parity.RTOL * np.abs(ops[k]) + parity.ATOL * step), (step, t, j, float(err.max()))
+                    worst = max(worst, float(err.max()))
+                    k += 1
+    print(f"7B set, 10 steps from zero: {len(osts)} blocks followed, largest parameter difference {worst:.3g}")
+    gstate.destroy()
 
 
 def test_full_size_7b_set_bf16_parameters_stochastic_rounding():
