@@ -3,6 +3,12 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..5] [--impl ours|reference]
 
+With --gpus N > 1 and no launcher in the environment the command starts N ranks itself (one per
+GPU, torch.distributed.run on 127.0.0.1); under a launcher it uses the ranks it is given.  Blocks
+are independent, so the ranks share nothing on the data path: each steps its own shard (same shapes,
+its own random streams) and the job's throughput is all ranks' parameters over the slowest rank's
+time (weak scaling).
+
 A step is one pass of the whole hot path (one solo_multi_step launch) over the workload's
 tensor set.  Default workload: the LLaMA-7B-shaped set (6.74 B parameters, 2-bit first and 3-bit
 second moments, block 128), the configuration the headline metric is quoted on; it fits one
@@ -141,6 +147,9 @@ def run_ours(args, rank, world):
     w, params, grads = build_workload(args.workload, device, args)
     B.set_kernel_policy(args.policy)
     state = B.State(list(w.sizes), w.bits_m, w.bits_v, w.block)
+    if world > 1:
+        # every rank steps its own shard of a job `world` times as large: same shapes, its own random streams
+        state.set_origin([rank * len(w.sizes) + t for t in range(len(w.sizes))], None)
     ts = B.TensorSet(params, grads, state)
     h = B.hyper(lr=w.lr, beta1=w.beta1, beta2=w.beta2, weight_decay=w.weight_decay, seed=1234,
                 fixed_alpha=args.fixed_alpha, v_codebook=args.v_codebook,
@@ -321,6 +330,17 @@ def run_reference(args, rank, world):
             "e2e": {"value": round(v, 5), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
 
 
+def spawn_ranks(n: int) -> int:
+    """Re-runs this command as `n` ranks on this node, one per GPU, and returns the launcher's exit code."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *sys.argv[1:]]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -345,8 +365,14 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # not under a launcher yet: start one rank per GPU (this same command under torch.distributed.run)
+        sys.exit(spawn_ranks(args.gpus))
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
+    if world != max(args.gpus, 1) and rank == 0:
+        print(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s); reporting {world}",
+              file=sys.stderr)
     if args.impl == "reference":
         out = run_reference(args, rank, world)
     else:

@@ -159,6 +159,24 @@ int solo_multi_step(const solo_tensor_list_t* list, const solo_hyper_t* hyper, i
                     void* stream);
 
 /*
+ * Sharding (Sec. 4.2, "Generalizability": optimizer states that are flattened and partitioned
+ * across workers, as under FSDP, suit element-wise optimizers such as this one).  Blocks are
+ * independent, so a worker may own any block-aligned piece of a tensor and step it with a state
+ * of its own; the only thing that ties a piece to its tensor is the random stream of the
+ * rounding noise, which is addressed by (tensor, element index).  This call tells a state where
+ * each of its tensors sits in that stream; both arrays are HOST arrays of the state's tensor count:
+ *   stream_id_host[t]    the number of the Philox stream of tensor t (0 .. 2^30 - 1); the
+ *                        default is t, the tensor's position in the list
+ *   elem_offset_host[t]  the index, within the whole tensor, of the first element that this
+ *                        state's tensor t holds; a multiple of the block size; default 0
+ * Either may be NULL (its default); both NULL restore the defaults.  With these set, stepping
+ * the pieces of a tensor on any number of workers gives the codes, scales and parameters of
+ * stepping the whole tensor at once.  Synchronizes the device; SOLO_EINVAL for an offset that is
+ * negative or not on a block boundary.
+ */
+int solo_state_set_origin(solo_state_t* state, const int32_t* stream_id_host, const int64_t* elem_offset_host);
+
+/*
  * The same step for a worker whose gradients arrive in HOST memory and that wants a HOST copy
  * of the updated parameters (the paper has no counterpart: it does not discuss where the
  * tensors live).  The parameters and the state stay resident on the device.  Every pointer
@@ -325,8 +343,9 @@ typedef struct {
  * cudaMalloc / cudaFree is not acceptable.  solo_state_create allocates; this entry point
  * never does.  The caller brings the state buffers (solo_raw_state_t); the small tables the
  * kernel needs besides them -- the tile and block offsets of every tensor, the first-moment
- * codebook and a status word, 32 KiB in all -- live in one fixed array inside the library
- * that every GPU loading the library holds until the process exits.
+ * codebook and a status word, 32 KiB, plus 8 KiB of zeros that stand for the default position
+ * of the tensors in the random stream -- live in fixed arrays inside the library that every GPU
+ * loading the library holds until the process exits.
  *
  *   num_tensors        1 .. SOLO_STATIC_MAX_TENSORS; more is refused with SOLO_ELIMIT
  *   param_dev, grad_dev  DEVICE arrays of num_tensors device pointers (as in solo_tensor_list_t)

@@ -116,6 +116,8 @@ def lib() -> C.CDLL:
     L.solo_state_export_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
     L.solo_state_export.argtypes = [vp, vp, C.c_size_t, vp]
     L.solo_state_import.argtypes = [vp, vp, C.c_size_t, vp]
+    L.solo_state_set_origin.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
+    L.solo_state_set_origin.restype = C.c_int
     L.solo_static_status.argtypes = [C.POINTER(C.c_int), vp]
     L.solo_static_status.restype = C.c_int
     L.solo_debug_stall_copy.argtypes = [i64]
@@ -177,6 +179,14 @@ class State:
             self.destroy()
         except Exception:
             pass
+
+    def set_origin(self, stream_ids=None, elem_offsets=None) -> None:
+        """solo_state_set_origin: where each tensor of this state sits in the random stream (the
+        tensor's stream number and the index of its first element within the whole tensor)."""
+        T = len(self.sizes)
+        ids = (C.c_int32 * T)(*[int(x) for x in stream_ids]) if stream_ids is not None else None
+        offs = (C.c_int64 * T)(*[int(x) for x in elem_offsets]) if elem_offsets is not None else None
+        _check(lib().solo_state_set_origin(self.handle, ids, offs), "solo_state_set_origin")
 
     def info(self) -> dict:
         n, nb = C.c_int64(), C.c_int64()

@@ -32,6 +32,8 @@ struct solo_state {
     float* tables_v = nullptr;    // the three baseline second-moment codebooks for bits_v, each y[K] | mid[K-1]
     int v_codebook = SOLO_V_LOG;  // selector of the last step (what solo_dequant decodes with)
     int* status = nullptr;
+    int32_t* origin_id = nullptr;   // [T] device: Philox stream of every tensor minus its position in the list (solo_state_set_origin)
+    int64_t* origin_ctr = nullptr;  // [T] device: stream position (element index / 8) of every tensor's first element
     size_t bytes_codes_m = 0, bytes_codes_v = 0;
     struct HostPipe* pipe = nullptr;   // staging of solo_multi_step_host, created at its first call
 };
@@ -261,6 +263,8 @@ void fill_state_args(const solo_state* s, StepArgs& a) {
     a.alpha = s->alpha;
     a.tables = s->tables_m;
     a.status = s->status;
+    a.origin_id = s->origin_id;
+    a.origin_ctr = s->origin_ctr;
 }
 
 // Second-moment quantizer of this step; the state remembers it for solo_dequant.
@@ -292,23 +296,30 @@ constexpr size_t STATIC_BYTES = STATIC_STATUS_OFF + 16;
 static_assert(STATIC_BYTES <= 32 * 1024, "documented size of the fixed scratch");
 
 static __device__ __align__(256) unsigned char g_static_scratch[STATIC_BYTES];
+// Zeros, never written: the default position in the random stream of every tensor of a
+// solo_multi_step_static call (read as the int32 and as the int64 array of StepArgs).
+static __device__ __align__(256) int64_t g_static_zero_origin[STATIC_MAX_T];
 
 // Device address of g_static_scratch on the current device (the symbol's name is only a
 // host-side handle).  Looked up once per device, with that device current.
-int static_scratch(int device, unsigned char** out) {
+int static_scratch(int device, unsigned char** out, const int64_t** zeros_out = nullptr) {
     static std::mutex mu;
     static unsigned char* ptr[64];
+    static const int64_t* zeros[64];
     if (device < 0 || device >= 64) return SOLO_EINVAL;
     std::lock_guard<std::mutex> lk(mu);
     if (!ptr[device]) {
-        void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+        void *p = nullptr, *z = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p ||
+            cudaGetSymbolAddress(&z, g_static_zero_origin) != cudaSuccess || !z) {
             cudaGetLastError();
             return SOLO_ECUDA;
         }
         ptr[device] = (unsigned char*)p;
+        zeros[device] = (const int64_t*)z;
     }
     *out = ptr[device];
+    if (zeros_out) *zeros_out = zeros[device];
     return SOLO_OK;
 }
 
@@ -381,6 +392,8 @@ int solo_state_create_multi(const int64_t* numel_host, int num_tensors, int bits
     alloc((void**)&s->tables_m, tm.size() * 4);
     alloc((void**)&s->tables_v, tv.size() * 4);
     alloc((void**)&s->status, 4);
+    alloc((void**)&s->origin_id, (size_t)T * 4);
+    alloc((void**)&s->origin_ctr, (size_t)T * 8);
     if (!ok) { solo_state_destroy(s); return SOLO_ENOMEM; }
     cudaError_t e = cudaSuccess;
     auto chk = [&](cudaError_t r) { if (e == cudaSuccess) e = r; };
@@ -390,6 +403,8 @@ int solo_state_create_multi(const int64_t* numel_host, int num_tensors, int bits
     chk(cudaMemset(s->scale_v, 0, scal_bytes));
     chk(cudaMemset(s->alpha, 0, scal_bytes));
     chk(cudaMemset(s->status, 0, 4));
+    chk(cudaMemset(s->origin_id, 0, (size_t)T * 4));
+    chk(cudaMemset(s->origin_ctr, 0, (size_t)T * 8));
     chk(cudaMemcpy(s->geom, geom.data(), geom.size() * 8, cudaMemcpyHostToDevice));
     chk(cudaMemcpy(s->tables_m, tm.data(), tm.size() * 4, cudaMemcpyHostToDevice));
     chk(cudaMemcpy(s->tables_v, tv.data(), tv.size() * 4, cudaMemcpyHostToDevice));
@@ -427,10 +442,33 @@ int solo_state_destroy(solo_state_t* s) {
         s->pipe = nullptr;
     }
     void* ptrs[] = {s->codes_m, s->codes_v, s->scale_m, s->scale_v, s->alpha,
-                    s->geom, s->tables_m, s->tables_v, s->status};
+                    s->geom, s->tables_m, s->tables_v, s->status, s->origin_id, s->origin_ctr};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     delete s;
+    return SOLO_OK;
+}
+
+int solo_state_set_origin(solo_state_t* s, const int32_t* stream_id_host, const int64_t* elem_offset_host) {
+    if (!s) return SOLO_EINVAL;
+    if (!on_state_device(s)) return SOLO_ESTATE;
+    const int T = s->num_tensors;
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return SOLO_ECUDA; }   // steps in flight read the arrays
+    std::vector<int32_t> id((size_t)T);
+    std::vector<int64_t> ctr((size_t)T);
+    for (int t = 0; t < T; ++t) {
+        const int32_t stream = stream_id_host ? stream_id_host[t] : t;
+        const int64_t off = elem_offset_host ? elem_offset_host[t] : 0;
+        // a shard starts on a block boundary of its tensor; the stream id shares a 32-bit word with the purpose
+        if (off < 0 || off % s->block != 0 || stream < 0 || stream >= (1 << 30)) return SOLO_EINVAL;
+        id[t] = stream - t;
+        ctr[t] = off / 8;
+    }
+    if (cudaMemcpy(s->origin_id, id.data(), (size_t)T * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(s->origin_ctr, ctr.data(), (size_t)T * 8, cudaMemcpyHostToDevice) != cudaSuccess) {
+        cudaGetLastError();
+        return SOLO_ECUDA;
+    }
     return SOLO_OK;
 }
 
@@ -614,7 +652,8 @@ int solo_multi_step_static(int32_t num_tensors, void* const* param_dev, const vo
     int device = -1;
     if (cudaGetDevice(&device) != cudaSuccess) { cudaGetLastError(); return SOLO_ECUDA; }
     unsigned char* scratch = nullptr;
-    rc = static_scratch(device, &scratch);
+    const int64_t* zero_origin = nullptr;
+    rc = static_scratch(device, &scratch, &zero_origin);
     if (rc) return rc;
     cudaStream_t stream = (cudaStream_t)stream_;
     // the tables below are copied from this call's stack: a captured copy would read a dead frame at replay
@@ -686,6 +725,8 @@ int solo_multi_step_static(int32_t num_tensors, void* const* param_dev, const vo
     a.tables = d_tables;
     a.tables_v = vtab ? d_tables_v : nullptr;
     a.status = d_status;
+    a.origin_id = (const int32_t*)zero_origin;
+    a.origin_ctr = zero_origin;
     reduce_hyper(hyper, step, block, a);
     a.param_list = param_dev;
     a.grad_list = grad_dev;

@@ -52,6 +52,11 @@ struct StepArgs {
     const float* tables;               // y[K], mid[K-1], inv_gap[K-1] of the first-moment codebook
     const float* tables_v;             // baseline second-moment codebook y[K], mid[K-1]; null: Eq. 6
     int* status;                       // device word: non-zero after a descriptor mismatch
+    // Position of every tensor of the list in the random stream (device arrays, never null; all zeros:
+    // "tensor t of the list is stream t, from its first element"): a shard of a larger tensor names the
+    // tensor's stream and the stream position (element index / 8) of the shard's first element.
+    const int32_t* origin_id;          // [T] stream number minus the tensor's position in the list
+    const int64_t* origin_ctr;         // [T]
     // hyper-parameters, already reduced to what the kernel multiplies with
     float beta1, beta2, omb1, omb2, step_size, inv_sqrt_bc2, eps, decay, weight_decay, p_quantile;
     float fixed_alpha;                 // in (0,1): base of every block; 0: base from the p-quantile
@@ -116,6 +121,18 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
         k1 += 0xBB67AE85u;
     }
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// The Philox stream of tensor `tensor` of the list and the counter of its first element.
+struct Origin {
+    uint32_t stream;
+    uint64_t ctr0;
+};
+__device__ __forceinline__ Origin origin_of(const StepArgs& a, int tensor) {
+    Origin o;
+    o.stream = (uint32_t)(tensor + __ldg(a.origin_id + tensor));
+    o.ctr0 = (uint64_t)__ldg(a.origin_ctr + tensor);
+    return o;
 }
 
 // 16-bit draw of element i (0..7) of a thread's eight: halfword i of the Philox block.
@@ -392,9 +409,10 @@ __global__ void __launch_bounds__(CTA) solo_step_kernel(const StepArgs a) {
         // ---- store parameters ----
         const bool sr = bf16p && a.param_sr;
         uint32_t wp[4] = {0u, 0u, 0u, 0u};
+        const Origin org = origin_of(a, tensor);
         if (sr) {
-            const uint64_t c = (uint64_t)e0 >> 3;
-            philox4x32_10((uint32_t)c, (uint32_t)(c >> 32), a.step32, (uint32_t)tensor * 4u + 2u,
+            const uint64_t c = org.ctr0 + ((uint64_t)e0 >> 3);
+            philox4x32_10((uint32_t)c, (uint32_t)(c >> 32), a.step32, org.stream * 4u + 2u,
                           a.seed_lo, a.seed_hi, wp);
         }
         if (vec) {
@@ -446,8 +464,8 @@ __global__ void __launch_bounds__(CTA) solo_step_kernel(const StepArgs a) {
             const float inv = 1.0f / dm_new;
             uint32_t wm[4];
             if (a.round_m) {
-                const uint64_t c = (uint64_t)e0 >> 3;             // one Philox block per 8 elements
-                philox4x32_10((uint32_t)c, (uint32_t)(c >> 32), a.step32, (uint32_t)tensor * 4u + 1u,
+                const uint64_t c = org.ctr0 + ((uint64_t)e0 >> 3);   // one Philox block per 8 elements
+                philox4x32_10((uint32_t)c, (uint32_t)(c >> 32), a.step32, org.stream * 4u + 1u,
                               a.seed_lo, a.seed_hi, wm);
             }
 #pragma unroll
@@ -504,8 +522,8 @@ __global__ void __launch_bounds__(CTA) solo_step_kernel(const StepArgs a) {
             const float inv_lambda = 1.0f / log2_sp(al_new);
             uint32_t wv[4];
             if (a.round_v) {
-                const uint64_t c = (uint64_t)e0 >> 3;
-                philox4x32_10((uint32_t)c, (uint32_t)(c >> 32), a.step32, (uint32_t)tensor * 4u,
+                const uint64_t c = org.ctr0 + ((uint64_t)e0 >> 3);
+                philox4x32_10((uint32_t)c, (uint32_t)(c >> 32), a.step32, org.stream * 4u,
                               a.seed_lo, a.seed_hi, wv);
             }
 #pragma unroll

@@ -699,11 +699,12 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
 
     // Adam(W) update of element i and, after every fourth, the store; issued between the
     // rounds of the selection below, which it does not depend on
-    const uint64_t ctr = (uint64_t)(uint32_t)tin * (TILE / EPT) + (uint32_t)tid;   // element index / 8
+    const Origin org = origin_of(a, tensor);
+    const uint64_t ctr = org.ctr0 + (uint64_t)(uint32_t)tin * (TILE / EPT) + (uint32_t)tid;   // position in the stream: element index / 8
     uint32_t wp[4] = {0u, 0u, 0u, 0u};                          // draws of the stochastic bf16 rounding
     const bool sr = PBF && a.param_sr;
     if (PBF && !FULL && sr)
-        philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, (uint32_t)tensor * 4u + 2u, a.rk, wp);
+        philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, org.stream * 4u + 2u, a.rk, wp);
     auto update = [&](int i) {
         if constexpr (PBF) {
             const float den = __fmaf_rn(__fsqrt_rn(vh[i]), a.inv_sqrt_bc2, a.eps);
@@ -712,7 +713,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
                 if (i == 7) {
                     uint32_t pp[4];
                     if (sr) {
-                        philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, (uint32_t)tensor * 4u + 2u, a.rk, wp);
+                        philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, org.stream * 4u + 2u, a.rk, wp);
 #pragma unroll
                         for (int j = 0; j < 4; ++j)
                             pp[j] = bf16_sr(p[2 * j], wp[j] & 0xFFFFu) | (bf16_sr(p[2 * j + 1], wp[j] >> 16) << 16);
@@ -804,7 +805,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
     bar_sync(1);
     uint32_t w[4] = {0u, 0u, 0u, 0u};
     if (warp != 0) {
-        if (round_v) philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, (uint32_t)tensor * 4u, a.rk, w);
+        if (round_v) philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, org.stream * 4u, a.rk, w);
     } else if (tid < NG) {
         const uint4 in = s.xin[par][tid];
         const float dm_new = __uint_as_float(in.x), dv_new = __uint_as_float(in.y);
@@ -828,7 +829,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
     }
     bar_sync(2);
     if (warp == 0 && round_v)
-        philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, (uint32_t)tensor * 4u, a.rk, w);
+        philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, org.stream * 4u, a.rk, w);
     float dr[EPT];                                               // the 16-bit draws d as binary32
 #pragma unroll
     for (int i = 0; i < 4; ++i) halves_to_float(w[i], dr[2 * i], dr[2 * i + 1]);

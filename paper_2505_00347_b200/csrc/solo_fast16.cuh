@@ -352,7 +352,15 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     // ---- (B) Adam(W) update, four (fp32) or eight (bf16) elements at a time ----
     // bf16 parameters: IEEE square root and division (see solo_fast.cuh), rounded to nearest even or
     // with the element's Philox draw (purpose 2, one block per eight elements)
-    const uint32_t ctr_lo = (uint32_t)tin * (TILE / 8) + 2u * (uint32_t)tid;   // element index / 8: even, below 2^32
+    // position of the thread's first element in the tensor's random stream (element index / 8): even,
+    // so the second group of eight never carries into the high word
+    auto stream_position = [&](uint32_t& lo, uint32_t& hi, uint32_t& c3) {
+        const Origin org = origin_of(a, tensor);
+        const uint64_t ctr = org.ctr0 + (uint64_t)((uint32_t)tin * (TILE / 8) + 2u * (uint32_t)tid);
+        lo = (uint32_t)ctr;
+        hi = (uint32_t)(ctr >> 32);
+        c3 = org.stream * 4u;
+    };
     if constexpr (!PBF) {
         // the thread's first eight elements (in its own order) at `sp[0]`, the others at `sp[1]`
         const unsigned char* const spb = st.p + 64 * tid;
@@ -396,8 +404,9 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
             }
             uint32_t pp[4];
             if (a.param_sr) {
-                uint32_t wp[4];
-                philox_rk(ctr_lo + he, 0u, a.step32, (uint32_t)tensor * 4u + 2u, a.rk, wp);
+                uint32_t wp[4], ctr_lo, ctr_hi, c3;
+                stream_position(ctr_lo, ctr_hi, c3);
+                philox_rk(ctr_lo + he, ctr_hi, a.step32, c3 + 2u, a.rk, wp);
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
                     pp[k] = bf16_sr(p[2 * k], wp[k] & 0xFFFFu) | (bf16_sr(p[2 * k + 1], wp[k] >> 16) << 16);
@@ -456,9 +465,11 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     uint32_t w[8];                                                // 16 halfwords: the draws of the 16 elements
     {
         // Philox4x32-10 on the counters of the thread's two groups of eight elements,
-        // (ctr_lo, 0, step, 4 * tensor) and (ctr_lo + 1, ...), in the thread's order; one round of both per call
-        uint32_t ca[4] = {ctr_lo + sw, 0u, a.step32, (uint32_t)tensor * 4u};
-        uint32_t cb[4] = {ctr_lo + (sw ^ 1u), 0u, a.step32, (uint32_t)tensor * 4u};
+        // (ctr, step, 4 * stream) and (ctr + 1, ...), in the thread's order; one round of both per call
+        uint32_t ctr_lo, ctr_hi, c3;
+        stream_position(ctr_lo, ctr_hi, c3);
+        uint32_t ca[4] = {ctr_lo + sw, ctr_hi, a.step32, c3};
+        uint32_t cb[4] = {ctr_lo + (sw ^ 1u), ctr_hi, a.step32, c3};
         auto philox_round = [&](int r) {
 #pragma unroll
             for (int b = 0; b < 2; ++b) {

@@ -56,3 +56,26 @@ def test_pack_helper_matches_oracle_layout():
     assert torch.all((st["alpha"] > 0) & (st["alpha"] < 1)) and torch.all(st["scale_v"] >= 0)
     again = synth.make_state((130, 64, 1), 2, 3, 64, seed=1)
     assert all(torch.equal(st[k], again[k]) for k in st)
+
+
+def test_partition_is_block_aligned_and_complete():
+    from paper_2505_00347_b200 import shard
+    sizes = (1, 129, 2048 * 3 + 5, 64, 128 * 7, 2047, 300)
+    for block in (64, 128, 2048):
+        nblk = [-(-n // block) for n in sizes]
+        for world in (1, 2, 3, 5, 8, 64):
+            parts = shard.partition(sizes, block, world)
+            assert len(parts) == world
+            counts = [sum(-(-p.numel // block) for p in r) for r in parts]
+            assert sum(counts) == sum(nblk) and max(counts) - min(counts) <= 1
+            seen = {t: [] for t in range(len(sizes))}
+            for r in parts:
+                for p in r:
+                    assert p.elem_offset % block == 0 and p.numel > 0
+                    seen[p.tensor].append((p.elem_offset, p.numel))
+            for t, n in enumerate(sizes):      # the pieces of a tensor tile it exactly, in order
+                pos = 0
+                for off, m in seen[t]:
+                    assert off == pos and (m % block == 0 or off + m == n)
+                    pos += m
+                assert pos == n
