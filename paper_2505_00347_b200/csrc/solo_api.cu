@@ -230,12 +230,15 @@ int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
     // worth its second launch only when there is work for many tiles per CTA (measured faster on the
     // 7B-shaped, the GPT-125M-shaped and the ragged set; a 1 Mi-element tensor is launch-bound)
     const bool large = s->tiles_total >= 8192;
-    if (streamlined && ((policy == 0 && large) || policy == 3) && s->block == 128 && plain && a.k_full == 13)
-        k16 = solo::fast16_kernel(s->bits_m, s->bits_v, a.param_bf16 != 0);
+    // p = 0.1: rank 7, 13, 26 of a block of 64, 128, 256
+    const bool rank16 = (s->block == 64 && a.k_full == 7) || (s->block == 128 && a.k_full == 13) ||
+                        (s->block == 256 && a.k_full == 26);
+    if (streamlined && ((policy == 0 && large) || policy == 3) && plain && rank16)
+        k16 = solo::fast16_kernel(s->bits_m, s->bits_v, s->block, a.param_bf16 != 0);
     if (k16) {
-        // blocks of 128, plain step: full tiles by the sixteen-per-thread kernel, whatever it leaves
+        // plain step: full tiles by the sixteen-per-thread kernel, whatever it leaves
         // (tails, tensors that are not 16-byte aligned) by the streamlined kernel
-        int rc = launch_kernel(k16, a, s->device, solo::CTA16, solo::fast16_kernel_smem(s->bits_m, s->bits_v, a.param_bf16 != 0), stream);
+        int rc = launch_kernel(k16, a, s->device, solo::CTA16, solo::fast16_kernel_smem(s->bits_m, s->bits_v, s->block, a.param_bf16 != 0), stream);
         if (rc) return rc;
         const bool all_full = !a.param_list && s->num_tensors == 1 && s->numel[0] % solo::TILE == 0;
         if (all_full) return SOLO_OK;

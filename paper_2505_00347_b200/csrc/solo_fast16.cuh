@@ -43,29 +43,34 @@ static_assert(CTA16 * EPT16 == TILE, "same tile as the other kernels");
 #define SOLO_F16_CTAS 7                 // resident CTAs per SM the fp32 kernel is compiled for
 #endif
 
-template <int BM, int BV, bool PBF>
+// G: lanes per block (4, 8 or 16 for blocks of 64, 128 or 256 elements); NG = 128 / G blocks per tile.
+template <int BM, int BV, bool PBF, int G>
 struct Fast16Shared {
+    static constexpr int NG = CTA16 / G;
+    static constexpr int ROUNDS = G == 4 ? 6 : G == 8 ? 12 : 25;   // rank of the p = 0.1 quantile minus one: 7, 13, 26
+    static constexpr int ROWS = ROUNDS < 15 ? ROUNDS : 16;         // G = 16: all fifteen further keys and a sentinel row
     // Sorted keys of the threads, one column per thread: row j holds the (j+2)-th smallest key.
-    // Twelve rounds of popping read rows 0..11 at most.
-    uint32_t sort[12][CTA16];
+    // The rounds of popping read rows 0..ROUNDS-1 at most; with 25 rounds a thread can run out of
+    // keys, and row 15 holds a sentinel above every key.
+    uint32_t sort[ROWS][CTA16];
     // per block: K_v second-moment levels alpha^k Delta_v and K_m first-moment levels y_k Delta_m.
     // Two arrays, so that the four blocks of a warp occupy distinct banks (up to eight levels).
-    float tab_v[16][1 << BV];
-    float tab_m[16][1 << BM];
+    float tab_v[NG][1 << BV];
+    float tab_m[NG][1 << BM];
     // Exchange with the first warp.  One copy is enough: xin is written before the tile's first
     // barrier and read between its two barriers, xout is written between the barriers and read
     // after the second, and nobody writes either again before passing those barriers.
-    uint4 xin[16];                       // per block: bits of Delta_m', Delta_v', x_p; .w != 0: the block's warp skips the tile
-    float4 xout[16];                     // per block: vanishing Delta_v' (1 or 0), 1/Delta_v', 1/log2(alpha'), rounding limit
+    uint4 xin[NG];                       // per block: bits of Delta_m', Delta_v', x_p; .w != 0: the block's warp skips the tile
+    float4 xout[NG];                     // per block: vanishing Delta_v' (1 or 0), 1/Delta_v', 1/log2(alpha'), rounding limit
     // per 3-bit moment and warp: the packed codes of the warp's 512 elements, for 128-bit stores
     static constexpr int N3 = (BM == 3 ? 1 : 0) + (BV == 3 ? 1 : 0);
     alignas(16) uint32_t cout[N3 > 0 ? N3 : 1][N3 > 0 ? 4 : 1][N3 > 0 ? 48 : 4];   // (a token array without 3-bit codes)
     struct Stage {
         alignas(16) unsigned char p[TILE * (PBF ? 2 : 4)];   // 2048 parameters
         alignas(16) unsigned char g[TILE * 2];                // 2048 bf16 gradients
-        uint32_t cm[64 * BM + 4];        // packed codes of the tile: 256 * bits bytes
+        uint32_t cm[64 * BM + 4];        // packed codes of the tile: 256 * bits bytes, from a 16-byte boundary
         uint32_t cv[64 * BV + 4];
-        float sc[3][16 + 4];             // Delta_m, Delta_v, alpha of the 16 blocks, from a 16-byte boundary
+        float sc[3][NG + 4];             // Delta_m, Delta_v, alpha of the tile's blocks, from a 16-byte boundary
     };
     alignas(16) Stage stage;
     alignas(8) unsigned long long mbar;
@@ -124,8 +129,14 @@ __device__ __forceinline__ void store_codes16(uint8_t* tile_codes, uint32_t* sta
         half[1] = (unsigned short)((h[0] >> 16) | (h[1] << 8));
         half[2] = (unsigned short)(h[1] >> 8);
         __syncwarp();
-        if (lane < 12)
-            __stcs(reinterpret_cast<uint4*>(tile_codes + warp * 192) + lane, reinterpret_cast<const uint4*>(stage)[lane]);
+        // the warp's 192 bytes: 128-bit words where the tile's codes start on a 16-byte boundary, else
+        // (3-bit codes of 64-element blocks, 24 bytes each, from an odd block on) 64-bit words
+        uint8_t* const dst = tile_codes + warp * 192;
+        if ((reinterpret_cast<uintptr_t>(tile_codes) & 15u) == 0) {
+            if (lane < 12) __stcs(reinterpret_cast<uint4*>(dst) + lane, reinterpret_cast<const uint4*>(stage)[lane]);
+        } else {
+            if (lane < 24) __stcs(reinterpret_cast<uint2*>(dst) + lane, reinterpret_cast<const uint2*>(stage)[lane]);
+        }
         __syncwarp();
     }
 }
@@ -160,54 +171,63 @@ __device__ constexpr unsigned char SORT16_PAIRS[62][2] = {
     {1, 9}, {5, 13}, {5, 9}, {3, 11}, {7, 15}, {7, 11}, {3, 5}, {7, 9}, {11, 13},
     {1, 2}, {3, 4}, {5, 6}, {7, 8}, {9, 10}, {11, 12}};
 
-// Minimum / maximum over the calling lane's group of eight lanes.  Three shuffle-and-compare steps
-// serve the warp's four groups at once; measured faster here than the full-mask reductions over a
-// transformed value that solo_fast.cuh uses for its groups of sixteen (four REDUX plus selects for
+// Minimum / maximum over the calling lane's group of G lanes.  The shuffle-and-compare steps serve
+// all groups of the warp at once; for groups of eight measured faster here than the full-mask reductions
+// over a transformed value that solo_fast.cuh uses for its groups of sixteen (four REDUX plus selects for
 // four groups): 294 vs 284 Gparams/s on the 7B set.
-__device__ __forceinline__ uint32_t group8_min(uint32_t x) {
+template <int G>
+__device__ __forceinline__ uint32_t group_min16(uint32_t x) {
 #pragma unroll
-    for (int d = 1; d < 8; d <<= 1) x = min(x, __shfl_xor_sync(0xffffffffu, x, d));
+    for (int d = 1; d < G; d <<= 1) x = min(x, __shfl_xor_sync(0xffffffffu, x, d));
     return x;
 }
-__device__ __forceinline__ uint32_t group8_max(uint32_t x) {
+template <int G>
+__device__ __forceinline__ uint32_t group_max16(uint32_t x) {
 #pragma unroll
-    for (int d = 1; d < 8; d <<= 1) x = max(x, __shfl_xor_sync(0xffffffffu, x, d));
+    for (int d = 1; d < G; d <<= 1) x = max(x, __shfl_xor_sync(0xffffffffu, x, d));
     return x;
 }
 
-// One selection round over groups of eight lanes, as pop_round in solo_fast.cuh (columns of
-// CTA16 words; at most twelve rounds, so no clamp; keys as they are, no transformed domain).
-template <bool LAST>
+// One selection round over groups of G lanes, as pop_round in solo_fast.cuh (columns of CTA16 words;
+// keys as they are, no transformed domain).  CLAMP: the offset stops at the sentinel row (needed when a
+// thread can be asked for more keys than it has).
+template <int G, bool LAST, bool CLAMP>
 __device__ __forceinline__ uint32_t pop_round16(uint32_t& head, int& off, const uint32_t* col, uint32_t le,
                                                 uint32_t self) {
-    const uint32_t tgt = group8_min(head);
+    const uint32_t tgt = group_min16<G>(head);
     if constexpr (LAST) return tgt;
     const uint32_t nxt = col[off];
     const uint32_t upto = __ballot_sync(0xffffffffu, head == tgt) & le;
     // if (upto == self) { head = nxt; off += CTA16; }
     asm("{\n\t.reg .pred p;\n\tsetp.eq.u32 p, %2, %3;\n\t@p mov.u32 %0, %4;\n\t@p add.s32 %1, %1, %5;\n\t}"
         : "+r"(head), "+r"(off) : "r"(upto), "r"(self), "r"(nxt), "n"(CTA16));
+    if constexpr (CLAMP) off = min(off, 15 * CTA16);
     return tgt;
 }
 
 // Bulk copies of one full tile's inputs into the stage (one thread; a bulk copy is a warp-wide
-// instruction, so copies issued by many lanes would be serialised lane by lane).  With blocks of 128
-// the tile's codes start on 16-byte boundaries (16 * bits bytes per block); the per-block scalars are
-// copied from the boundary at or below the first.
+// instruction, so copies issued by many lanes would be serialised lane by lane).  The per-block
+// scalars are copied from the 16-byte boundary at or below the first.
 // `extra_tx`: bytes announced on top of what is copied (test hook: the wait for this tile then runs out).
-template <int BM, int BV, bool PBF>
-__device__ __forceinline__ void issue_tile_copy16(const StepArgs& a, Fast16Shared<BM, BV, PBF>& s, const char* pt,
+template <int BM, int BV, bool PBF, int G>
+__device__ __forceinline__ void issue_tile_copy16(const StepArgs& a, Fast16Shared<BM, BV, PBF, G>& s, const char* pt,
                                                   const char* gt, int64_t jb_tile, uint32_t extra_tx) {
-    typename Fast16Shared<BM, BV, PBF>::Stage& st = s.stage;
+    constexpr int NG = CTA16 / G;
+    typename Fast16Shared<BM, BV, PBF, G>::Stage& st = s.stage;
     const uint32_t bar = smem_u32(&s.mbar);
-    const uint32_t bytes_s = (16u + ((jb_tile & 3) ? 4u : 0u)) * 4u;
+    // byte offsets of the tile's codes (2 * G * bits bytes per block); only 3-bit codes in blocks of 64
+    // (24 bytes) can start 8 bytes off a 16-byte boundary: they are copied from the boundary below, with
+    // 16 bytes more (the state's arrays carry that slack), and read with an offset
+    const int64_t bm0 = jb_tile * (2 * G * BM), bv0 = jb_tile * (2 * G * BV);
+    const uint32_t bytes_m = 256 * BM + ((bm0 & 15) ? 16u : 0u), bytes_v = 256 * BV + ((bv0 & 15) ? 16u : 0u);
+    const uint32_t bytes_s = (NG + ((jb_tile & 3) ? 4u : 0u)) * 4u;
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar),
-                 "r"((uint32_t)(TILE * (PBF ? 2 : 4) + TILE * 2 + 256 * BM + 256 * BV) + 3u * bytes_s + extra_tx)
+                 "r"((uint32_t)(TILE * (PBF ? 2 : 4) + TILE * 2) + bytes_m + bytes_v + 3u * bytes_s + extra_tx)
                  : "memory");
     bulk_copy(st.p, pt, TILE * (PBF ? 2 : 4), bar);
     bulk_copy(st.g, gt, TILE * 2, bar);
-    bulk_copy(st.cm, a.codes_m + jb_tile * (16 * BM), 256 * BM, bar);
-    bulk_copy(st.cv, a.codes_v + jb_tile * (16 * BV), 256 * BV, bar);
+    bulk_copy(st.cm, a.codes_m + (bm0 & ~(int64_t)15), bytes_m, bar);
+    bulk_copy(st.cv, a.codes_v + (bv0 & ~(int64_t)15), bytes_v, bar);
     const int64_t j0 = jb_tile & ~(int64_t)3;
     bulk_copy(st.sc[0], a.scale_m + j0, bytes_s, bar);
     bulk_copy(st.sc[1], a.scale_v + j0, bytes_s, bar);
@@ -252,13 +272,15 @@ __device__ __forceinline__ void block_scalars16(const StepArgs& a, Shared& s, co
 // known to all eight lanes after the maximum); (D) the sort and the selection rounds, with the Philox
 // rounds of the thread's two blocks of draws issued between them (they depend on nothing); (E) the
 // exchange with the first warp, the second moment's codes, the stores.
-template <int BM, int BV, bool PBF, bool DECAY>
-__device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, BV, PBF>& s, const float* s_y, const float* s_mid,
+template <int BM, int BV, bool PBF, int G, bool DECAY>
+__device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, BV, PBF, G>& s, const float* s_y, const float* s_mid,
                                             char* pbase, const char* gbase, const int tin, const int64_t jb_tile,
                                             const int tensor, Ahead16& ah, const bool next_full, const int64_t tile_no) {
-    constexpr int KM = 1 << BM, KV = 1 << BV, G = 8, NG = 16;     // 8 lanes per block, 16 blocks per tile
+    using Shared = Fast16Shared<BM, BV, PBF, G>;
+    constexpr int KM = 1 << BM, KV = 1 << BV, NG = Shared::NG;    // G lanes per block, NG blocks per tile
+    constexpr int ROUNDS = Shared::ROUNDS;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int gl = tid & (G - 1), grp = tid >> 3;
+    const int gl = tid & (G - 1), grp = tid / G;
     const uint32_t sw = ((uint32_t)tid >> 2) & 1u;               // 1: this thread takes elements 8..15 first (see the top of the file)
 
     const int64_t tile_elem0 = (int64_t)tin * TILE;
@@ -272,7 +294,7 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     // CTA's first full tile, or the first after a tensor change or a tile that was not full): every
     // thread has passed both barriers of the last tile that used the stage, so nobody reads it still.
     if (!ah.staged && tid == 0)
-        issue_tile_copy16<BM, BV, PBF>(a, s, pt, gt, jb_tile, tile_no + 1 == a.debug_stall_tile_p1 ? 16u : 0u);
+        issue_tile_copy16<BM, BV, PBF, G>(a, s, pt, gt, jb_tile, tile_no + 1 == a.debug_stall_tile_p1 ? 16u : 0u);
     const uint32_t mine = ah.fill;
     ah.fill += 1u;
     ah.staged = next_full;
@@ -287,21 +309,22 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
         if (gl == 0) s.xin[grp] = make_uint4(0u, 0u, 0u, 1u);
         bar_sync16(1);
         if (next_full && tid == 32)
-            issue_tile_copy16<BM, BV, PBF>(a, s, pt + TILE * PSZ, gt + TILE * 2, jb_tile + NG,
+            issue_tile_copy16<BM, BV, PBF, G>(a, s, pt + TILE * PSZ, gt + TILE * 2, jb_tile + NG,
                                            tile_no + 2 == a.debug_stall_tile_p1 ? 16u : 0u);
         if (tid < NG) block_scalars16<KV>(a, s, jb_tile, tid);
         bar_sync16(2);
         return;
     }
 
-    const typename Fast16Shared<BM, BV, PBF>::Stage& st = s.stage;
+    const typename Shared::Stage& st = s.stage;
     float mh[EPT16], vh[EPT16];
     uint32_t mx_v = 0;
     float mx_m_f = 0.0f;
     {
         uint32_t cm[2], cv[2];                                    // eight codes per word
-        load_codes16<BM>(st.cm, tid, sw, cm);
-        load_codes16<BV>(st.cv, tid, sw, cv);
+        // (word offsets of codes that do not start on a 16-byte boundary: 0 or 2, see issue_tile_copy16)
+        load_codes16<BM>(st.cm + ((int)((jb_tile * (2 * G * BM)) & 15) >> 2), tid, sw, cm);
+        load_codes16<BV>(st.cv + ((int)((jb_tile * (2 * G * BV)) & 15) >> 2), tid, sw, cv);
         const int so = (int)(jb_tile & 3) + grp;
         const float dm = st.sc[0][so], dv = st.sc[1][so], al = st.sc[2][so];
 
@@ -422,7 +445,7 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     }
 
     // ---- (C) first moment: block scale, nearest level (Eq. 1), see fast_tile ----
-    const uint32_t mx_m = group8_max(__float_as_uint(mx_m_f));
+    const uint32_t mx_m = group_max16<G>(__float_as_uint(mx_m_f));
     uint32_t om[2] = {0u, 0u};                                    // eight codes per word
     const float dm_new = __uint_as_float(mx_m);
     const float inv_m = __frcp_rn(dm_new);
@@ -460,7 +483,7 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     }
 
     // ---- (D) second moment: block scale and the p-quantile (k = 13 of 128); the draws of Eq. 6 ----
-    mx_v = group8_max(mx_v);
+    mx_v = group_max16<G>(mx_v);
     uint32_t x_p;
     uint32_t w[8];                                                // 16 halfwords: the draws of the 16 elements
     {
@@ -497,20 +520,24 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
         } else {
             sort16_low13(key);
         }
+        if constexpr (ROUNDS > 12) cswap(key[13], key[14]);     // all sixteen in order
         uint32_t* const col = &s.sort[0][tid];
+        constexpr int KEPT = ROUNDS < 15 ? ROUNDS : 15;           // keys after the smallest that can be asked for
 #pragma unroll
-        for (int j = 1; j <= 12; ++j) col[(j - 1) * CTA16] = key[j];
-        // twelve rounds pop the twelve smallest keys of the block, the thirteenth minimum is x_p
+        for (int j = 1; j <= KEPT; ++j) col[(j - 1) * CTA16] = key[j];
+        // ROUNDS rounds pop the ROUNDS smallest keys of the block, the next minimum is x_p
         const uint32_t self = 1u << lane;
-        const uint32_t le = (self | (self - 1u)) & (0xFFu << (lane & ~(G - 1)));
+        const uint32_t le = (self | (self - 1u)) & ((G == 32 ? 0xFFFFFFFFu : ((1u << G) - 1u)) << (lane & ~(G - 1)));
         uint32_t head = key[0];
         int off = 0;
 #pragma unroll
-        for (int r = 0; r < 12; ++r) {
-            pop_round16<false>(head, off, col, le, self);
+        for (int r = 0; r < ROUNDS; ++r) {
+            pop_round16<G, false, (ROUNDS > 15)>(head, off, col, le, self);
             if (r < 10) philox_round(r);
         }
-        x_p = pop_round16<true>(head, off, col, le, self);
+#pragma unroll
+        for (int r = ROUNDS; r < 10; ++r) philox_round(r);
+        x_p = pop_round16<G, true, false>(head, off, col, le, self);
 #pragma unroll
         for (int i = 0; i < 4; ++i) { w[i] = ca[i]; w[4 + i] = cb[i]; }
     }
@@ -520,7 +547,7 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     bar_sync16(1);
     // every thread has read what it needs from the stage
     if (next_full && tid == 32)
-        issue_tile_copy16<BM, BV, PBF>(a, s, pt + TILE * PSZ, gt + TILE * 2, jb_tile + NG,
+        issue_tile_copy16<BM, BV, PBF, G>(a, s, pt + TILE * PSZ, gt + TILE * 2, jb_tile + NG,
                                        tile_no + 2 == a.debug_stall_tile_p1 ? 16u : 0u);
     if (tid < NG) block_scalars16<KV>(a, s, jb_tile, tid);
     bar_sync16(2);
@@ -587,15 +614,16 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     // ---- store the codes ----
     const uint32_t om_e[2] = {sw ? om[1] : om[0], sw ? om[0] : om[1]};      // back to element order
     const uint32_t ov_e[2] = {sw ? ov[1] : ov[0], sw ? ov[0] : ov[1]};
-    store_codes16<BM>(a.codes_m + jb_tile * (16 * BM), s.cout[0][BM == 3 ? warp : 0], tid, om_e);
-    store_codes16<BV>(a.codes_v + jb_tile * (16 * BV), s.cout[(BM == 3 && BV == 3) ? 1 : 0][BV == 3 ? warp : 0], tid, ov_e);
+    store_codes16<BM>(a.codes_m + jb_tile * (2 * G * BM), s.cout[0][BM == 3 ? warp : 0], tid, om_e);
+    store_codes16<BV>(a.codes_v + jb_tile * (2 * G * BV), s.cout[(BM == 3 && BV == 3) ? 1 : 0][BV == 3 ? warp : 0], tid, ov_e);
 }
 
-template <int BM, int BV, bool PBF>
-__global__ void __launch_bounds__(CTA16, (PBF || BM != 2) ? 6 : SOLO_F16_CTAS) solo_step_fast16_kernel(const StepArgs a) {
+template <int BM, int BV, bool PBF, int G>
+__global__ void __launch_bounds__(CTA16, (PBF || BM != 2 || G == 16) ? 6 : SOLO_F16_CTAS) solo_step_fast16_kernel(const StepArgs a) {
     constexpr int KM = 1 << BM;
+    using Shared = Fast16Shared<BM, BV, PBF, G>;
     extern __shared__ __align__(16) unsigned char fast16_smem[];
-    Fast16Shared<BM, BV, PBF>& s = *reinterpret_cast<Fast16Shared<BM, BV, PBF>*>(fast16_smem);
+    Shared& s = *reinterpret_cast<Shared*>(fast16_smem);
     __shared__ float s_y[KM];
     __shared__ float s_mid[KM];
     const int tid = threadIdx.x;
@@ -603,6 +631,7 @@ __global__ void __launch_bounds__(CTA16, (PBF || BM != 2) ? 6 : SOLO_F16_CTAS) s
         s_y[tid] = a.tables[tid];
         if (tid < KM - 1) s_mid[tid] = a.tables[KM + tid];
     }
+    if constexpr (Shared::ROWS == 16) s.sort[15][tid] = KEY_MAX;   // never overwritten: rows 0..14 hold keys
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s.mbar)) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -642,9 +671,9 @@ __global__ void __launch_bounds__(CTA16, (PBF || BM != 2) ? 6 : SOLO_F16_CTAS) s
         if (skip || tin >= full_tiles) continue;
         const bool next_full = tin + 1 < full_tiles && tile + 1 < tile_end;
         if (decay)
-            fast16_tile<BM, BV, PBF, true>(a, s, s_y, s_mid, pbase, gbase, tin, jb0 + (int64_t)tin * 16, tensor, ah, next_full, tile);
+            fast16_tile<BM, BV, PBF, G, true>(a, s, s_y, s_mid, pbase, gbase, tin, jb0 + (int64_t)tin * Shared::NG, tensor, ah, next_full, tile);
         else
-            fast16_tile<BM, BV, PBF, false>(a, s, s_y, s_mid, pbase, gbase, tin, jb0 + (int64_t)tin * 16, tensor, ah, next_full, tile);
+            fast16_tile<BM, BV, PBF, G, false>(a, s, s_y, s_mid, pbase, gbase, tin, jb0 + (int64_t)tin * Shared::NG, tensor, ah, next_full, tile);
     }
     // A thread that gave up on a copy waits once more, again bounded, for the last one that was issued,
     // so that no copy is still writing to the stage when the CTA's shared memory is released.

@@ -1,14 +1,24 @@
-// The sixteen-elements-per-thread kernels: 2/3/4-bit states except 4-bit / 4-bit (measured slower
-// than the eight-per-thread kernel: 223 vs 236 Gparams/s), block 128, fp32 or bf16 parameters, plain
-// step.
+// The sixteen-elements-per-thread kernels for one block size (SOLO_G = 4, 8, 16 lanes per block:
+// blocks of 64, 128, 256 elements): 2/3/4-bit states except 4-bit / 4-bit (measured slower than the
+// eight-per-thread kernel: 210 vs 227 Gparams/s at block 128), fp32 or bf16 parameters, plain step.
 #include "solo_dispatch.h"
 #include "solo_fast16.cuh"
 
+#ifndef SOLO_G
+#error "compile with -DSOLO_G=4|8|16"
+#endif
+
+#define SOLO_CAT_(a, b) a##b
+#define SOLO_CAT(a, b) SOLO_CAT_(a, b)
+
 namespace solo {
 
-#define SOLO_K16(BM, BV) (param_bf16 ? solo_step_fast16_kernel<BM, BV, true> : solo_step_fast16_kernel<BM, BV, false>)
+#define SOLO_K16(BM, BV) \
+    (param_bf16 ? solo_step_fast16_kernel<BM, BV, true, SOLO_G> : solo_step_fast16_kernel<BM, BV, false, SOLO_G>)
+#define SOLO_S16(BM, BV) \
+    (param_bf16 ? sizeof(Fast16Shared<BM, BV, true, SOLO_G>) : sizeof(Fast16Shared<BM, BV, false, SOLO_G>))
 
-StepKernel fast16_kernel(int bits_m, int bits_v, bool param_bf16) {
+StepKernel SOLO_CAT(fast16_kernel_g, SOLO_G)(int bits_m, int bits_v, bool param_bf16) {
     switch (bits_m * 10 + bits_v) {
         case 22: return SOLO_K16(2, 2);
         case 23: return SOLO_K16(2, 3);
@@ -22,16 +32,16 @@ StepKernel fast16_kernel(int bits_m, int bits_v, bool param_bf16) {
     }
 }
 
-size_t fast16_kernel_smem(int bits_m, int bits_v, bool param_bf16) {
+size_t SOLO_CAT(fast16_smem_g, SOLO_G)(int bits_m, int bits_v, bool param_bf16) {
     switch (bits_m * 10 + bits_v) {
-        case 22: return param_bf16 ? sizeof(Fast16Shared<2, 2, true>) : sizeof(Fast16Shared<2, 2, false>);
-        case 23: return param_bf16 ? sizeof(Fast16Shared<2, 3, true>) : sizeof(Fast16Shared<2, 3, false>);
-        case 24: return param_bf16 ? sizeof(Fast16Shared<2, 4, true>) : sizeof(Fast16Shared<2, 4, false>);
-        case 32: return param_bf16 ? sizeof(Fast16Shared<3, 2, true>) : sizeof(Fast16Shared<3, 2, false>);
-        case 33: return param_bf16 ? sizeof(Fast16Shared<3, 3, true>) : sizeof(Fast16Shared<3, 3, false>);
-        case 34: return param_bf16 ? sizeof(Fast16Shared<3, 4, true>) : sizeof(Fast16Shared<3, 4, false>);
-        case 42: return param_bf16 ? sizeof(Fast16Shared<4, 2, true>) : sizeof(Fast16Shared<4, 2, false>);
-        case 43: return param_bf16 ? sizeof(Fast16Shared<4, 3, true>) : sizeof(Fast16Shared<4, 3, false>);
+        case 22: return SOLO_S16(2, 2);
+        case 23: return SOLO_S16(2, 3);
+        case 24: return SOLO_S16(2, 4);
+        case 32: return SOLO_S16(3, 2);
+        case 33: return SOLO_S16(3, 3);
+        case 34: return SOLO_S16(3, 4);
+        case 42: return SOLO_S16(4, 2);
+        case 43: return SOLO_S16(4, 3);
         default: return 0;
     }
 }

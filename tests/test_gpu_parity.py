@@ -83,7 +83,7 @@ def test_bits_and_blocks_random_state(bits_m, bits_v, block):
     hk = dict(lr=1e-3, beta1=0.8, beta2=0.999, weight_decay=0.01, seed=5)
     # block 128 with widths up to 4 bits: policy 3 is the sixteen-per-thread kernel plus the
     # streamlined kernel for the tails (policy 0 picks it for large sets only)
-    policies = (0, 3, 1) if block == 128 and max(bits_m, bits_v) <= 4 else (0, 1)
+    policies = (0, 3, 1) if block in (64, 128, 256) and max(bits_m, bits_v) <= 4 else (0, 1)
     # a random packed state pairs huge first moments with tiny second moments: update terms far above
     # the parameters themselves, where the faster kernels' quotient (a few 1e-7 of the term) shows
     rep = run_lockstep(sizes, bits_m, bits_v, block, hk, 2, gf, params, state0=st0, policies=policies,
@@ -175,7 +175,7 @@ def test_bf16_parameters_every_kernel(bits_m, bits_v, block, param_round):
               param_round=param_round)
     st0 = synth.make_state(sizes, bits_m, bits_v, block, seed=block + bits_m)
     # (2, 3, 128): policy 3 adds the sixteen-per-thread kernel (policy 0 uses it for large sets only)
-    policies = (0, 3, 1) if block == 128 and max(bits_m, bits_v) <= 4 else (0, 1)
+    policies = (0, 3, 1) if block in (64, 128, 256) and max(bits_m, bits_v) <= 4 else (0, 1)
     run_lockstep(sizes, bits_m, bits_v, block, hk, 2, gf, params, state0=st0, policies=policies)
     run_lockstep(sizes, bits_m, bits_v, block, hk, 3, gf, params, policies=policies)
 
@@ -217,6 +217,35 @@ def test_block_128_plain_step_all_three_kernels(bits_m, bits_v):
     w1 = synth.workload(1, sizes=(2048 * 6,))
     p1, g1 = _inputs(w1)
     run_lockstep(w1.sizes, bits_m, bits_v, 128, hk, 3, g1, p1, policies=(3, 2), multi=False)   # one launch: all tiles full
+
+
+@pytest.mark.parametrize("block", [64, 256])
+@pytest.mark.parametrize("bits_m,bits_v", [(2, 3), (2, 2), (3, 3), (4, 2), (3, 4), (4, 3)])
+def test_blocks_64_and_256_plain_step_all_three_kernels(bits_m, bits_v, block):
+    """The sixteen-per-thread kernel at the other two block sizes it exists for (four and sixteen
+    lanes per block: six and twenty-five selection rounds, 3-bit codes of 64-element blocks that start
+    off a 16-byte boundary, threads that run out of keys) against the streamlined and the general
+    kernel and one oracle run: many full tiles, tails, tiny tensors, ties and zero blocks."""
+    if block == 256 and bits_m != 2:
+        pytest.skip("at block 256 the sixteen-per-thread kernel is used with 2-bit first moments only")
+    sizes = (2048 * 9 + 700, 3, 2048 * 4, block * 3, 2048 + block, 127, 2048 * 2 + 1, block)
+    w = synth.workload(4, sizes=sizes)
+    params, gf = _inputs(w)
+    hk = dict(lr=2e-5, beta1=0.5, beta2=0.999, weight_decay=0.0, seed=4321)
+    st0 = synth.make_state(sizes, bits_m, bits_v, block, seed=6)
+    print(run_lockstep(sizes, bits_m, bits_v, block, hk, 3, gf, params, state0=st0, policies=(3, 2, 1),
+                       update_tol=RANDOM_STATE_TOL))
+    run_lockstep(sizes, bits_m, bits_v, block, hk, 4, gf, params, policies=(3, 2, 1))
+
+    def ties(t):                                # duplicated second moments: tied keys, one lane with most of the smallest
+        gs = [synth.make_grad(w, i, t) for i in range(len(sizes))]
+        m = gs[0][1::3].numel()
+        gs[0][0:3 * m:3] = gs[0][1::3]
+        gs[2][:16] = 0.0
+        gs[2][2048:2048 + 16] = 1e-30
+        return gs
+
+    run_lockstep(sizes, bits_m, bits_v, block, dict(hk, weight_decay=0.01), 3, ties, params, policies=(3, 2, 1))
 
 
 def test_streamlined_kernel_rounding_guard_is_sound():
@@ -293,7 +322,7 @@ def test_nan_and_inf_gradients_follow_one_rule(bits_m, bits_v, block):
             gs[0][4096:4096 + 128] = float("nan")   # a whole block of NaN
         return gs
 
-    policies = (3, 2, 1) if block == 128 and max(bits_m, bits_v) <= 4 else (0, 1)
+    policies = (3, 2, 1) if block in (64, 128, 256) and max(bits_m, bits_v) <= 4 else (0, 1)
     run_lockstep(sizes, bits_m, bits_v, block, dict(seed=9, weight_decay=0.0), 3, gf, params, policies=policies)
     # and on its own state for three steps: no hang, status clean, untouched blocks finite
     from paper_2505_00347_b200 import binding as B

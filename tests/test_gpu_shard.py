@@ -77,7 +77,8 @@ def _step_sharded(B, sizes, params, grads_fn, bm, bv, block, h, steps, st0, worl
     (2, 3, 128, dict(), (3, 2, 1)),
     (4, 4, 128, dict(round_m=1), (0,)),
     (2, 3, 128, dict(param_dtype=1, param_round=1), (3, 2, 1)),
-    (3, 2, 64, dict(), (0, 1)),
+    (3, 2, 64, dict(), (3, 0, 1)),
+    (2, 3, 256, dict(), (3, 0, 1)),
     (4, 2, 2048, dict(param_dtype=1, param_round=1), (0, 1)),
 ])
 def test_pieces_reproduce_the_whole(bm, bv, block, extra, policies):

@@ -46,7 +46,7 @@ def pad4(n):
 
 
 @pytest.mark.parametrize("bits_m,bits_v,block,policies", [
-    (2, 3, 128, (3, 2, 1)), (4, 4, 128, (3, 2, 1)), (3, 3, 64, (0, 1)), (4, 2, 256, (0, 1)),
+    (2, 3, 128, (3, 2, 1)), (4, 4, 128, (3, 2, 1)), (3, 3, 64, (3, 0, 1)), (4, 2, 256, (3, 0, 1)),
     (2, 2, 2048, (0, 1)), (8, 8, 128, (0, 1)), (3, 8, 64, (0, 1)),
 ])
 def test_nothing_is_written_outside_the_arrays(bits_m, bits_v, block, policies):
