@@ -42,7 +42,8 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per parameter of the step kernel from an ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum over the parameters of the captured launch, taken on
 # the first three tensors of the 7B-shaped set and scaled by the element count; see profiles/).
-# Valid for the 2-bit / 3-bit, block 128 streamlined kernel only; None for anything else.
+# Reported for that workload and kernel only (the LLaMA-7B-shaped set, 2-bit / 3-bit, block 128, default
+# kernel policy); null for anything else.
 NCU_TRAFFIC_BYTES_PER_PARAM = 11.11
 
 
@@ -260,8 +261,8 @@ def run_ours(args, rank, world):
                      "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
                      "traffic": (round(NCU_TRAFFIC_BYTES_PER_PARAM * n)
                                  if (NCU_TRAFFIC_BYTES_PER_PARAM is not None and args.policy == 0 and
-                                     not args.param_bf16 and not args.v_codebook and
-                                     (w.bits_m, w.bits_v, w.block) == (2, 3, 128)) else None)},
+                                     not args.param_bf16 and not args.v_codebook and not args.fixed_alpha and
+                                     w.cfg == 3 and (w.bits_m, w.bits_v, w.block) == (2, 3, 128)) else None)},
         "gpu_launches": int(launches),
         "clocks": clk,
     }
