@@ -294,16 +294,16 @@ __device__ __forceinline__ uint32_t warp_codes_finish(uint32_t w, int lane) {
     return __funnelshift_r(lo, hi, o) & 0xFFFFFFu;
 }
 template <int BITS>
-__device__ __forceinline__ void warp_store_codes(uint8_t* warp_base, int lane, uint32_t c, bool keep) {
+__device__ __forceinline__ void warp_store_codes(uint8_t* warp_base, int lane, uint32_t c) {
     if constexpr (BITS == 2) {
-        if (keep) __stcs(reinterpret_cast<unsigned short*>(warp_base) + lane, (unsigned short)c);
+        __stcs(reinterpret_cast<unsigned short*>(warp_base) + lane, (unsigned short)c);
     } else if constexpr (BITS == 4) {
-        if (keep) __stcs(reinterpret_cast<unsigned int*>(warp_base) + lane, c);
+        __stcs(reinterpret_cast<unsigned int*>(warp_base) + lane, c);
     } else {
         const int a = (4 * lane) / 3, o = 32 * lane - 24 * a;        // o in {0, 8, 16} for lane < 24
         const uint32_t lo = __shfl_sync(0xffffffffu, c, a & 31);
         const uint32_t hi = __shfl_sync(0xffffffffu, c, (a + 1) & 31);
-        if (lane < 24 && keep)
+        if (lane < 24)
             __stcs(reinterpret_cast<unsigned int*>(warp_base) + lane, (lo >> (o & 31)) | (hi << ((24 - o) & 31)));
     }
 }
@@ -553,7 +553,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
         ah.staged = next_full;
         if (!mbar_wait(smem_u32(&s.mbar[mine & 1u]), (mine >> 1) & 1u, ah.failed ? 1 : MBAR_POLLS)) {
             // the copy was never seen to arrive: flag it (solo_state_status reports bit 1); what the
-            // stage holds is worked on as it is, but nothing derived from it is stored (see `keep`)
+            // warp then leaves the tile alone (below)
             if (!ah.failed) atomicOr(a.status, 2);
             ah.failed = true;
         }
@@ -615,12 +615,45 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
         }
     }
 
-    // A warp in which any lane gave up waiting for its inputs stores nothing for this tile: parameters
-    // and state keep their old values.  Blocks of 2048 span the CTA, which then decides as a whole.
-    bool keep = true;
+    // Per-block scalars of the tile's blocks (one block per calling thread, tid < NG), from what the blocks'
+    // lanes left in xin: stores the new scales and base of the blocks whose warp did not skip the tile
+    // and leaves what the quantization needs in xout / xflag.
+    auto block_scalars = [&]() {
+        const uint4 in = s.xin[par][tid];
+        const float dm_new = __uint_as_float(in.x), dv_new = __uint_as_float(in.y);
+        const bool zero_m = dm_new < TINY, zero_v = dv_new < TINY;
+        const float inv_dm = 1.0f / dm_new;
+        const float inv_dv = 1.0f / dv_new;
+        const float rho = fminf(fmaxf(__uint_as_float(in.z) * inv_dv, RHO_MIN), RHO_MAX);
+        const float lam = log2_sp(rho) * (1.0f / (float)(KV - 1));
+        const float al_new = fixed_base ? a.fixed_alpha : exp2_sp(lam);
+        const float inv_lambda = 1.0f / log2_sp(al_new);
+        const float guard = __fmaf_rn(fabsf(inv_lambda), LG2_ABS, LG2_REL * (float)(KV + 1));
+        s.xout[par][tid] = make_float4(inv_dm, inv_dv, inv_lambda, 0.5f - guard);
+        s.xflag[par][tid] = (zero_m ? 1u : 0u) | (zero_v ? 2u : 0u);
+        const bool blk_exists = FULL || (int64_t)tid * B < rem_tile;
+        if (blk_exists && in.w == 0u) {
+            const int64_t j = jb_tile + tid;
+            a.scale_m[j] = zero_m ? 0.0f : dm_new;
+            a.scale_v[j] = zero_v ? 0.0f : dv_new;
+            a.alpha[j] = zero_v ? 0.5f : al_new;
+        }
+    };
+
+    // A warp in which any lane gave up waiting for its inputs leaves the tile alone: it stores nothing
+    // (parameters and state keep their old values), flags its blocks for the first warp and only keeps the
+    // CTA's two barriers and, if it is the first warp, the other warps' scalars going.  Blocks of 2048 span
+    // the CTA, which decides as a whole and has nothing to keep going.
     if (FULL) {
-        if constexpr (G == CTA) keep = !__syncthreads_or(ah.failed ? 1 : 0);
-        else keep = !__any_sync(0xffffffffu, ah.failed);
+        if constexpr (G == CTA) {
+            if (__syncthreads_or(ah.failed ? 1 : 0)) return;
+        } else if (__any_sync(0xffffffffu, ah.failed)) {
+            if (gl == 0) s.xin[par][grp] = make_uint4(0u, 0u, 0u, 1u);
+            bar_sync(1);
+            if (tid < NG) block_scalars();
+            bar_sync(2);
+            return;
+        }
     }
 
     // ---- per-block level tables: alpha^k Delta_v and y_k Delta_m (Eq. 2) ----
@@ -724,7 +757,7 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
                             pp[j] = *reinterpret_cast<const uint32_t*>(&h);
                         }
                     }
-                    if (keep) __stcs(reinterpret_cast<uint4*>(pt) + tid, make_uint4(pp[0], pp[1], pp[2], pp[3]));
+                    __stcs(reinterpret_cast<uint4*>(pt) + tid, make_uint4(pp[0], pp[1], pp[2], pp[3]));
                 }
             } else if (i < nv) {
                 reinterpret_cast<uint16_t*>(pt)[tid * EPT + i] =
@@ -739,8 +772,8 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
         const float q1 = __fmaf_rn(__fmaf_rn(-den, q0, mh[i]), rc, q0);
         p[i] = __fmaf_rn(-a.step_size, q1, p[i] * a.decay);
         if (FULL) {
-            if (i == 3 && keep) __stcs(reinterpret_cast<float4*>(pt) + 2 * tid, make_float4(p[0], p[1], p[2], p[3]));
-            if (i == 7 && keep) __stcs(reinterpret_cast<float4*>(pt) + 2 * tid + 1, make_float4(p[4], p[5], p[6], p[7]));
+            if (i == 3) __stcs(reinterpret_cast<float4*>(pt) + 2 * tid, make_float4(p[0], p[1], p[2], p[3]));
+            if (i == 7) __stcs(reinterpret_cast<float4*>(pt) + 2 * tid + 1, make_float4(p[4], p[5], p[6], p[7]));
         } else {
             if (i < nv) reinterpret_cast<float*>(pt)[tid * EPT + i] = p[i];
         }
@@ -801,31 +834,13 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
     }
 
     // ---- per-block scalars, once per block, by the first warp; the others draw xi meanwhile ----
-    if (gl == 0) s.xin[par][grp] = make_uint4(mx_m, mx_v, x_p, keep ? 0u : 1u);   // .w: the block's warp stores nothing
+    if (gl == 0) s.xin[par][grp] = make_uint4(mx_m, mx_v, x_p, 0u);   // .w != 0: the block's warp skipped the tile
     bar_sync(1);
     uint32_t w[4] = {0u, 0u, 0u, 0u};
     if (warp != 0) {
         if (round_v) philox_rk((uint32_t)ctr, (uint32_t)(ctr >> 32), a.step32, org.stream * 4u, a.rk, w);
     } else if (tid < NG) {
-        const uint4 in = s.xin[par][tid];
-        const float dm_new = __uint_as_float(in.x), dv_new = __uint_as_float(in.y);
-        const bool zero_m = dm_new < TINY, zero_v = dv_new < TINY;
-        const float inv_dm = 1.0f / dm_new;
-        const float inv_dv = 1.0f / dv_new;
-        const float rho = fminf(fmaxf(__uint_as_float(in.z) * inv_dv, RHO_MIN), RHO_MAX);
-        const float lam = log2_sp(rho) * (1.0f / (float)(KV - 1));
-        const float al_new = fixed_base ? a.fixed_alpha : exp2_sp(lam);
-        const float inv_lambda = 1.0f / log2_sp(al_new);
-        const float guard = __fmaf_rn(fabsf(inv_lambda), LG2_ABS, LG2_REL * (float)(KV + 1));
-        s.xout[par][tid] = make_float4(inv_dm, inv_dv, inv_lambda, 0.5f - guard);
-        s.xflag[par][tid] = (zero_m ? 1u : 0u) | (zero_v ? 2u : 0u);
-        const bool blk_exists = FULL || (int64_t)tid * B < rem_tile;
-        if (blk_exists && in.w == 0u) {
-            const int64_t j = jb_tile + tid;
-            a.scale_m[j] = zero_m ? 0.0f : dm_new;
-            a.scale_v[j] = zero_v ? 0.0f : dv_new;
-            a.alpha[j] = zero_v ? 0.5f : al_new;
-        }
+        block_scalars();
     }
     bar_sync(2);
     if (warp == 0 && round_v)
@@ -935,10 +950,10 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
 
     // ---- store the codes ----
     if (FULL) {
-        if constexpr (BM == 8) { if (keep) __stcs(reinterpret_cast<uint2*>(wcm) + lane, make_uint2(om, om_hi)); }
-        else warp_store_codes<BM>(wcm, lane, om, keep);
-        if constexpr (BV == 8) { if (keep) __stcs(reinterpret_cast<uint2*>(wcv) + lane, make_uint2(ov, ov_hi)); }
-        else warp_store_codes<BV>(wcv, lane, ov, keep);
+        if constexpr (BM == 8) __stcs(reinterpret_cast<uint2*>(wcm) + lane, make_uint2(om, om_hi));
+        else warp_store_codes<BM>(wcm, lane, om);
+        if constexpr (BV == 8) __stcs(reinterpret_cast<uint2*>(wcv) + lane, make_uint2(ov, ov_hi));
+        else warp_store_codes<BV>(wcv, lane, ov);
     } else if (have_block) {
         store_codes<BM>(wcm + lane * BM, ((uint64_t)om_hi << 32) | om);
         store_codes<BV>(wcv + lane * BV, ((uint64_t)ov_hi << 32) | ov);

@@ -1,13 +1,13 @@
-// Sixteen elements per thread: the streamlined step for the paper's default block size and
-// plain step (2/3/4-bit states, blocks of 128, fp32 or bf16 parameters; no L2 term in the gradient, no AdaBelief, base from the p = 0.1 quantile, xi
-// drawn).
+// Sixteen elements per thread: the streamlined step for the plain step (2/3/4-bit states, blocks of
+// 64, 128 or 256, fp32 or bf16 parameters; no L2 term in the gradient, no AdaBelief, base from the
+// p = 0.1 quantile, xi drawn).
 //
 // Same arithmetic, element for element, as solo_step_fast_kernel (solo_fast.cuh); what changes
 // is the work split.  A CTA of 128 threads owns a tile of 2048 consecutive elements, a thread
-// sixteen of them, a block of 128 elements eight consecutive lanes, a warp four blocks.  The
-// per-thread work that does not depend on the element count (waiting for the staged inputs,
-// addressing, the level tables, the exchange with the first warp, the rounds of the selection)
-// is spent once per sixteen elements instead of once per eight.
+// sixteen of them, a block of 64 / 128 / 256 elements G = 4 / 8 / 16 consecutive lanes, a warp eight,
+// four or two blocks.  The per-thread work that does not depend on the element count (waiting for the
+// staged inputs, addressing, the level tables, the exchange with the first warp, the rounds of the
+// selection) is spent once per sixteen elements instead of once per eight.
 //
 // Resources are cut for seven resident CTAs per SM (28 warps): at most 72 registers per thread
 // and one input stage of 13.6 KB (21.5 KB of shared memory in all).  The stage is read only
