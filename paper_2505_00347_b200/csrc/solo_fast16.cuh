@@ -39,6 +39,12 @@ static_assert(CTA16 * EPT16 == TILE, "same tile as the other kernels");
 #ifndef SOLO_F16_MIX
 #define SOLO_F16_MIX 1                  // 1: the first moment's codes are computed between the exchanges of the sort
 #endif
+#ifndef SOLO_F16_M3FMA
+#define SOLO_F16_M3FMA 1                // 3-bit first moments: seven saturated multiply-adds instead of a 3-step table search
+#endif
+#ifndef SOLO_F16_M4FMA
+#define SOLO_F16_M4FMA 1                // 4-bit first moments: two levels of three saturated multiply-adds
+#endif
 #ifndef SOLO_F16_CTAS
 #define SOLO_F16_CTAS 7                 // resident CTAs per SM the fp32 kernel is compiled for
 #endif
@@ -274,6 +280,7 @@ __device__ __forceinline__ void block_scalars16(const StepArgs& a, Shared& s, co
 // exchange with the first warp, the second moment's codes, the stores.
 template <int BM, int BV, bool PBF, int G, bool DECAY>
 __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, BV, PBF, G>& s, const float* s_y, const float* s_mid,
+                                            const float4* s_mid4,
                                             char* pbase, const char* gbase, const int tin, const int64_t jb_tile,
                                             const int tensor, Ahead16& ah, const bool next_full, const int64_t tile_no) {
     using Shared = Fast16Shared<BM, BV, PBF, G>;
@@ -453,6 +460,21 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     // (r - mid) * 2^100 on the FMA pipe (exactly 0 or 1, see fast_tile), accumulated in binary32
     constexpr float BIG = 0x1p100f;
     const float n0 = -s_mid[0] * BIG, n1 = -s_mid[1] * BIG, n2 = -s_mid[BM == 2 ? 2 : 1] * BIG;
+    constexpr bool M3_FMA = BM == 3 && SOLO_F16_M3FMA;           // 3-bit: all seven comparisons that way (24 bits per word: exact)
+    float n3[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    if constexpr (M3_FMA) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) n3[k] = -s_mid[3 + k] * BIG;
+    }
+    // 4-bit: the same comparisons in two levels of three: mid[3], mid[7], mid[11] give the quarter s of
+    // the codebook, the three midpoints inside it come from a table row addressed by s (s_mid4, scaled
+    // like n0..n2); code = 4 s + their count.  Four codes (16 bits) per binary32 accumulator.
+    constexpr bool M4_FMA = BM == 4 && SOLO_F16_M4FMA;
+    float nq[3] = {0.0f, 0.0f, 0.0f};
+    if constexpr (M4_FMA) {
+        nq[0] = -s_mid[3] * BIG; nq[1] = -s_mid[7] * BIG; nq[2] = -s_mid[11] * BIG;
+    }
+    float omf4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
     float omf[2] = {0.0f, 0.0f};
     auto quant_m = [&](int i) {                                   // call with i = 15, 14, ..., 0
         const float r = mh[i] * inv_m;
@@ -461,6 +483,25 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
             acc = __fmaf_rn(acc, 4.0f, __saturatef(__fmaf_rn(r, BIG, n0)));
             acc += __saturatef(__fmaf_rn(r, BIG, n1));
             acc += __saturatef(__fmaf_rn(r, BIG, n2));
+        } else if constexpr (M3_FMA) {
+            float& acc = omf[i >> 3];
+            acc = __fmaf_rn(acc, 8.0f, __saturatef(__fmaf_rn(r, BIG, n0)));
+            acc += __saturatef(__fmaf_rn(r, BIG, n1));
+            acc += __saturatef(__fmaf_rn(r, BIG, -s_mid[2] * BIG));
+#pragma unroll
+            for (int k = 0; k < 4; ++k) acc += __saturatef(__fmaf_rn(r, BIG, n3[k]));
+        } else if constexpr (M4_FMA) {
+            const float c0 = __saturatef(__fmaf_rn(r, BIG, nq[0]));
+            const float c1 = __saturatef(__fmaf_rn(r, BIG, nq[1]));
+            const float c2 = __saturatef(__fmaf_rn(r, BIG, nq[2]));
+            // 2^23 + 16 s: the low bits of the pattern are the byte offset of row s
+            const float t = __fmaf_rn(c2, 16.0f, __fmaf_rn(c1, 16.0f, __fmaf_rn(c0, 16.0f, 8388608.0f)));
+            const float4 row = *reinterpret_cast<const float4*>(reinterpret_cast<const char*>(s_mid4) + (__float_as_uint(t) & 0x30u));
+            const float sq = (c0 + c1) + c2;
+            float code = __fmaf_rn(sq, 4.0f, __saturatef(__fmaf_rn(r, BIG, row.x)));
+            code += __saturatef(__fmaf_rn(r, BIG, row.y));
+            code += __saturatef(__fmaf_rn(r, BIG, row.z));
+            omf4[i >> 2] = __fmaf_rn(omf4[i >> 2], 16.0f, code);
         } else {
             uint32_t q = 0;
 #pragma unroll
@@ -470,9 +511,13 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
         }
     };
     auto quant_m_done = [&]() {
-        if constexpr (BM == 2) {
+        if constexpr (BM == 2 || M3_FMA) {
             om[0] = (uint32_t)omf[0];
             om[1] = (uint32_t)omf[1];
+        }
+        if constexpr (M4_FMA) {
+            om[0] = (uint32_t)omf4[0] | ((uint32_t)omf4[1] << 16);
+            om[1] = (uint32_t)omf4[2] | ((uint32_t)omf4[3] << 16);
         }
         if (dm_new < TINY) { om[0] = 0; om[1] = 0; }             // vanishing block: all codes 0
     };
@@ -626,11 +671,15 @@ __global__ void __launch_bounds__(CTA16, (PBF || BM != 2 || G == 16) ? 6 : SOLO_
     Shared& s = *reinterpret_cast<Shared*>(fast16_smem);
     __shared__ float s_y[KM];
     __shared__ float s_mid[KM];
+    __shared__ float4 s_mid4[4];             // 4-bit first moments: per quarter of the codebook, its three inner midpoints times -2^100
     const int tid = threadIdx.x;
     if (tid < KM) {
         s_y[tid] = a.tables[tid];
         if (tid < KM - 1) s_mid[tid] = a.tables[KM + tid];
     }
+    if (BM == 4 && tid < 4)
+        s_mid4[tid] = make_float4(-a.tables[KM + 4 * tid] * 0x1p100f, -a.tables[KM + 4 * tid + 1] * 0x1p100f,
+                                  -a.tables[KM + 4 * tid + 2] * 0x1p100f, 0.0f);
     if constexpr (Shared::ROWS == 16) s.sort[15][tid] = KEY_MAX;   // never overwritten: rows 0..14 hold keys
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s.mbar)) : "memory");
@@ -671,9 +720,9 @@ __global__ void __launch_bounds__(CTA16, (PBF || BM != 2 || G == 16) ? 6 : SOLO_
         if (skip || tin >= full_tiles) continue;
         const bool next_full = tin + 1 < full_tiles && tile + 1 < tile_end;
         if (decay)
-            fast16_tile<BM, BV, PBF, G, true>(a, s, s_y, s_mid, pbase, gbase, tin, jb0 + (int64_t)tin * Shared::NG, tensor, ah, next_full, tile);
+            fast16_tile<BM, BV, PBF, G, true>(a, s, s_y, s_mid, s_mid4, pbase, gbase, tin, jb0 + (int64_t)tin * Shared::NG, tensor, ah, next_full, tile);
         else
-            fast16_tile<BM, BV, PBF, G, false>(a, s, s_y, s_mid, pbase, gbase, tin, jb0 + (int64_t)tin * Shared::NG, tensor, ah, next_full, tile);
+            fast16_tile<BM, BV, PBF, G, false>(a, s, s_y, s_mid, s_mid4, pbase, gbase, tin, jb0 + (int64_t)tin * Shared::NG, tensor, ah, next_full, tile);
     }
     // A thread that gave up on a copy waits once more, again bounded, for the last one that was issued,
     // so that no copy is still writing to the stage when the CTA's shared memory is released.

@@ -28,6 +28,7 @@ StepKernel SOLO_CAT(fast16_kernel_g, SOLO_G)(int bits_m, int bits_v, bool param_
         case 34: return SOLO_K16(3, 4);
         case 42: return SOLO_K16(4, 2);
         case 43: return SOLO_K16(4, 3);
+        case 44: return SOLO_K16(4, 4);
         default: return nullptr;
     }
 }
@@ -42,6 +43,7 @@ size_t SOLO_CAT(fast16_smem_g, SOLO_G)(int bits_m, int bits_v, bool param_bf16) 
         case 34: return SOLO_S16(3, 4);
         case 42: return SOLO_S16(4, 2);
         case 43: return SOLO_S16(4, 3);
+        case 44: return SOLO_S16(4, 4);
         default: return 0;
     }
 }
