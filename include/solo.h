@@ -289,8 +289,8 @@ float solo_default_beta1(int bits_m, int from_scratch);
  * Kernel selection.  0 (default): every width and block size with the logarithmic
  * second-moment quantizer, nearest rounding of the first moment and eps >= 1e-12 runs the
  * streamlined kernel (fp32 or bf16 parameters), everything else the general one; tensor sets of
- * at least 8192 tiles of 2048 elements with 2/3/4-bit states (other than 4-bit / 4-bit), blocks of
- * 64 or 128 (256 with 2-bit first moments) and the plain Adam(W) step with p = 0.1 run their
+ * at least 8192 tiles of 2048 elements with 2/3/4-bit states, blocks of 64, 128 or 256 and the
+ * plain Adam(W) step with p = 0.1 run their
  * full tiles in a kernel with sixteen elements per thread and the remaining tiles in the
  * streamlined kernel (two launches).  1: always the general kernel.  2: like 0 without the
  * sixteen-per-thread kernel.  3: like 0 with the sixteen-per-thread kernel whatever the tensor

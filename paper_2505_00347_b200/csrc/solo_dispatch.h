@@ -38,7 +38,7 @@ StepKernel fast_kernel_bm3(int bv_index, int block, bool param_bf16, bool plain)
 StepKernel fast_kernel_bm4(int bv_index, int block, bool param_bf16, bool plain);
 StepKernel fast_kernel_bm8(int bv_index, int block, bool param_bf16, bool plain);
 StepKernel fast_kernel(int bits_m, int bits_v, int block, bool param_bf16, bool plain);
-// Sixteen elements per thread: 2/3/4-bit states (not 4-bit / 4-bit), blocks of 64, 128 or 256, fp32 or
+// Sixteen elements per thread: 2/3/4-bit states, blocks of 64, 128 or 256, fp32 or
 // bf16 parameters, the plain step with p = 0.1; full tiles of aligned tensors only (the rest is left to a
 // launch of the streamlined kernel with StepArgs::only_partial).  Launched with CTA16 = 128 threads.
 // Null / 0 for other widths and block sizes.  One translation unit per block size.

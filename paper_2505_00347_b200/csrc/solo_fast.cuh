@@ -497,7 +497,7 @@ __device__ __forceinline__ void bar_sync(int id) {
 // carries the copy-ahead state; next_full / next_dtin describe the CTA's next tile.
 template <int BM, int BV, int G, bool FULL, bool PBF, bool PLAIN>
 __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>& s, const float* s_y,
-                                          const float* s_mid, char* pbase, const char* gbase,
+                                          const float* s_mid, const float4* s_mid4, char* pbase, const char* gbase,
                                           const int64_t n, const int tin, const int64_t jb_tile,
                                           const int tensor, const int par, Ahead& ah, const bool next_full,
                                           const int next_dtin, const int64_t tile_no) {
@@ -872,6 +872,45 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
                 omf += __saturatef(__fmaf_rn(r, BIG, n2));
             }
             om = (uint32_t)omf;
+        } else if constexpr (BM == 3 && FULL && G != CTA) {
+            // the same for all seven midpoints (measured faster than the 3-step table search, whose
+            // look-ups and compares run on the busier pipes, except with blocks of 2048, where the seven
+            // thresholds cost registers the CTA-wide select needs); eight 3-bit codes are 24 bits: exact in binary32
+            constexpr float BIG = 0x1p100f;
+            float n[7];
+#pragma unroll
+            for (int k = 0; k < 7; ++k) n[k] = -s_mid[k] * BIG;
+            float omf = 0.0f;
+#pragma unroll
+            for (int i = EPT - 1; i >= 0; --i) {
+                const float r = mh[i] * inv;
+                omf = __fmaf_rn(omf, 8.0f, __saturatef(__fmaf_rn(r, BIG, n[0])));
+#pragma unroll
+                for (int k = 1; k < 7; ++k) omf += __saturatef(__fmaf_rn(r, BIG, n[k]));
+            }
+            om = (uint32_t)omf;
+        } else if constexpr (BM == 4 && FULL) {
+            // two levels of three such comparisons: mid[3], mid[7], mid[11] give the quarter s of the
+            // codebook, the three midpoints inside it come from a table row addressed by s (s_mid4: the
+            // midpoints times -2^100); code = 4 s + their count.  Four codes (16 bits) per accumulator.
+            constexpr float BIG = 0x1p100f;
+            const float nq0 = -s_mid[3] * BIG, nq1 = -s_mid[7] * BIG, nq2 = -s_mid[11] * BIG;
+            float omf[2] = {0.0f, 0.0f};
+#pragma unroll
+            for (int i = EPT - 1; i >= 0; --i) {
+                const float r = mh[i] * inv;
+                const float c0 = __saturatef(__fmaf_rn(r, BIG, nq0));
+                const float c1 = __saturatef(__fmaf_rn(r, BIG, nq1));
+                const float c2 = __saturatef(__fmaf_rn(r, BIG, nq2));
+                // 2^23 + 16 s: the low bits of the pattern are the byte offset of row s
+                const float t = __fmaf_rn(c2, 16.0f, __fmaf_rn(c1, 16.0f, __fmaf_rn(c0, 16.0f, 8388608.0f)));
+                const float4 row = *reinterpret_cast<const float4*>(reinterpret_cast<const char*>(s_mid4) + (__float_as_uint(t) & 0x30u));
+                float code = __fmaf_rn((c0 + c1) + c2, 4.0f, __saturatef(__fmaf_rn(r, BIG, row.x)));
+                code += __saturatef(__fmaf_rn(r, BIG, row.y));
+                code += __saturatef(__fmaf_rn(r, BIG, row.z));
+                omf[i >> 2] = __fmaf_rn(omf[i >> 2], 16.0f, code);
+            }
+            om = (uint32_t)omf[0] | ((uint32_t)omf[1] << 16);
         } else if constexpr (BM == 2) {
             const float mid0 = s_mid[0], mid1 = s_mid[1], mid2 = s_mid[2];
 #pragma unroll
@@ -967,11 +1006,15 @@ __global__ void __launch_bounds__(CTA, (BM == 8 || BV == 8) ? 3 : 4) solo_step_f
     FastShared<BM, BV>& s = *reinterpret_cast<FastShared<BM, BV>*>(fast_smem);
     __shared__ float s_y[KM];
     __shared__ float s_mid[KM];
+    __shared__ float4 s_mid4[4];     // 4-bit first moments: per quarter of the codebook, its three inner midpoints times -2^100
     const int tid = threadIdx.x;
     for (int i = tid; i < KM; i += CTA) {
         s_y[i] = a.tables[i];
         if (i < KM - 1) s_mid[i] = a.tables[KM + i];
     }
+    if (BM == 4 && tid < 4)
+        s_mid4[tid] = make_float4(-a.tables[KM + 4 * tid] * 0x1p100f, -a.tables[KM + 4 * tid + 1] * 0x1p100f,
+                                  -a.tables[KM + 4 * tid + 2] * 0x1p100f, 0.0f);
     for (int r = 7; r < 16; ++r) s.sort[r][tid] = (G == 16 && (tid & G)) ? ~KEY_MAX : KEY_MAX;   // sentinels, v domain
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s.mbar[0])) : "memory");
@@ -1024,10 +1067,10 @@ __global__ void __launch_bounds__(CTA, (BM == 8 || BV == 8) ? 3 : 4) solo_step_f
         }
         const int64_t jb_tile = jb0 + (int64_t)tin * (CTA / G);
         if (tin < full_tiles)
-            fast_tile<BM, BV, G, true, PBF, PLAIN>(a, s, s_y, s_mid, pbase, gbase, 0, tin, jb_tile, tensor, par, ah,
+            fast_tile<BM, BV, G, true, PBF, PLAIN>(a, s, s_y, s_mid, s_mid4, pbase, gbase, 0, tin, jb_tile, tensor, par, ah,
                                        tin + step < full_tiles && tile + step < tile_end, step, tile);
         else
-            fast_tile<BM, BV, G, false, PBF, PLAIN>(a, s, s_y, s_mid, pbase, gbase, __ldg(a.numel + tensor), tin, jb_tile,
+            fast_tile<BM, BV, G, false, PBF, PLAIN>(a, s, s_y, s_mid, s_mid4, pbase, gbase, __ldg(a.numel + tensor), tin, jb_tile,
                                                     tensor, par, ah, false, 0, tile);
         par ^= 1;
     }

@@ -1,6 +1,5 @@
 // The sixteen-elements-per-thread kernels for one block size (SOLO_G = 4, 8, 16 lanes per block:
-// blocks of 64, 128, 256 elements): 2/3/4-bit states except 4-bit / 4-bit (measured slower than the
-// eight-per-thread kernel: 210 vs 227 Gparams/s at block 128), fp32 or bf16 parameters, plain step.
+// blocks of 64, 128, 256 elements): 2/3/4-bit states, fp32 or bf16 parameters, plain step.
 #include "solo_dispatch.h"
 #include "solo_fast16.cuh"
 

@@ -220,14 +220,12 @@ def test_block_128_plain_step_all_three_kernels(bits_m, bits_v):
 
 
 @pytest.mark.parametrize("block", [64, 256])
-@pytest.mark.parametrize("bits_m,bits_v", [(2, 3), (2, 2), (3, 3), (4, 2), (3, 4), (4, 3)])
+@pytest.mark.parametrize("bits_m,bits_v", [(2, 3), (2, 2), (3, 3), (4, 2), (3, 4), (4, 3), (4, 4)])
 def test_blocks_64_and_256_plain_step_all_three_kernels(bits_m, bits_v, block):
     """The sixteen-per-thread kernel at the other two block sizes it exists for (four and sixteen
     lanes per block: six and twenty-five selection rounds, 3-bit codes of 64-element blocks that start
     off a 16-byte boundary, threads that run out of keys) against the streamlined and the general
     kernel and one oracle run: many full tiles, tails, tiny tensors, ties and zero blocks."""
-    if block == 256 and bits_m != 2:
-        pytest.skip("at block 256 the sixteen-per-thread kernel is used with 2-bit first moments only")
     sizes = (2048 * 9 + 700, 3, 2048 * 4, block * 3, 2048 + block, 127, 2048 * 2 + 1, block)
     w = synth.workload(4, sizes=sizes)
     params, gf = _inputs(w)
