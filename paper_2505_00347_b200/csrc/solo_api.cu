@@ -233,10 +233,11 @@ int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
     // p = 0.1: rank 7, 13, 26 of a block of 64, 128, 256
     const bool rank16 = (s->block == 64 && a.k_full == 7) || (s->block == 128 && a.k_full == 13) ||
                         (s->block == 256 && a.k_full == 26);
-    if (streamlined && ((policy == 0 && large) || policy == 3) && plain && rank16)
-        k16 = solo::fast16_kernel(s->bits_m, s->bits_v, s->block, a.param_bf16 != 0);
+    // (a fixed base needs no quantile, so any p goes with it)
+    if (streamlined && ((policy == 0 && large) || policy == 3) && (rank16 || a.fixed_alpha > 0.0f))
+        k16 = solo::fast16_kernel(s->bits_m, s->bits_v, s->block, a.param_bf16 != 0, plain);
     if (k16) {
-        // plain step: full tiles by the sixteen-per-thread kernel, whatever it leaves
+        // full tiles by the sixteen-per-thread kernel, whatever it leaves
         // (tails, tensors that are not 16-byte aligned) by the streamlined kernel
         int rc = launch_kernel(k16, a, s->device, solo::CTA16, solo::fast16_kernel_smem(s->bits_m, s->bits_v, s->block, a.param_bf16 != 0), stream);
         if (rc) return rc;

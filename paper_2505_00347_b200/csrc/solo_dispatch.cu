@@ -30,11 +30,11 @@ StepKernel fast_kernel(int bits_m, int bits_v, int block, bool param_bf16, bool 
     }
 }
 
-StepKernel fast16_kernel(int bits_m, int bits_v, int block, bool param_bf16) {
+StepKernel fast16_kernel(int bits_m, int bits_v, int block, bool param_bf16, bool plain) {
     switch (block) {
-        case 64: return fast16_kernel_g4(bits_m, bits_v, param_bf16);
-        case 128: return fast16_kernel_g8(bits_m, bits_v, param_bf16);
-        case 256: return fast16_kernel_g16(bits_m, bits_v, param_bf16);   // twenty-five selection rounds: +0 to +11 % over the eight-per-thread kernel
+        case 64: return fast16_kernel_g4(bits_m, bits_v, param_bf16, plain);
+        case 128: return fast16_kernel_g8(bits_m, bits_v, param_bf16, plain);
+        case 256: return fast16_kernel_g16(bits_m, bits_v, param_bf16, plain);   // twenty-five selection rounds: +0 to +11 % over the eight-per-thread kernel
         default: return nullptr;
     }
 }

@@ -251,14 +251,15 @@ struct Ahead16 {
 // what the blocks' lanes left in xin: stores Delta_m', Delta_v', alpha' of the blocks whose warp did not
 // skip the tile and leaves what Eq. 6 needs in xout.
 template <int KV, class Shared>
-__device__ __forceinline__ void block_scalars16(const StepArgs& a, Shared& s, const int64_t jb_tile, const int tid) {
+__device__ __forceinline__ void block_scalars16(const StepArgs& a, Shared& s, const int64_t jb_tile, const int tid,
+                                                const bool fixed_base) {
     const uint4 in = s.xin[tid];
     const float dm_new = __uint_as_float(in.x), dv_new = __uint_as_float(in.y);
     const bool zero_m = dm_new < TINY, zero_v = dv_new < TINY;
     const float inv_dv = __frcp_rn(dv_new);
     const float rho = fminf(fmaxf(__uint_as_float(in.z) * inv_dv, RHO_MIN), RHO_MAX);
     const float lam = log2_sp(rho) * (1.0f / (float)(KV - 1));
-    const float al_new = exp2_sp(lam);
+    const float al_new = fixed_base ? a.fixed_alpha : exp2_sp(lam);
     const float inv_lambda = __frcp_rn(log2_sp(al_new));
     const float guard = __fmaf_rn(fabsf(inv_lambda), LG2_ABS, LG2_REL * (float)(KV + 1));
     s.xout[tid] = make_float4(zero_v ? 1.0f : 0.0f, inv_dv, inv_lambda, 0.5f - guard);
@@ -278,7 +279,7 @@ __device__ __forceinline__ void block_scalars16(const StepArgs& a, Shared& s, co
 // known to all eight lanes after the maximum); (D) the sort and the selection rounds, with the Philox
 // rounds of the thread's two blocks of draws issued between them (they depend on nothing); (E) the
 // exchange with the first warp, the second moment's codes, the stores.
-template <int BM, int BV, bool PBF, int G, bool DECAY>
+template <int BM, int BV, bool PBF, int G, bool DECAY, bool PLAIN>
 __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, BV, PBF, G>& s, const float* s_y, const float* s_mid,
                                             const float4* s_mid4,
                                             char* pbase, const char* gbase, const int tin, const int64_t jb_tile,
@@ -289,6 +290,11 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gl = tid & (G - 1), grp = tid / G;
     const uint32_t sw = ((uint32_t)tid >> 2) & 1u;               // 1: this thread takes elements 8..15 first (see the top of the file)
+    // PLAIN: the step of the paper as it stands (no L2 term in the gradient, no AdaBelief, base from the
+    // p-quantile, xi drawn); the other instantiation reads these modes from the arguments
+    const bool l2 = !PLAIN && a.l2, belief = !PLAIN && a.belief;
+    const bool fixed_base = !PLAIN && a.fixed_alpha > 0.0f;
+    const bool round_v = PLAIN || a.round_v;
 
     const int64_t tile_elem0 = (int64_t)tin * TILE;
     constexpr int PSZ = PBF ? 2 : 4;                              // bytes per parameter
@@ -318,7 +324,7 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
         if (next_full && tid == 32)
             issue_tile_copy16<BM, BV, PBF, G>(a, s, pt + TILE * PSZ, gt + TILE * 2, jb_tile + NG,
                                            tile_no + 2 == a.debug_stall_tile_p1 ? 16u : 0u);
-        if (tid < NG) block_scalars16<KV>(a, s, jb_tile, tid);
+        if (tid < NG) block_scalars16<KV>(a, s, jb_tile, tid, fixed_base);
         bar_sync16(2);
         return;
     }
@@ -365,14 +371,42 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
         for (int h = 0; h < 2; ++h) {
             const uint4 gw = *sg[h];
             const uint32_t gg[4] = {gw.x, gw.y, gw.z, gw.w};
+            float g8[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                g8[k] = __uint_as_float((k & 1) ? (gg[k >> 1] & 0xffff0000u) : (gg[k >> 1] << 16));
+            if (l2) {                                             // Adam: the decay term joins the gradient
+                float p8[8];
+                if constexpr (PBF) {
+                    const uint4 pw = reinterpret_cast<const uint4*>(st.p)[2 * tid + ((uint32_t)h ^ sw)];
+                    const uint32_t pin[4] = {pw.x, pw.y, pw.z, pw.w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        p8[2 * k] = __uint_as_float(pin[k] << 16);
+                        p8[2 * k + 1] = __uint_as_float(pin[k] & 0xffff0000u);
+                    }
+                } else {
+                    const float4* const ph = reinterpret_cast<const float4*>(st.p + 64 * tid + 32u * ((uint32_t)h ^ sw));
+                    const float4 pa = ph[0], pb = ph[1];
+                    p8[0] = pa.x; p8[1] = pa.y; p8[2] = pa.z; p8[3] = pa.w;
+                    p8[4] = pb.x; p8[5] = pb.y; p8[6] = pb.z; p8[7] = pb.w;
+                }
+#pragma unroll
+                for (int k = 0; k < 8; ++k) g8[k] = __fmaf_rn(a.weight_decay, p8[k], g8[k]);
+            }
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
                 const int i = 8 * h + k;
-                const float gi = __uint_as_float((k & 1) ? (gg[k >> 1] & 0xffff0000u) : (gg[k >> 1] << 16));
+                const float gi = g8[k];
                 const float mt = *reinterpret_cast<const float*>(tab_m + (BM == 2 ? om16(i) : i < 8 ? om4a(i) : om4b(i - 8)));
                 const float vt = *reinterpret_cast<const float*>(tab_v + (i < 8 ? ov4a(i) : ov4b(i - 8)));
                 mh[i] = __fmaf_rn(a.beta1, mt, a.omb1 * gi);
-                vh[i] = __fmaf_rn(a.beta2, vt, a.omb2 * (gi * gi));
+                if (belief) {                                     // AdaBelief: (g - m^)^2, plus eps
+                    const float sig = gi - mh[i];
+                    vh[i] = __fmaf_rn(a.beta2, vt, a.omb2 * (sig * sig)) + a.eps;
+                } else {
+                    vh[i] = __fmaf_rn(a.beta2, vt, a.omb2 * (gi * gi));
+                }
                 mx_m_f = max_abs_nan(mx_m_f, mh[i]);
                 mx_v = max(mx_v, __float_as_uint(vh[i]));
             }
@@ -552,37 +586,53 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
                 c[2] = n2;
             }
         };
-        uint32_t key[EPT16];
+        if (fixed_base) {
+            // every block keeps the given base: no quantile to find
+            if constexpr (SOLO_F16_MIX) {
 #pragma unroll
-        for (int i = 0; i < EPT16; ++i) key[i] = __float_as_uint(vh[i]);
-        if constexpr (SOLO_F16_MIX) {
-#pragma unroll
-            for (int k = 0; k < 62; ++k) {
-                cswap(key[SORT16_PAIRS[k][0]], key[SORT16_PAIRS[k][1]]);
-                if ((k & 3) == 3 || k == 61) quant_m(15 - (k >> 2));
+                for (int i = EPT16 - 1; i >= 0; --i) quant_m(i);
+                quant_m_done();
             }
-            quant_m_done();
+            if (round_v) {
+#pragma unroll
+                for (int r = 0; r < 10; ++r) philox_round(r);
+            }
+            x_p = 0u;
         } else {
-            sort16_low13(key);
+            uint32_t key[EPT16];
+#pragma unroll
+            for (int i = 0; i < EPT16; ++i) key[i] = __float_as_uint(vh[i]);
+            if constexpr (SOLO_F16_MIX) {
+#pragma unroll
+                for (int k = 0; k < 62; ++k) {
+                    cswap(key[SORT16_PAIRS[k][0]], key[SORT16_PAIRS[k][1]]);
+                    if ((k & 3) == 3 || k == 61) quant_m(15 - (k >> 2));
+                }
+                quant_m_done();
+            } else {
+                sort16_low13(key);
+            }
+            if constexpr (ROUNDS > 12) cswap(key[13], key[14]); // all sixteen in order
+            uint32_t* const col = &s.sort[0][tid];
+            constexpr int KEPT = ROUNDS < 15 ? ROUNDS : 15;       // keys after the smallest that can be asked for
+#pragma unroll
+            for (int j = 1; j <= KEPT; ++j) col[(j - 1) * CTA16] = key[j];
+            // ROUNDS rounds pop the ROUNDS smallest keys of the block, the next minimum is x_p
+            const uint32_t self = 1u << lane;
+            const uint32_t le = (self | (self - 1u)) & ((G == 32 ? 0xFFFFFFFFu : ((1u << G) - 1u)) << (lane & ~(G - 1)));
+            uint32_t head = key[0];
+            int off = 0;
+#pragma unroll
+            for (int r = 0; r < ROUNDS; ++r) {
+                pop_round16<G, false, (ROUNDS > 15)>(head, off, col, le, self);
+                if (r < 10 && round_v) philox_round(r);
+            }
+            if (round_v) {
+#pragma unroll
+                for (int r = ROUNDS; r < 10; ++r) philox_round(r);
+            }
+            x_p = pop_round16<G, true, false>(head, off, col, le, self);
         }
-        if constexpr (ROUNDS > 12) cswap(key[13], key[14]);     // all sixteen in order
-        uint32_t* const col = &s.sort[0][tid];
-        constexpr int KEPT = ROUNDS < 15 ? ROUNDS : 15;           // keys after the smallest that can be asked for
-#pragma unroll
-        for (int j = 1; j <= KEPT; ++j) col[(j - 1) * CTA16] = key[j];
-        // ROUNDS rounds pop the ROUNDS smallest keys of the block, the next minimum is x_p
-        const uint32_t self = 1u << lane;
-        const uint32_t le = (self | (self - 1u)) & ((G == 32 ? 0xFFFFFFFFu : ((1u << G) - 1u)) << (lane & ~(G - 1)));
-        uint32_t head = key[0];
-        int off = 0;
-#pragma unroll
-        for (int r = 0; r < ROUNDS; ++r) {
-            pop_round16<G, false, (ROUNDS > 15)>(head, off, col, le, self);
-            if (r < 10) philox_round(r);
-        }
-#pragma unroll
-        for (int r = ROUNDS; r < 10; ++r) philox_round(r);
-        x_p = pop_round16<G, true, false>(head, off, col, le, self);
 #pragma unroll
         for (int i = 0; i < 4; ++i) { w[i] = ca[i]; w[4 + i] = cb[i]; }
     }
@@ -594,7 +644,7 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     if (next_full && tid == 32)
         issue_tile_copy16<BM, BV, PBF, G>(a, s, pt + TILE * PSZ, gt + TILE * 2, jb_tile + NG,
                                        tile_no + 2 == a.debug_stall_tile_p1 ? 16u : 0u);
-    if (tid < NG) block_scalars16<KV>(a, s, jb_tile, tid);
+    if (tid < NG) block_scalars16<KV>(a, s, jb_tile, tid, fixed_base);
     bar_sync16(2);
     const float4 sc = s.xout[grp];
 
@@ -606,8 +656,9 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
         constexpr float MAGIC = 12582912.0f;
         constexpr uint32_t MAGIC_BITS = 0x4B400000u;
         const float ils = il * (1.0f / KM1);
-        const float xs1 = (float)(0x1p-16 / (KV - 1));
-        const float xs0 = (float)((-0.5 + 0x1p-17) / (KV - 1));
+        // xi = (d + 1/2) / 2^16 - 1/2 (exact), scaled like t; zero without the dither
+        const float xs1 = round_v ? (float)(0x1p-16 / (KV - 1)) : 0.0f;
+        const float xs0 = round_v ? (float)((-0.5 + 0x1p-17) / (KV - 1)) : 0.0f;
         float worst = 0.0f;
         uint32_t acc[2] = {0u, 0u};
 #pragma unroll
@@ -632,7 +683,7 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
         if (__any_sync(0xffffffffu, worst > lim)) {
             // too close to a rounding boundary for the approximate logarithm somewhere in the warp:
             // the exact sequence for all sixteen
-            const float x1 = 0x1p-16f, x0 = -0.5f + 0x1p-17f;
+            const float x1 = round_v ? 0x1p-16f : 0.0f, x0 = round_v ? -0.5f + 0x1p-17f : 0.0f;
             ov[0] = 0;
             ov[1] = 0;
 #pragma unroll
@@ -663,8 +714,8 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     store_codes16<BV>(a.codes_v + jb_tile * (2 * G * BV), s.cout[(BM == 3 && BV == 3) ? 1 : 0][BV == 3 ? warp : 0], tid, ov_e);
 }
 
-template <int BM, int BV, bool PBF, int G>
-__global__ void __launch_bounds__(CTA16, (PBF || BM != 2 || G == 16) ? 6 : SOLO_F16_CTAS) solo_step_fast16_kernel(const StepArgs a) {
+template <int BM, int BV, bool PBF, int G, bool PLAIN>
+__global__ void __launch_bounds__(CTA16, (PBF || BM != 2 || G == 16 || !PLAIN) ? 6 : SOLO_F16_CTAS) solo_step_fast16_kernel(const StepArgs a) {
     constexpr int KM = 1 << BM;
     using Shared = Fast16Shared<BM, BV, PBF, G>;
     extern __shared__ __align__(16) unsigned char fast16_smem[];
@@ -720,9 +771,9 @@ __global__ void __launch_bounds__(CTA16, (PBF || BM != 2 || G == 16) ? 6 : SOLO_
         if (skip || tin >= full_tiles) continue;
         const bool next_full = tin + 1 < full_tiles && tile + 1 < tile_end;
         if (decay)
-            fast16_tile<BM, BV, PBF, G, true>(a, s, s_y, s_mid, s_mid4, pbase, gbase, tin, jb0 + (int64_t)tin * Shared::NG, tensor, ah, next_full, tile);
+            fast16_tile<BM, BV, PBF, G, true, PLAIN>(a, s, s_y, s_mid, s_mid4, pbase, gbase, tin, jb0 + (int64_t)tin * Shared::NG, tensor, ah, next_full, tile);
         else
-            fast16_tile<BM, BV, PBF, G, false>(a, s, s_y, s_mid, s_mid4, pbase, gbase, tin, jb0 + (int64_t)tin * Shared::NG, tensor, ah, next_full, tile);
+            fast16_tile<BM, BV, PBF, G, false, PLAIN>(a, s, s_y, s_mid, s_mid4, pbase, gbase, tin, jb0 + (int64_t)tin * Shared::NG, tensor, ah, next_full, tile);
     }
     // A thread that gave up on a copy waits once more, again bounded, for the last one that was issued,
     // so that no copy is still writing to the stage when the CTA's shared memory is released.

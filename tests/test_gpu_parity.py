@@ -108,7 +108,9 @@ def test_mode_flags_at_other_widths(bits_m, bits_v, block, hk):
     base = dict(lr=1e-3, beta1=0.6, beta2=0.999, weight_decay=0.01, seed=13)
     base.update(hk)
     st0 = synth.make_state(sizes, bits_m, bits_v, block, seed=19)
-    print(run_lockstep(sizes, bits_m, bits_v, block, base, 2, gf, params, state0=st0, update_tol=RANDOM_STATE_TOL))
+    # policy 3: the sixteen-per-thread kernel's instantiation that reads the modes (where it exists)
+    print(run_lockstep(sizes, bits_m, bits_v, block, base, 2, gf, params, state0=st0, update_tol=RANDOM_STATE_TOL,
+                       policies=(0, 3, 1)))
 
 
 @pytest.mark.parametrize("hk", [
@@ -140,10 +142,11 @@ def test_hyper_parameter_modes(hk):
     base = dict(lr=1e-3, beta1=0.8, beta2=0.999, weight_decay=0.01, seed=3)
     base.update(hk)
     st0 = synth.make_state(sizes, 4, 3, 128, seed=17)
-    print(run_lockstep(sizes, 4, 3, 128, base, 3, gf, params, state0=st0, update_tol=RANDOM_STATE_TOL))
+    print(run_lockstep(sizes, 4, 3, 128, base, 3, gf, params, state0=st0, update_tol=RANDOM_STATE_TOL,
+                       policies=(0, 3, 1)))
     # from the zero state the plain bar holds, except at a learning rate of 0.1 (updates of the
     # parameters' own size)
-    print(run_lockstep(sizes, 4, 3, 128, base, 3, gf, params,
+    print(run_lockstep(sizes, 4, 3, 128, base, 3, gf, params, policies=(0, 3, 1),
                        update_tol=RANDOM_STATE_TOL if base["lr"] > 1e-2 else 0.0))
 
 
