@@ -153,7 +153,7 @@ def run_ours(args, rank, world):
         state.set_origin([rank * len(w.sizes) + t for t in range(len(w.sizes))], None)
     ts = B.TensorSet(params, grads, state)
     h = B.hyper(lr=w.lr, beta1=w.beta1, beta2=w.beta2, weight_decay=w.weight_decay, seed=1234,
-                fixed_alpha=args.fixed_alpha, v_codebook=args.v_codebook,
+                fixed_alpha=args.fixed_alpha, v_codebook=args.v_codebook, round_m=args.round_m,
                 param_dtype=1 if args.param_bf16 else 0, param_round=1 if args.param_bf16 == 2 else 0)
     n = w.numel
     step_no = 0
@@ -251,7 +251,8 @@ def run_ours(args, rank, world):
                                f"{' (stochastic rounding)' if args.param_bf16 == 2 else ''}, bf16 grads, "
                                "one solo_multi_step call per step"
                                + (f", fixed base {args.fixed_alpha}" if args.fixed_alpha else "")
-                               + (f", baseline v codebook {args.v_codebook}" if args.v_codebook else ""),
+                               + (f", baseline v codebook {args.v_codebook}" if args.v_codebook else "")
+                               + (", first moment rounded stochastically (Eq. 5)" if args.round_m else ""),
                    "l2": "working set (params+grads+state) far larger than the 126 MB L2; no flush needed"
                          if n * abytes > 1e9 else "working set fits L2: launch-bound point, not a bandwidth point",
                    "bytes_per_param": round(abytes, 4),
@@ -261,7 +262,7 @@ def run_ours(args, rank, world):
                      "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
                      "traffic": (round(NCU_TRAFFIC_BYTES_PER_PARAM * n)
                                  if (NCU_TRAFFIC_BYTES_PER_PARAM is not None and args.policy == 0 and
-                                     not args.param_bf16 and not args.v_codebook and not args.fixed_alpha and
+                                     not args.param_bf16 and not args.v_codebook and not args.fixed_alpha and not args.round_m and
                                      w.cfg == 3 and (w.bits_m, w.bits_v, w.block) == (2, 3, 128)) else None)},
         "gpu_launches": int(launches),
         "clocks": clk,
@@ -357,6 +358,8 @@ def main():
                     help="fixed base of the logarithmic codebook (no quantile step); 0 = the paper's quantile rule")
     ap.add_argument("--v-codebook", type=int, default=0, choices=[0, 1, 2, 3],
                     help="second-moment quantizer: 0 SOLO (default), 1 unsigned DE, 2 linear, 3 linear without zero")
+    ap.add_argument("--round-m", type=int, default=0, choices=[0, 1],
+                    help="first moment: 0 nearest level (Eq. 1, default), 1 stochastic rounding (Eq. 5)")
     ap.add_argument("--param-bf16", type=int, default=0, choices=[0, 1, 2],
                     help="bf16 parameters: 1 nearest-even, 2 stochastic rounding (default 0: fp32)")
     ap.add_argument("--cpu-sample", type=int, default=1 << 27)

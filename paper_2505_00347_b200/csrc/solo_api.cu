@@ -223,9 +223,11 @@ int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
     a.debug_stall_tile_p1 = g_stall_tile_p1.exchange(0, std::memory_order_relaxed);
     const bool cta_group = s->block == 2048;
     const int policy = g_policy.load(std::memory_order_relaxed);
-    const bool streamlined = policy != 1 && !a.round_m && !a.tables_v && a.eps >= 1e-12f &&
-                             s->tiles_total < ((int64_t)1 << 31) - ((int64_t)1 << 20);   // 32-bit tile arithmetic with headroom
-    const bool plain = !a.l2 && !a.belief && a.fixed_alpha == 0.0f && a.round_v;
+    const bool fast_ok = policy != 1 && a.eps >= 1e-12f &&
+                         s->tiles_total < ((int64_t)1 << 31) - ((int64_t)1 << 20);   // 32-bit tile arithmetic with headroom
+    // the eight-per-thread streamlined kernel has neither the baseline second-moment codebooks nor Eq. 5
+    const bool streamlined = fast_ok && !a.tables_v && !a.round_m;
+    const bool plain = !a.l2 && !a.belief && a.fixed_alpha == 0.0f && a.round_v && !a.tables_v && !a.round_m;
     solo::StepKernel k16 = nullptr;
     // worth its second launch only when there is work for many tiles per CTA (measured faster on the
     // 7B-shaped, the GPT-125M-shaped and the ragged set; a 1 Mi-element tensor is launch-bound)
@@ -233,12 +235,12 @@ int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
     // p = 0.1: rank 7, 13, 26 of a block of 64, 128, 256
     const bool rank16 = (s->block == 64 && a.k_full == 7) || (s->block == 128 && a.k_full == 13) ||
                         (s->block == 256 && a.k_full == 26);
-    // (a fixed base needs no quantile, so any p goes with it)
-    if (streamlined && ((policy == 0 && large) || policy == 3) && (rank16 || a.fixed_alpha > 0.0f))
+    // (a fixed base or a baseline codebook needs no quantile, so any p goes with them)
+    if (fast_ok && ((policy == 0 && large) || policy == 3) && (rank16 || a.fixed_alpha > 0.0f || a.tables_v))
         k16 = solo::fast16_kernel(s->bits_m, s->bits_v, s->block, a.param_bf16 != 0, plain);
     if (k16) {
-        // full tiles by the sixteen-per-thread kernel, whatever it leaves
-        // (tails, tensors that are not 16-byte aligned) by the streamlined kernel
+        // full tiles by the sixteen-per-thread kernel, whatever it leaves (tails, tensors that are
+        // not 16-byte aligned) by the streamlined kernel, or by the general one where that has no path
         int rc = launch_kernel(k16, a, s->device, solo::CTA16, solo::fast16_kernel_smem(s->bits_m, s->bits_v, s->block, a.param_bf16 != 0), stream);
         if (rc) return rc;
         const bool all_full = !a.param_list && s->num_tensors == 1 && s->numel[0] % solo::TILE == 0;

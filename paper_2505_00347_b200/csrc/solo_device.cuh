@@ -40,7 +40,7 @@ struct StepArgs {
     int32_t num_tensors;
     int64_t total_tiles;               // the launch covers tiles [tile_first, total_tiles)
     int64_t tile_first;
-    int32_t only_partial;              // streamlined kernel: skip full tiles of aligned tensors (another launch did them)
+    int32_t only_partial;              // streamlined and general kernel: skip full tiles of aligned tensors (another launch did them)
     int64_t debug_stall_tile_p1;       // test hook of the staged kernels: 1 + the number of the tile whose input copy
                                        // announces 16 bytes more than it brings (the wait for it runs out); 0: none
     // state
@@ -325,14 +325,30 @@ __global__ void __launch_bounds__(CTA) solo_step_kernel(const StepArgs a) {
     const int gl = tid & (G - 1);                              // thread within its block
     const bool bf16p = a.param_bf16 != 0;
 
-    for (int64_t tile = a.tile_first + blockIdx.x; tile < a.total_tiles; tile += gridDim.x) {
+    // Tiles are dealt out in turn.  After a launch that did the full tiles of the aligned tensors
+    // (only_partial) a CTA takes a contiguous share instead and jumps over each tensor's full tiles, so
+    // that it visits a few tiles per tensor of its share rather than every tile of the launch.
+    const int64_t share = (a.total_tiles - a.tile_first + gridDim.x - 1) / gridDim.x;
+    const int64_t tile_begin = a.only_partial ? min(a.tile_first + (int64_t)blockIdx.x * share, a.total_tiles)
+                                              : a.tile_first + blockIdx.x;
+    const int64_t tile_end = a.only_partial ? min(tile_begin + share, a.total_tiles) : a.total_tiles;
+    const int64_t stride = a.only_partial ? 1 : (int64_t)gridDim.x;
+    for (int64_t tile = tile_begin; tile < tile_end; tile += stride) {
         const int tensor = a.num_tensors > 1 ? find_tensor(a.tile_start, a.num_tensors, tile) : 0;
         const int64_t n = __ldg(a.numel + tensor);
         if (a.numel_check != nullptr && __ldg(a.numel_check + tensor) != n) {
             if (tid == 0) atomicOr(a.status, 1);
             continue;
         }
-        const int64_t e0 = (tile - __ldg(a.tile_start + tensor)) * TILE + (int64_t)tid * EPT;
+        const int64_t tin = tile - __ldg(a.tile_start + tensor);
+        char* pbase = (char*)(a.param_list ? a.param_list[tensor] : a.param_single);
+        const char* gbase = (const char*)(a.grad_list ? a.grad_list[tensor] : a.grad_single);
+        const bool aligned = ((((uintptr_t)pbase) | ((uintptr_t)gbase)) & 15u) == 0;
+        if (a.only_partial && aligned && tin < n / TILE) {           // another launch did the full tiles:
+            tile += n / TILE - tin - 1;                               // on to the tensor's first tile that is not full
+            continue;
+        }
+        const int64_t e0 = tin * TILE + (int64_t)tid * EPT;
         const int64_t blk_in_tensor = e0 / B;
         const int64_t blk_elem0 = blk_in_tensor * B;
         if (!CTA_GROUP && blk_elem0 >= n) continue;            // the whole group has no block
@@ -340,9 +356,7 @@ __global__ void __launch_bounds__(CTA) solo_step_kernel(const StepArgs a) {
         const int nv = (int)max((int64_t)0, min((int64_t)EPT, n - e0));
         const int64_t jb = __ldg(a.block_start + tensor) + blk_in_tensor;
 
-        char* pbase = (char*)(a.param_list ? a.param_list[tensor] : a.param_single);
-        const char* gbase = (const char*)(a.grad_list ? a.grad_list[tensor] : a.grad_single);
-        const bool vec = nv == EPT && ((((uintptr_t)pbase) | ((uintptr_t)gbase)) & 15u) == 0;
+        const bool vec = nv == EPT && aligned;
 
         // ---- load ----
         float p[EPT], g[EPT];

@@ -1,6 +1,9 @@
 // Sixteen elements per thread: the streamlined step for the plain step (2/3/4-bit states, blocks of
 // 64, 128 or 256, fp32 or bf16 parameters; no L2 term in the gradient, no AdaBelief, base from the
-// p = 0.1 quantile, xi drawn).
+// p = 0.1 quantile, xi drawn).  A second instantiation (PLAIN = false) reads the other modes from the
+// arguments: L2 term, AdaBelief, a fixed base, no dither, stochastic rounding of the first moment
+// (Eq. 5), and the baseline second-moment codebooks (a fixed level table instead of the logarithmic
+// levels: no quantile, no draws, nearest level).
 //
 // Same arithmetic, element for element, as solo_step_fast_kernel (solo_fast.cuh); what changes
 // is the work split.  A CTA of 128 threads owns a tile of 2048 consecutive elements, a thread
@@ -25,7 +28,8 @@
 // its parameter is stored) follows the swap; nothing else depends on the order.
 //
 // This kernel processes full tiles of 16-byte aligned tensors only; every other tile is left to
-// a second launch of solo_step_fast_kernel with StepArgs::only_partial set.
+// a second launch with StepArgs::only_partial set: of solo_step_fast_kernel, or of the general kernel
+// where that one has no path (the baseline codebooks).
 #pragma once
 
 #include "solo_dispatch.h"
@@ -252,14 +256,15 @@ struct Ahead16 {
 // skip the tile and leaves what Eq. 6 needs in xout.
 template <int KV, class Shared>
 __device__ __forceinline__ void block_scalars16(const StepArgs& a, Shared& s, const int64_t jb_tile, const int tid,
-                                                const bool fixed_base) {
+                                                const bool fixed_base, const bool vtab) {
     const uint4 in = s.xin[tid];
     const float dm_new = __uint_as_float(in.x), dv_new = __uint_as_float(in.y);
     const bool zero_m = dm_new < TINY, zero_v = dv_new < TINY;
     const float inv_dv = __frcp_rn(dv_new);
     const float rho = fminf(fmaxf(__uint_as_float(in.z) * inv_dv, RHO_MIN), RHO_MAX);
     const float lam = log2_sp(rho) * (1.0f / (float)(KV - 1));
-    const float al_new = fixed_base ? a.fixed_alpha : exp2_sp(lam);
+    // (a baseline codebook has no base: the array keeps its initial 1/2)
+    const float al_new = vtab ? 0.5f : fixed_base ? a.fixed_alpha : exp2_sp(lam);
     const float inv_lambda = __frcp_rn(log2_sp(al_new));
     const float guard = __fmaf_rn(fabsf(inv_lambda), LG2_ABS, LG2_REL * (float)(KV + 1));
     s.xout[tid] = make_float4(zero_v ? 1.0f : 0.0f, inv_dv, inv_lambda, 0.5f - guard);
@@ -281,7 +286,8 @@ __device__ __forceinline__ void block_scalars16(const StepArgs& a, Shared& s, co
 // exchange with the first warp, the second moment's codes, the stores.
 template <int BM, int BV, bool PBF, int G, bool DECAY, bool PLAIN>
 __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, BV, PBF, G>& s, const float* s_y, const float* s_mid,
-                                            const float4* s_mid4,
+                                            const float4* s_mid4, const float* s_yv, const float4* s_nv,
+                                            const float2* s_yg, const float4* s_br,
                                             char* pbase, const char* gbase, const int tin, const int64_t jb_tile,
                                             const int tensor, Ahead16& ah, const bool next_full, const int64_t tile_no) {
     using Shared = Fast16Shared<BM, BV, PBF, G>;
@@ -293,8 +299,11 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     // PLAIN: the step of the paper as it stands (no L2 term in the gradient, no AdaBelief, base from the
     // p-quantile, xi drawn); the other instantiation reads these modes from the arguments
     const bool l2 = !PLAIN && a.l2, belief = !PLAIN && a.belief;
-    const bool fixed_base = !PLAIN && a.fixed_alpha > 0.0f;
-    const bool round_v = PLAIN || a.round_v;
+    // baseline codebook for the second moment: levels s_yv, nearest level by the midpoints in s_nv
+    const bool vtab = !PLAIN && a.tables_v != nullptr;
+    const bool fixed_base = !PLAIN && (a.fixed_alpha > 0.0f || vtab);   // no quantile to find
+    const bool round_v = PLAIN || (a.round_v && !vtab);
+    const bool round_m = !PLAIN && a.round_m;                     // Eq. 5 instead of Eq. 1 for the first moment
 
     const int64_t tile_elem0 = (int64_t)tin * TILE;
     constexpr int PSZ = PBF ? 2 : 4;                              // bytes per parameter
@@ -324,7 +333,7 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
         if (next_full && tid == 32)
             issue_tile_copy16<BM, BV, PBF, G>(a, s, pt + TILE * PSZ, gt + TILE * 2, jb_tile + NG,
                                            tile_no + 2 == a.debug_stall_tile_p1 ? 16u : 0u);
-        if (tid < NG) block_scalars16<KV>(a, s, jb_tile, tid, fixed_base);
+        if (tid < NG) block_scalars16<KV>(a, s, jb_tile, tid, fixed_base, vtab);
         bar_sync16(2);
         return;
     }
@@ -351,7 +360,7 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
             for (int i = 1; i < BV; ++i) a2[i] = a2[i - 1] * a2[i - 1];
 #pragma unroll
             for (int r0 = 0; r0 < KV; r0 += G)
-                if (r0 + gl < KV) tab_vf[r0 + gl] = pow_sm<BV>(a2, (uint32_t)(r0 + gl)) * dv;
+                if (r0 + gl < KV) tab_vf[r0 + gl] = (vtab ? s_yv[r0 + gl] : pow_sm<BV>(a2, (uint32_t)(r0 + gl))) * dv;
 #pragma unroll
             for (int r0 = 0; r0 < KM; r0 += G)
                 if (r0 + gl < KM) tab_mf[r0 + gl] = s_y[r0 + gl] * dm;
@@ -556,9 +565,89 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
         if (dm_new < TINY) { om[0] = 0; om[1] = 0; }             // vanishing block: all codes 0
     };
     if constexpr (!SOLO_F16_MIX) {
+        if (!round_m) {
 #pragma unroll
-        for (int i = EPT16 - 1; i >= 0; --i) quant_m(i);
-        quant_m_done();
+            for (int i = EPT16 - 1; i >= 0; --i) quant_m(i);
+            quant_m_done();
+        }
+    }
+    if (round_m) {
+        // Eq. 5: q = number of levels y_1 .. y_{K-2} that r reaches (the lower end of its bracket), plus
+        // one when the element's draw u (Philox purpose 1) falls below (r - y_q) / (y_{q+1} - y_q).
+        // "r >= y" is counted on the FMA pipe as the saturation of t - y'*2^100 with t = r*2^100 and y'
+        // the binary32 just below y (exactly 0 or 1: two distinct binary32 near a level differ by far
+        // more than 2^-100); the level 0 as the saturation of t*2^100 + 1 (t = +-0: 1; else |t*2^100| >=
+        // 2^51, or infinite).  NaN counts nowhere and is never below anything: code 0.
+        uint32_t wm[8];
+        {
+            uint32_t ctr_lo, ctr_hi, c3;
+            stream_position(ctr_lo, ctr_hi, c3);
+            uint32_t w4[4];
+            philox_rk(ctr_lo + sw, ctr_hi, a.step32, c3 + 1u, a.rk, w4);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) wm[i] = w4[i];
+            philox_rk(ctr_lo + (sw ^ 1u), ctr_hi, a.step32, c3 + 1u, a.rk, w4);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) wm[4 + i] = w4[i];
+        }
+        constexpr int Z = KM / 2 - 1;                             // index of the level 0
+        float nb[BM == 4 ? 3 : KM - 2];                           // nb[j - 1]: threshold of level j, BM == 4: of levels 4, 8, 12
+        if constexpr (BM == 4) {
+            const float4 c4 = s_br[4];
+            nb[0] = c4.x; nb[1] = c4.y; nb[2] = c4.z;
+        } else {
+            const float4 ba = s_br[0];
+            nb[0] = ba.x; nb[1] = ba.y;
+            if constexpr (BM == 3) {
+                const float4 bb = s_br[1];
+                nb[2] = ba.z; nb[3] = ba.w; nb[4] = bb.x; nb[5] = bb.y;
+            }
+        }
+        float accm[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+        for (int j = EPT16 / 2 - 1; j >= 0; --j) {
+            float d[2];                                           // the 16-bit draws of elements 2j, 2j + 1 as binary32
+            halves_to_float(wm[j], d[0], d[1]);
+#pragma unroll
+            for (int e = 1; e >= 0; --e) {
+                const int i = 2 * j + e;
+                const float r = mh[i] * inv_m;
+                const float t = r * BIG;
+                float qf;
+                if constexpr (BM == 4) {
+                    const float c0 = __saturatef(t + nb[0]);
+                    const float c1 = __saturatef(t + nb[1]);
+                    const float c2 = __saturatef(t + nb[2]);
+                    const float o = __fmaf_rn(c2, 16.0f, __fmaf_rn(c1, 16.0f, __fmaf_rn(c0, 16.0f, 8388608.0f)));
+                    // row s: thresholds of levels 4s+1, 4s+2, 4s+3 (.w: the factor of t for the third,
+                    // 2^100 where that level is 0)
+                    const float4 row = *reinterpret_cast<const float4*>(reinterpret_cast<const char*>(s_br) + (__float_as_uint(o) & 0x30u));
+                    qf = __fmaf_rn((c0 + c1) + c2, 4.0f, __saturatef(t + row.x));
+                    qf += __saturatef(t + row.y);
+                    qf += __saturatef(__fmaf_rn(t, row.w, row.z));
+                } else {
+                    qf = 0.0f;
+#pragma unroll
+                    for (int l = 1; l <= KM - 2; ++l)
+                        qf += l == Z ? __saturatef(__fmaf_rn(t, BIG, 1.0f)) : __saturatef(t + nb[l - 1]);
+                }
+                // the bracket's lower level and the reciprocal of its width, from the pair table
+                const float o8 = __fmaf_rn(qf, 8.0f, 8388608.0f);
+                const float2 yg = *reinterpret_cast<const float2*>(reinterpret_cast<const char*>(s_yg) + (__float_as_uint(o8) & 0xF8u));
+                const float frac = (r - yg.x) * yg.y;
+                const float code = qf + (d[e] < frac * 65536.0f ? 1.0f : 0.0f);     // u = d / 2^16 < frac
+                if constexpr (BM == 4) accm[i >> 2] = __fmaf_rn(accm[i >> 2], 16.0f, code);
+                else accm[i >> 3] = __fmaf_rn(accm[i >> 3], (float)KM, code);
+            }
+        }
+        if constexpr (BM == 4) {
+            om[0] = (uint32_t)accm[0] | ((uint32_t)accm[1] << 16);
+            om[1] = (uint32_t)accm[2] | ((uint32_t)accm[3] << 16);
+        } else {
+            om[0] = (uint32_t)accm[0];
+            om[1] = (uint32_t)accm[1];
+        }
+        if (dm_new < TINY) { om[0] = 0; om[1] = 0; }             // vanishing block: all codes 0
     }
 
     // ---- (D) second moment: block scale and the p-quantile (k = 13 of 128); the draws of Eq. 6 ----
@@ -589,9 +678,11 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
         if (fixed_base) {
             // every block keeps the given base: no quantile to find
             if constexpr (SOLO_F16_MIX) {
+                if (!round_m) {
 #pragma unroll
-                for (int i = EPT16 - 1; i >= 0; --i) quant_m(i);
-                quant_m_done();
+                    for (int i = EPT16 - 1; i >= 0; --i) quant_m(i);
+                    quant_m_done();
+                }
             }
             if (round_v) {
 #pragma unroll
@@ -602,7 +693,7 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
             uint32_t key[EPT16];
 #pragma unroll
             for (int i = 0; i < EPT16; ++i) key[i] = __float_as_uint(vh[i]);
-            if constexpr (SOLO_F16_MIX) {
+            if (SOLO_F16_MIX && !round_m) {
 #pragma unroll
                 for (int k = 0; k < 62; ++k) {
                     cswap(key[SORT16_PAIRS[k][0]], key[SORT16_PAIRS[k][1]]);
@@ -644,13 +735,59 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     if (next_full && tid == 32)
         issue_tile_copy16<BM, BV, PBF, G>(a, s, pt + TILE * PSZ, gt + TILE * 2, jb_tile + NG,
                                        tile_no + 2 == a.debug_stall_tile_p1 ? 16u : 0u);
-    if (tid < NG) block_scalars16<KV>(a, s, jb_tile, tid, fixed_base);
+    if (tid < NG) block_scalars16<KV>(a, s, jb_tile, tid, fixed_base, vtab);
     bar_sync16(2);
     const float4 sc = s.xout[grp];
 
     // second moment: Eq. 6, see fast_tile
     uint32_t ov[2];
-    {
+    if (vtab) {
+        // Eq. 1 on the fixed codebook: code = number of midpoints below r, counted like the first
+        // moment's (saturated multiply-adds, exactly 0 or 1 each: r and a midpoint, if they differ at all,
+        // differ by far more than 2^-100, the smallest midpoint of these codebooks being about 1e-4)
+        const float inv = sc.y;
+        if constexpr (BV <= 3) {
+            const float4 na = s_nv[0], nb = s_nv[1];
+            float acc[2] = {0.0f, 0.0f};                         // eight codes, at most 24 bits: exact
+#pragma unroll
+            for (int i = EPT16 - 1; i >= 0; --i) {
+                const float r = vh[i] * inv;
+                float& c = acc[i >> 3];
+                c = __fmaf_rn(c, (float)KV, __saturatef(__fmaf_rn(r, BIG, na.x)));
+                c += __saturatef(__fmaf_rn(r, BIG, na.y));
+                c += __saturatef(__fmaf_rn(r, BIG, na.z));
+                if constexpr (BV == 3) {
+                    c += __saturatef(__fmaf_rn(r, BIG, na.w));
+                    c += __saturatef(__fmaf_rn(r, BIG, nb.x));
+                    c += __saturatef(__fmaf_rn(r, BIG, nb.y));
+                    c += __saturatef(__fmaf_rn(r, BIG, nb.z));
+                }
+            }
+            ov[0] = (uint32_t)acc[0];
+            ov[1] = (uint32_t)acc[1];
+        } else {
+            // sixteen levels in two steps of three comparisons, as for 4-bit first moments: row 3 holds
+            // the midpoints 3, 7, 11, rows 4..7 the three midpoints inside each quarter
+            const float4 nq4 = s_nv[3];
+            float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};            // four codes each
+#pragma unroll
+            for (int i = EPT16 - 1; i >= 0; --i) {
+                const float r = vh[i] * inv;
+                const float c0 = __saturatef(__fmaf_rn(r, BIG, nq4.x));
+                const float c1 = __saturatef(__fmaf_rn(r, BIG, nq4.y));
+                const float c2 = __saturatef(__fmaf_rn(r, BIG, nq4.z));
+                const float t = __fmaf_rn(c2, 16.0f, __fmaf_rn(c1, 16.0f, __fmaf_rn(c0, 16.0f, 8388608.0f)));
+                const float4 row = *reinterpret_cast<const float4*>(reinterpret_cast<const char*>(s_nv + 4) + (__float_as_uint(t) & 0x30u));
+                float code = __fmaf_rn((c0 + c1) + c2, 4.0f, __saturatef(__fmaf_rn(r, BIG, row.x)));
+                code += __saturatef(__fmaf_rn(r, BIG, row.y));
+                code += __saturatef(__fmaf_rn(r, BIG, row.z));
+                acc[i >> 2] = __fmaf_rn(acc[i >> 2], 16.0f, code);
+            }
+            ov[0] = (uint32_t)acc[0] | ((uint32_t)acc[1] << 16);
+            ov[1] = (uint32_t)acc[2] | ((uint32_t)acc[3] << 16);
+        }
+        if (sc.x != 0.0f) { ov[0] = 0; ov[1] = 0; }              // vanishing block: all codes 0
+    } else {
         const float inv = sc.y, il = sc.z, lim = sc.w;
         constexpr float KM1 = (float)(KV - 1);
         constexpr float MAGIC = 12582912.0f;
@@ -722,6 +859,10 @@ __global__ void __launch_bounds__(CTA16, (PBF || BM != 2 || G == 16 || !PLAIN) ?
     Shared& s = *reinterpret_cast<Shared*>(fast16_smem);
     __shared__ float s_y[KM];
     __shared__ float s_mid[KM];
+    __shared__ float2 s_yg[PLAIN ? 1 : KM];                    // Eq. 5: see the set-up below
+    __shared__ float4 s_br[PLAIN ? 1 : (BM == 4 ? 5 : 2)];
+    __shared__ float s_yv[PLAIN ? 1 : 1 << BV];               // baseline second-moment codebook: its levels,
+    __shared__ float4 s_nv[PLAIN ? 1 : 8];                     // its midpoints times -2^100 (rows as the tile function reads them)
     __shared__ float4 s_mid4[4];             // 4-bit first moments: per quarter of the codebook, its three inner midpoints times -2^100
     const int tid = threadIdx.x;
     if (tid < KM) {
@@ -731,6 +872,53 @@ __global__ void __launch_bounds__(CTA16, (PBF || BM != 2 || G == 16 || !PLAIN) ?
     if (BM == 4 && tid < 4)
         s_mid4[tid] = make_float4(-a.tables[KM + 4 * tid] * 0x1p100f, -a.tables[KM + 4 * tid + 1] * 0x1p100f,
                                   -a.tables[KM + 4 * tid + 2] * 0x1p100f, 0.0f);
+    if constexpr (!PLAIN) {
+        if (a.round_m) {
+            // Eq. 5: per level q <= K-2 the pair (y_q, 1 / (y_{q+1} - y_q)); thresholds of "r >= y_j" as
+            // -y'_j * 2^100, y'_j the binary32 just below y_j (rows as the tile function reads them:
+            // 2- and 3-bit, levels 1..6 in rows 0, 1; 4-bit, row s = levels 4s+1..4s+3 and row 4 = levels
+            // 4, 8, 12).  The level 0 is compared another way; a level past K-2 gets -infinity: never reached.
+            const float* const yk = a.tables;
+            auto below = [&](int j) {
+                const float y = yk[j];
+                return -__uint_as_float(__float_as_uint(y) + (y < 0.0f ? 1u : 0xFFFFFFFFu)) * 0x1p100f;
+            };
+            if (tid < KM - 1) s_yg[tid] = make_float2(yk[tid], a.tables[2 * KM - 1 + tid]);
+            if (BM <= 3 && tid < 2) {
+                float t4[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int j = 4 * tid + k + 1;
+                    t4[k] = j <= KM - 2 && j != KM / 2 - 1 ? below(j) : 0.0f;
+                }
+                s_br[tid] = make_float4(t4[0], t4[1], t4[2], t4[3]);
+            }
+            if (BM == 4 && tid < 4) {
+                const int j = 4 * tid + 1;
+                const bool zero3 = j + 2 == KM / 2 - 1;            // the row's third level is the level 0
+                s_br[tid] = make_float4(below(j), below(j + 1),
+                                        zero3 ? 1.0f : j + 2 <= KM - 2 ? below(j + 2) : -__int_as_float(0x7f800000),
+                                        zero3 ? 0x1p100f : 1.0f);
+            }
+            if (BM == 4 && tid == 4) s_br[4] = make_float4(below(4), below(8), below(12), 0.0f);
+        }
+        if (a.tables_v != nullptr) {
+            constexpr int KV = 1 << BV;
+            const float* const midv = a.tables_v + KV;            // KV - 1 midpoints
+            if (tid < KV) s_yv[tid] = a.tables_v[tid];
+            if (tid < 2) {                                         // rows 0, 1: midpoints 0..7 (rows of 3 or 7 are padded)
+                float m4[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) m4[k] = 4 * tid + k < KV - 1 ? -midv[4 * tid + k] * 0x1p100f : 0.0f;
+                s_nv[tid] = make_float4(m4[0], m4[1], m4[2], m4[3]);
+            }
+            if (BV == 4 && tid == 3)
+                s_nv[3] = make_float4(-midv[3] * 0x1p100f, -midv[7] * 0x1p100f, -midv[11] * 0x1p100f, 0.0f);
+            if (BV == 4 && tid >= 4 && tid < 8)
+                s_nv[tid] = make_float4(-midv[4 * (tid - 4)] * 0x1p100f, -midv[4 * (tid - 4) + 1] * 0x1p100f,
+                                        -midv[4 * (tid - 4) + 2] * 0x1p100f, 0.0f);
+        }
+    }
     if constexpr (Shared::ROWS == 16) s.sort[15][tid] = KEY_MAX;   // never overwritten: rows 0..14 hold keys
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s.mbar)) : "memory");
@@ -771,9 +959,9 @@ __global__ void __launch_bounds__(CTA16, (PBF || BM != 2 || G == 16 || !PLAIN) ?
         if (skip || tin >= full_tiles) continue;
         const bool next_full = tin + 1 < full_tiles && tile + 1 < tile_end;
         if (decay)
-            fast16_tile<BM, BV, PBF, G, true, PLAIN>(a, s, s_y, s_mid, s_mid4, pbase, gbase, tin, jb0 + (int64_t)tin * Shared::NG, tensor, ah, next_full, tile);
+            fast16_tile<BM, BV, PBF, G, true, PLAIN>(a, s, s_y, s_mid, s_mid4, s_yv, s_nv, s_yg, s_br, pbase, gbase, tin, jb0 + (int64_t)tin * Shared::NG, tensor, ah, next_full, tile);
         else
-            fast16_tile<BM, BV, PBF, G, false, PLAIN>(a, s, s_y, s_mid, s_mid4, pbase, gbase, tin, jb0 + (int64_t)tin * Shared::NG, tensor, ah, next_full, tile);
+            fast16_tile<BM, BV, PBF, G, false, PLAIN>(a, s, s_y, s_mid, s_mid4, s_yv, s_nv, s_yg, s_br, pbase, gbase, tin, jb0 + (int64_t)tin * Shared::NG, tensor, ah, next_full, tile);
     }
     // A thread that gave up on a copy waits once more, again bounded, for the last one that was issued,
     // so that no copy is still writing to the stage when the CTA's shared memory is released.

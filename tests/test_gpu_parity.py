@@ -96,7 +96,8 @@ def test_bits_and_blocks_random_state(bits_m, bits_v, block):
 @pytest.mark.parametrize("bits_m,bits_v,block", [(2, 3, 128), (3, 2, 64), (4, 4, 256), (2, 2, 2048), (8, 4, 64),
                                                  (2, 8, 256)])
 @pytest.mark.parametrize("hk", [dict(adamw=0, weight_decay=0.1), dict(round_v=0, belief=1),
-                                dict(fixed_alpha=0.5, param_dtype=1)])
+                                dict(fixed_alpha=0.5, param_dtype=1), dict(round_m=1, seed=0xABCDEF012345),
+                                dict(round_m=1, v_codebook=2, adamw=0)])
 def test_mode_flags_at_other_widths(bits_m, bits_v, block, hk):
     """The streamlined kernel has one instantiation for the paper's plain step and one that reads
     the mode flags at run time; the latter at other widths and block sizes than the mode test."""
@@ -151,17 +152,21 @@ def test_hyper_parameter_modes(hk):
 
 
 @pytest.mark.parametrize("sel", [1, 2, 3])
-@pytest.mark.parametrize("bits_v,block", [(2, 64), (3, 128), (4, 2048), (8, 256)])
-def test_baseline_second_moment_codebooks(sel, bits_v, block):
+@pytest.mark.parametrize("bits_m,bits_v,block", [(4, 2, 64), (4, 3, 128), (4, 4, 2048), (4, 8, 256), (2, 4, 256),
+                                                 (3, 4, 128), (2, 2, 128), (3, 3, 64)])
+def test_baseline_second_moment_codebooks(sel, bits_m, bits_v, block):
     """Sec. 4 baselines for the unsigned state (unsigned DE, linear, linear without zero;
-    Appendix A) at every width, from a random packed state and from zero, ragged sizes."""
-    sizes = (block * 5 + 3, 1, 2048 * 2 + 9, block - 1)
+    Appendix A) at every width, from a random packed state and from zero, ragged sizes.
+    Policy 3: full tiles in the sixteen-per-thread kernel (widths up to 4 bits, blocks up to 256),
+    the rest in the general kernel; policy 1: the general kernel alone."""
+    sizes = (block * 5 + 3, 1, 2048 * 2 + 9, block - 1, 2048 * 3)
     w = synth.workload(4, sizes=sizes)                            # zero blocks and zero elements
     params, gf = _inputs(w)
     hk = dict(lr=1e-3, beta1=0.8, beta2=0.999, weight_decay=0.01, seed=5, v_codebook=sel)
-    st0 = synth.make_state(sizes, 4, bits_v, block, seed=sel * 1000 + bits_v * 10 + block)
-    run_lockstep(sizes, 4, bits_v, block, hk, 2, gf, params, state0=st0)
-    run_lockstep(sizes, 4, bits_v, block, hk, 3, gf, params)
+    st0 = synth.make_state(sizes, bits_m, bits_v, block, seed=sel * 1000 + bits_v * 10 + block)
+    run_lockstep(sizes, bits_m, bits_v, block, hk, 2, gf, params, state0=st0, policies=(0, 3, 1),
+                 update_tol=RANDOM_STATE_TOL)
+    run_lockstep(sizes, bits_m, bits_v, block, hk, 3, gf, params, policies=(0, 3, 1))
 
 
 @pytest.mark.parametrize("param_round", [0, 1])
