@@ -151,7 +151,7 @@ int solo_step(void* param_dev, const void* grad_dev, solo_state_t* state,
 /*
  * The same step over every tensor of the list, ragged block tails included, in one kernel
  * launch -- or in two when the kernel with sixteen elements per thread is selected (see
- * solo_set_kernel_policy: large sets at block 128; it takes the full 2048-element tiles and a
+ * solo_set_kernel_policy: large sets at blocks of 64, 128 or 256; it takes the full 2048-element tiles and a
  * second, short launch the tiles that are not full; policy 2 keeps every set to one launch).
  * Tensor t uses Philox stream t.  Asynchronous on `stream`.
  */
@@ -289,10 +289,12 @@ float solo_default_beta1(int bits_m, int from_scratch);
  * Kernel selection.  0 (default): every width and block size with the logarithmic
  * second-moment quantizer, nearest rounding of the first moment and eps >= 1e-12 runs the
  * streamlined kernel (fp32 or bf16 parameters), everything else the general one; tensor sets of
- * at least 8192 tiles of 2048 elements with 2/3/4-bit states, blocks of 64, 128 or 256 and the
- * plain Adam(W) step with p = 0.1 run their
- * full tiles in a kernel with sixteen elements per thread and the remaining tiles in the
- * streamlined kernel (two launches).  1: always the general kernel.  2: like 0 without the
+ * at least 8192 tiles of 2048 elements with 2/3/4-bit states and blocks of 64, 128 or 256 run
+ * their full tiles in a kernel with sixteen elements per thread and the remaining tiles in the
+ * streamlined kernel, or in the general one where the streamlined kernel does not apply (two
+ * launches).  That kernel covers every mode of solo_hyper_t (Eq. 5 rounding and the baseline
+ * second-moment codebooks included) as long as the quantile is the p = 0.1 one or none is taken
+ * (fixed base, baseline codebook).  1: always the general kernel.  2: like 0 without the
  * sixteen-per-thread kernel.  3: like 0 with the sixteen-per-thread kernel whatever the tensor
  * sizes.  All produce the same packed state and the same bf16 parameters; the fp32 parameters
  * of the two faster kernels are identical to each other and differ from the IEEE sequence of

@@ -38,9 +38,11 @@ StepKernel fast_kernel_bm3(int bv_index, int block, bool param_bf16, bool plain)
 StepKernel fast_kernel_bm4(int bv_index, int block, bool param_bf16, bool plain);
 StepKernel fast_kernel_bm8(int bv_index, int block, bool param_bf16, bool plain);
 StepKernel fast_kernel(int bits_m, int bits_v, int block, bool param_bf16, bool plain);
-// Sixteen elements per thread: 2/3/4-bit states, blocks of 64, 128 or 256, fp32 or
-// bf16 parameters, the quantile rank of p = 0.1 or a fixed base; `plain` as for fast_kernel; full tiles of aligned tensors only (the rest is left to a
-// launch of the streamlined kernel with StepArgs::only_partial).  Launched with CTA16 = 128 threads.
+// Sixteen elements per thread: 2/3/4-bit states, blocks of 64, 128 or 256, fp32 or bf16 parameters, the
+// quantile rank of p = 0.1 or no quantile (fixed base, baseline codebook); `plain` as for fast_kernel
+// (the other instantiation also has Eq. 5 rounding and the baseline second-moment codebooks); full tiles
+// of aligned tensors only (the rest is left to a launch of the streamlined or of the general kernel with
+// StepArgs::only_partial).  Launched with CTA16 = 128 threads.
 // Null / 0 for other widths and block sizes.  One translation unit per block size.
 constexpr int CTA16 = 128;         // threads per CTA of that kernel
 StepKernel fast16_kernel_g4(int bits_m, int bits_v, bool param_bf16, bool plain);

@@ -198,13 +198,28 @@ __device__ __forceinline__ uint32_t group_max16(uint32_t x) {
     return x;
 }
 
+// Minimum of the group's keys as each lane holds them.  Groups of sixteen: the two groups of a warp are
+// served by one full-mask minimum and one maximum, the upper group (`hi`) holding its keys complemented
+// (its minimum is the complement of the warp's maximum; keys are 31-bit, so the lower group's keys stay
+// below and the upper group's above 2^31); a lane holds the minimum iff its own value equals the result.
+template <int G>
+__device__ __forceinline__ uint32_t group_min16k(uint32_t x, bool hi) {
+    if constexpr (G == 16) {
+        const uint32_t lo = __reduce_min_sync(0xffffffffu, x);
+        const uint32_t up = __reduce_max_sync(0xffffffffu, x);
+        return hi ? up : lo;
+    } else {
+        return group_min16<G>(x);
+    }
+}
+
 // One selection round over groups of G lanes, as pop_round in solo_fast.cuh (columns of CTA16 words;
-// keys as they are, no transformed domain).  CLAMP: the offset stops at the sentinel row (needed when a
-// thread can be asked for more keys than it has).
+// keys as they are, or complemented in the upper group of sixteen).  CLAMP: the offset stops at the
+// sentinel row (needed when a thread can be asked for more keys than it has).
 template <int G, bool LAST, bool CLAMP>
 __device__ __forceinline__ uint32_t pop_round16(uint32_t& head, int& off, const uint32_t* col, uint32_t le,
-                                                uint32_t self) {
-    const uint32_t tgt = group_min16<G>(head);
+                                                uint32_t self, bool hi) {
+    const uint32_t tgt = group_min16k<G>(head, hi);
     if constexpr (LAST) return tgt;
     const uint32_t nxt = col[off];
     const uint32_t upto = __ballot_sync(0xffffffffu, head == tgt) & le;
@@ -706,23 +721,26 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
             if constexpr (ROUNDS > 12) cswap(key[13], key[14]); // all sixteen in order
             uint32_t* const col = &s.sort[0][tid];
             constexpr int KEPT = ROUNDS < 15 ? ROUNDS : 15;       // keys after the smallest that can be asked for
+            // (upper group of sixteen lanes: complemented, see group_min16k)
+            const bool hi = G == 16 && (lane & 16);
+            const uint32_t vx = hi ? 0xFFFFFFFFu : 0u;
 #pragma unroll
-            for (int j = 1; j <= KEPT; ++j) col[(j - 1) * CTA16] = key[j];
+            for (int j = 1; j <= KEPT; ++j) col[(j - 1) * CTA16] = key[j] ^ vx;
             // ROUNDS rounds pop the ROUNDS smallest keys of the block, the next minimum is x_p
             const uint32_t self = 1u << lane;
             const uint32_t le = (self | (self - 1u)) & ((G == 32 ? 0xFFFFFFFFu : ((1u << G) - 1u)) << (lane & ~(G - 1)));
-            uint32_t head = key[0];
+            uint32_t head = key[0] ^ vx;
             int off = 0;
 #pragma unroll
             for (int r = 0; r < ROUNDS; ++r) {
-                pop_round16<G, false, (ROUNDS > 15)>(head, off, col, le, self);
+                pop_round16<G, false, (ROUNDS > 15)>(head, off, col, le, self, hi);
                 if (r < 10 && round_v) philox_round(r);
             }
             if (round_v) {
 #pragma unroll
                 for (int r = ROUNDS; r < 10; ++r) philox_round(r);
             }
-            x_p = pop_round16<G, true, false>(head, off, col, le, self);
+            x_p = pop_round16<G, true, false>(head, off, col, le, self, hi) ^ vx;
         }
 #pragma unroll
         for (int i = 0; i < 4; ++i) { w[i] = ca[i]; w[4 + i] = cb[i]; }
@@ -919,7 +937,8 @@ __global__ void __launch_bounds__(CTA16, (PBF || BM != 2 || G == 16 || !PLAIN) ?
                                         -midv[4 * (tid - 4) + 2] * 0x1p100f, 0.0f);
         }
     }
-    if constexpr (Shared::ROWS == 16) s.sort[15][tid] = KEY_MAX;   // never overwritten: rows 0..14 hold keys
+    // (never overwritten: rows 0..14 hold keys; complemented for the upper group of sixteen lanes)
+    if constexpr (Shared::ROWS == 16) s.sort[15][tid] = (G == 16 && (tid & 16)) ? ~KEY_MAX : KEY_MAX;
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s.mbar)) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");

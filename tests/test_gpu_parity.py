@@ -306,7 +306,8 @@ def test_ragged_zero_blocks_and_zero_elements():
         assert rep.exempt_m + rep.exempt_v <= 3
 
 
-@pytest.mark.parametrize("bits_m,bits_v,block", [(2, 3, 128), (4, 4, 128), (3, 2, 64), (2, 2, 2048), (8, 4, 256)])
+@pytest.mark.parametrize("bits_m,bits_v,block", [(2, 3, 128), (4, 4, 128), (3, 2, 64), (2, 2, 2048), (8, 4, 256),
+                                                 (4, 3, 256)])
 def test_nan_and_inf_gradients_follow_one_rule(bits_m, bits_v, block):
     """The paper says nothing about non-finite gradients; the rule here is that they propagate: a
     NaN in a block makes that block's scale NaN and its codes 0, an infinity makes the scale
