@@ -32,9 +32,8 @@ UNITS = [
     ("solo_fast_inst.cu", "solo_fast_bm3.o", ["-DSOLO_BM=3"]),
     ("solo_fast_inst.cu", "solo_fast_bm4.o", ["-DSOLO_BM=4"]),
     ("solo_fast_inst.cu", "solo_fast_bm8.o", ["-DSOLO_BM=8"]),
-    ("solo_fast16_inst.cu", "solo_fast16_g4.o", ["-DSOLO_G=4"]),
-    ("solo_fast16_inst.cu", "solo_fast16_g8.o", ["-DSOLO_G=8"]),
-    ("solo_fast16_inst.cu", "solo_fast16_g16.o", ["-DSOLO_G=16"]),
+    *[("solo_fast16_inst.cu", f"solo_fast16_g{g}_m{m}.o", [f"-DSOLO_G={g}", f"-DSOLO_MODES={m}"])
+      for g in (4, 8, 16) for m in (0, 1, 2)],
 ]
 
 

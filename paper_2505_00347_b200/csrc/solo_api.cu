@@ -237,7 +237,8 @@ int launch_step(solo_state* s, StepArgs& a, cudaStream_t stream) {
                         (s->block == 256 && a.k_full == 26);
     // (a fixed base or a baseline codebook needs no quantile, so any p goes with them)
     if (fast_ok && ((policy == 0 && large) || policy == 3) && (rank16 || a.fixed_alpha > 0.0f || a.tables_v))
-        k16 = solo::fast16_kernel(s->bits_m, s->bits_v, s->block, a.param_bf16 != 0, plain);
+        k16 = solo::fast16_kernel(s->bits_m, s->bits_v, s->block, a.param_bf16 != 0,
+                                  plain ? 0 : (a.tables_v || a.round_m) ? 2 : 1);
     if (k16) {
         // full tiles by the sixteen-per-thread kernel, whatever it leaves (tails, tensors that are
         // not 16-byte aligned) by the streamlined kernel, or by the general one where that has no path

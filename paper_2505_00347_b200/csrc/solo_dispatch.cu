@@ -30,13 +30,18 @@ StepKernel fast_kernel(int bits_m, int bits_v, int block, bool param_bf16, bool 
     }
 }
 
-StepKernel fast16_kernel(int bits_m, int bits_v, int block, bool param_bf16, bool plain) {
+StepKernel fast16_kernel(int bits_m, int bits_v, int block, bool param_bf16, int modes) {
+#define SOLO_PICK16(G)                                                                   \
+    (modes == 0 ? fast16_kernel_g##G##_m0(bits_m, bits_v, param_bf16)                    \
+                : modes == 1 ? fast16_kernel_g##G##_m1(bits_m, bits_v, param_bf16)       \
+                             : fast16_kernel_g##G##_m2(bits_m, bits_v, param_bf16))
     switch (block) {
-        case 64: return fast16_kernel_g4(bits_m, bits_v, param_bf16, plain);
-        case 128: return fast16_kernel_g8(bits_m, bits_v, param_bf16, plain);
-        case 256: return fast16_kernel_g16(bits_m, bits_v, param_bf16, plain);   // twenty-five selection rounds: +0 to +11 % over the eight-per-thread kernel
+        case 64: return SOLO_PICK16(4);
+        case 128: return SOLO_PICK16(8);
+        case 256: return SOLO_PICK16(16);   // twenty-five selection rounds
         default: return nullptr;
     }
+#undef SOLO_PICK16
 }
 
 size_t fast16_kernel_smem(int bits_m, int bits_v, int block, bool param_bf16) {

@@ -39,19 +39,26 @@ StepKernel fast_kernel_bm4(int bv_index, int block, bool param_bf16, bool plain)
 StepKernel fast_kernel_bm8(int bv_index, int block, bool param_bf16, bool plain);
 StepKernel fast_kernel(int bits_m, int bits_v, int block, bool param_bf16, bool plain);
 // Sixteen elements per thread: 2/3/4-bit states, blocks of 64, 128 or 256, fp32 or bf16 parameters, the
-// quantile rank of p = 0.1 or no quantile (fixed base, baseline codebook); `plain` as for fast_kernel
-// (the other instantiation also has Eq. 5 rounding and the baseline second-moment codebooks); full tiles
+// quantile rank of p = 0.1 or no quantile (fixed base, baseline codebook); `modes`: 0 as `plain` for
+// fast_kernel, 1 the modes fast_kernel reads at run time, 2 those plus Eq. 5 rounding and the baseline
+// second-moment codebooks; full tiles
 // of aligned tensors only (the rest is left to a launch of the streamlined or of the general kernel with
 // StepArgs::only_partial).  Launched with CTA16 = 128 threads.
-// Null / 0 for other widths and block sizes.  One translation unit per block size.
+// Null / 0 for other widths and block sizes.  One translation unit per block size and set of modes.
 constexpr int CTA16 = 128;         // threads per CTA of that kernel
-StepKernel fast16_kernel_g4(int bits_m, int bits_v, bool param_bf16, bool plain);
-StepKernel fast16_kernel_g8(int bits_m, int bits_v, bool param_bf16, bool plain);
-StepKernel fast16_kernel_g16(int bits_m, int bits_v, bool param_bf16, bool plain);
+StepKernel fast16_kernel_g4_m0(int bits_m, int bits_v, bool param_bf16);
+StepKernel fast16_kernel_g4_m1(int bits_m, int bits_v, bool param_bf16);
+StepKernel fast16_kernel_g4_m2(int bits_m, int bits_v, bool param_bf16);
+StepKernel fast16_kernel_g8_m0(int bits_m, int bits_v, bool param_bf16);
+StepKernel fast16_kernel_g8_m1(int bits_m, int bits_v, bool param_bf16);
+StepKernel fast16_kernel_g8_m2(int bits_m, int bits_v, bool param_bf16);
+StepKernel fast16_kernel_g16_m0(int bits_m, int bits_v, bool param_bf16);
+StepKernel fast16_kernel_g16_m1(int bits_m, int bits_v, bool param_bf16);
+StepKernel fast16_kernel_g16_m2(int bits_m, int bits_v, bool param_bf16);
 size_t fast16_smem_g4(int bits_m, int bits_v, bool param_bf16);
 size_t fast16_smem_g8(int bits_m, int bits_v, bool param_bf16);
 size_t fast16_smem_g16(int bits_m, int bits_v, bool param_bf16);
-StepKernel fast16_kernel(int bits_m, int bits_v, int block, bool param_bf16, bool plain);
+StepKernel fast16_kernel(int bits_m, int bits_v, int block, bool param_bf16, int modes);
 size_t fast16_kernel_smem(int bits_m, int bits_v, int block, bool param_bf16);
 // Dynamic shared memory the streamlined kernel for these widths is launched with.
 size_t fast_kernel_smem(int bits_m, int bits_v);

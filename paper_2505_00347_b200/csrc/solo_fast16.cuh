@@ -1,9 +1,10 @@
 // Sixteen elements per thread: the streamlined step for the plain step (2/3/4-bit states, blocks of
 // 64, 128 or 256, fp32 or bf16 parameters; no L2 term in the gradient, no AdaBelief, base from the
-// p = 0.1 quantile, xi drawn).  A second instantiation (PLAIN = false) reads the other modes from the
-// arguments: L2 term, AdaBelief, a fixed base, no dither, stochastic rounding of the first moment
-// (Eq. 5), and the baseline second-moment codebooks (a fixed level table instead of the logarithmic
-// levels: no quantile, no draws, nearest level).
+// p = 0.1 quantile, xi drawn: MODES = 0).  Two more instantiations read other modes from the arguments:
+// MODES = 1 the L2 term, AdaBelief, a fixed base, no dither; MODES = 2 also stochastic rounding of the
+// first moment (Eq. 5) and the baseline second-moment codebooks (a fixed level table instead of the
+// logarithmic levels: no quantile, no draws, nearest level).  (One instantiation for all of them
+// measured 11 % slower on the modes of MODES = 1 than the one that leaves Eq. 5 and the tables out.)
 //
 // Same arithmetic, element for element, as solo_step_fast_kernel (solo_fast.cuh); what changes
 // is the work split.  A CTA of 128 threads owns a tile of 2048 consecutive elements, a thread
@@ -50,23 +51,32 @@ static_assert(CTA16 * EPT16 == TILE, "same tile as the other kernels");
 #define SOLO_F16_M4FMA 1                // 4-bit first moments: two levels of three saturated multiply-adds
 #endif
 #ifndef SOLO_F16_CTAS
-#define SOLO_F16_CTAS 7                 // resident CTAs per SM the fp32 kernel is compiled for
+#define SOLO_F16_CTAS 7                 // resident CTAs per SM the plain fp32 kernel for blocks of 64 and 128 is compiled for (72 registers)
+#endif
+#ifndef SOLO_F16_CTAS_WIDE
+#define SOLO_F16_CTAS_WIDE 6            // the same for every other instantiation
 #endif
 
-// G: lanes per block (4, 8 or 16 for blocks of 64, 128 or 256 elements); NG = 128 / G blocks per tile.
+// G: lanes per block (4, 8 or 16 for blocks of 64, 128 or 256 elements; 128: the CTA is one block of
+// 2048); NG = 128 / G blocks per tile.
 template <int BM, int BV, bool PBF, int G>
 struct Fast16Shared {
     static constexpr int NG = CTA16 / G;
     static constexpr int ROUNDS = G == 4 ? 6 : G == 8 ? 12 : 25;   // rank of the p = 0.1 quantile minus one: 7, 13, 26
     static constexpr int ROWS = ROUNDS < 15 ? ROUNDS : 16;         // G = 16: all fifteen further keys and a sentinel row
+    static constexpr int NT = G == 128 ? 4 : NG;                   // level tables: one per block, or one per warp of the one block
     // Sorted keys of the threads, one column per thread: row j holds the (j+2)-th smallest key.
     // The rounds of popping read rows 0..ROUNDS-1 at most; with 25 rounds a thread can run out of
-    // keys, and row 15 holds a sentinel above every key.
-    uint32_t sort[ROWS][CTA16];
+    // keys, and row 15 holds a sentinel above every key.  G = 128: the 2048 bins of the radix select.
+    alignas(16) uint32_t sort[ROWS][CTA16];
+    // G = 128: the CTA-wide selection's small state (see cta_select16) and the warps' maxima
+    uint32_t scan[G == 128 ? 16 : 1];
+    uint32_t list[G == 128 ? 32 : 1];
+    uint32_t red[G == 128 ? 8 : 1];
     // per block: K_v second-moment levels alpha^k Delta_v and K_m first-moment levels y_k Delta_m.
     // Two arrays, so that the four blocks of a warp occupy distinct banks (up to eight levels).
-    float tab_v[NG][1 << BV];
-    float tab_m[NG][1 << BM];
+    float tab_v[NT][1 << BV];
+    float tab_m[NT][1 << BM];
     // Exchange with the first warp.  One copy is enough: xin is written before the tile's first
     // barrier and read between its two barriers, xout is written between the barriers and read
     // after the second, and nobody writes either again before passing those barriers.
@@ -245,7 +255,8 @@ __device__ __forceinline__ void issue_tile_copy16(const StepArgs& a, Fast16Share
     // 16 bytes more (the state's arrays carry that slack), and read with an offset
     const int64_t bm0 = jb_tile * (2 * G * BM), bv0 = jb_tile * (2 * G * BV);
     const uint32_t bytes_m = 256 * BM + ((bm0 & 15) ? 16u : 0u), bytes_v = 256 * BV + ((bv0 & 15) ? 16u : 0u);
-    const uint32_t bytes_s = (NG + ((jb_tile & 3) ? 4u : 0u)) * 4u;
+    // (a single block's scalar lies within the 16 bytes that start at the boundary below it)
+    const uint32_t bytes_s = NG >= 4 ? (NG + ((jb_tile & 3) ? 4u : 0u)) * 4u : 16u;
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar),
                  "r"((uint32_t)(TILE * (PBF ? 2 : 4) + TILE * 2) + bytes_m + bytes_v + 3u * bytes_s + extra_tx)
                  : "memory");
@@ -299,7 +310,7 @@ __device__ __forceinline__ void block_scalars16(const StepArgs& a, Shared& s, co
 // known to all eight lanes after the maximum); (D) the sort and the selection rounds, with the Philox
 // rounds of the thread's two blocks of draws issued between them (they depend on nothing); (E) the
 // exchange with the first warp, the second moment's codes, the stores.
-template <int BM, int BV, bool PBF, int G, bool DECAY, bool PLAIN>
+template <int BM, int BV, bool PBF, int G, bool DECAY, int MODES>
 __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, BV, PBF, G>& s, const float* s_y, const float* s_mid,
                                             const float4* s_mid4, const float* s_yv, const float4* s_nv,
                                             const float2* s_yg, const float4* s_br,
@@ -312,13 +323,15 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     const int gl = tid & (G - 1), grp = tid / G;
     const uint32_t sw = ((uint32_t)tid >> 2) & 1u;               // 1: this thread takes elements 8..15 first (see the top of the file)
     // PLAIN: the step of the paper as it stands (no L2 term in the gradient, no AdaBelief, base from the
-    // p-quantile, xi drawn); the other instantiation reads these modes from the arguments
+    // p-quantile, xi drawn); the other instantiations read these modes from the arguments, EXT also
+    // Eq. 5 and the baseline codebooks
+    constexpr bool PLAIN = MODES == 0, EXT = MODES == 2;
     const bool l2 = !PLAIN && a.l2, belief = !PLAIN && a.belief;
     // baseline codebook for the second moment: levels s_yv, nearest level by the midpoints in s_nv
-    const bool vtab = !PLAIN && a.tables_v != nullptr;
+    const bool vtab = EXT && a.tables_v != nullptr;
     const bool fixed_base = !PLAIN && (a.fixed_alpha > 0.0f || vtab);   // no quantile to find
     const bool round_v = PLAIN || (a.round_v && !vtab);
-    const bool round_m = !PLAIN && a.round_m;                     // Eq. 5 instead of Eq. 1 for the first moment
+    const bool round_m = EXT && a.round_m;                     // Eq. 5 instead of Eq. 1 for the first moment
 
     const int64_t tile_elem0 = (int64_t)tin * TILE;
     constexpr int PSZ = PBF ? 2 : 4;                              // bytes per parameter
@@ -869,18 +882,19 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
     store_codes16<BV>(a.codes_v + jb_tile * (2 * G * BV), s.cout[(BM == 3 && BV == 3) ? 1 : 0][BV == 3 ? warp : 0], tid, ov_e);
 }
 
-template <int BM, int BV, bool PBF, int G, bool PLAIN>
-__global__ void __launch_bounds__(CTA16, (PBF || BM != 2 || G == 16 || !PLAIN) ? 6 : SOLO_F16_CTAS) solo_step_fast16_kernel(const StepArgs a) {
+template <int BM, int BV, bool PBF, int G, int MODES>
+__global__ void __launch_bounds__(CTA16, (PBF || G == 16 || MODES != 0) ? SOLO_F16_CTAS_WIDE : SOLO_F16_CTAS) solo_step_fast16_kernel(const StepArgs a) {
     constexpr int KM = 1 << BM;
+    constexpr bool EXT = MODES == 2;
     using Shared = Fast16Shared<BM, BV, PBF, G>;
     extern __shared__ __align__(16) unsigned char fast16_smem[];
     Shared& s = *reinterpret_cast<Shared*>(fast16_smem);
     __shared__ float s_y[KM];
     __shared__ float s_mid[KM];
-    __shared__ float2 s_yg[PLAIN ? 1 : KM];                    // Eq. 5: see the set-up below
-    __shared__ float4 s_br[PLAIN ? 1 : (BM == 4 ? 5 : 2)];
-    __shared__ float s_yv[PLAIN ? 1 : 1 << BV];               // baseline second-moment codebook: its levels,
-    __shared__ float4 s_nv[PLAIN ? 1 : 8];                     // its midpoints times -2^100 (rows as the tile function reads them)
+    __shared__ float2 s_yg[EXT ? KM : 1];                    // Eq. 5: see the set-up below
+    __shared__ float4 s_br[EXT ? (BM == 4 ? 5 : 2) : 1];
+    __shared__ float s_yv[EXT ? 1 << BV : 1];               // baseline second-moment codebook: its levels,
+    __shared__ float4 s_nv[EXT ? 8 : 1];                     // its midpoints times -2^100 (rows as the tile function reads them)
     __shared__ float4 s_mid4[4];             // 4-bit first moments: per quarter of the codebook, its three inner midpoints times -2^100
     const int tid = threadIdx.x;
     if (tid < KM) {
@@ -890,7 +904,7 @@ __global__ void __launch_bounds__(CTA16, (PBF || BM != 2 || G == 16 || !PLAIN) ?
     if (BM == 4 && tid < 4)
         s_mid4[tid] = make_float4(-a.tables[KM + 4 * tid] * 0x1p100f, -a.tables[KM + 4 * tid + 1] * 0x1p100f,
                                   -a.tables[KM + 4 * tid + 2] * 0x1p100f, 0.0f);
-    if constexpr (!PLAIN) {
+    if constexpr (EXT) {
         if (a.round_m) {
             // Eq. 5: per level q <= K-2 the pair (y_q, 1 / (y_{q+1} - y_q)); thresholds of "r >= y_j" as
             // -y'_j * 2^100, y'_j the binary32 just below y_j (rows as the tile function reads them:
@@ -978,9 +992,9 @@ __global__ void __launch_bounds__(CTA16, (PBF || BM != 2 || G == 16 || !PLAIN) ?
         if (skip || tin >= full_tiles) continue;
         const bool next_full = tin + 1 < full_tiles && tile + 1 < tile_end;
         if (decay)
-            fast16_tile<BM, BV, PBF, G, true, PLAIN>(a, s, s_y, s_mid, s_mid4, s_yv, s_nv, s_yg, s_br, pbase, gbase, tin, jb0 + (int64_t)tin * Shared::NG, tensor, ah, next_full, tile);
+            fast16_tile<BM, BV, PBF, G, true, MODES>(a, s, s_y, s_mid, s_mid4, s_yv, s_nv, s_yg, s_br, pbase, gbase, tin, jb0 + (int64_t)tin * Shared::NG, tensor, ah, next_full, tile);
         else
-            fast16_tile<BM, BV, PBF, G, false, PLAIN>(a, s, s_y, s_mid, s_mid4, s_yv, s_nv, s_yg, s_br, pbase, gbase, tin, jb0 + (int64_t)tin * Shared::NG, tensor, ah, next_full, tile);
+            fast16_tile<BM, BV, PBF, G, false, MODES>(a, s, s_y, s_mid, s_mid4, s_yv, s_nv, s_yg, s_br, pbase, gbase, tin, jb0 + (int64_t)tin * Shared::NG, tensor, ah, next_full, tile);
     }
     // A thread that gave up on a copy waits once more, again bounded, for the last one that was issued,
     // so that no copy is still writing to the stage when the CTA's shared memory is released.

@@ -541,13 +541,13 @@ def test_argument_validation():
 
 
 def _full_size_sampled(cfg: int, random_per_tensor: int, need_bytes: float, overrides=None, step: int = 3,
-                       param_bf16: int = 0):
+                       param_bf16: int = 0, hyper_kw=None):
     """A benchmark workload at its full size, one solo_multi_step launch in the configuration
     bench.py times, from a seeded random packed state.  Blocks are independent, so the oracle
     recomputes a sample of them one by one from copies of their inputs taken before the step:
     the first and the last block of every tensor plus `random_per_tensor` random ones.
     param_bf16: 0 fp32 parameters, 1 bf16 rounded to nearest, 2 bf16 rounded stochastically (the
-    stored patterns are then compared bit for bit)."""
+    stored patterns are then compared bit for bit).  hyper_kw: other fields of the step's hyper-parameters."""
     from paper_2505_00347_b200 import binding as B
     free, _ = torch.cuda.mem_get_info()
     if free < need_bytes:
@@ -589,6 +589,7 @@ def _full_size_sampled(cfg: int, random_per_tensor: int, need_bytes: float, over
     kw = dict(lr=w.lr, beta1=w.beta1, beta2=w.beta2, weight_decay=w.weight_decay, seed=1234)
     if param_bf16:
         kw.update(param_dtype=1, param_round=1 if param_bf16 == 2 else 0)
+    kw.update(hyper_kw or {})
     ho, hg = parity.hyper_pair(**kw)
     B.solo_multi_step(B.TensorSet(params, grads, gstate), hg, step)
     torch.cuda.synchronize()
@@ -731,3 +732,17 @@ def test_full_size_gpt125m_set_sampled_blocks():
 def test_full_size_sweep_tensor_sampled_blocks(bits, block):
     """One 268,435,456-element tensor at other widths and block sizes."""
     _full_size_sampled(5, 400, 6e9, overrides=dict(bits_m=bits, bits_v=bits, block=block))
+
+
+@pytest.mark.parametrize("bits,block,hk", [
+    (3, 128, dict(v_codebook=3)),
+    (4, 256, dict(round_m=1)),
+    (2, 64, dict(fixed_alpha=0.5, belief=1)),
+    (4, 128, dict(v_codebook=1, round_m=1, adamw=0, weight_decay=0.01)),
+    (2, 256, dict(round_v=0, v_codebook=2)),
+])
+def test_full_size_sweep_tensor_other_modes(bits, block, hk):
+    """The same tensor in the modes that the sixteen-per-thread kernel reads at run time (baseline
+    second-moment codebooks, Eq. 5 rounding, fixed base, AdaBelief, L2 term), in the launch
+    configuration the default policy picks for a set of this size."""
+    _full_size_sampled(5, 400, 6e9, overrides=dict(bits_m=bits, bits_v=bits, block=block), hyper_kw=hk)
