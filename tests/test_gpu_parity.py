@@ -114,6 +114,25 @@ def test_mode_flags_at_other_widths(bits_m, bits_v, block, hk):
                        policies=(0, 3, 1)))
 
 
+@pytest.mark.parametrize("bits_m,bits_v,block", [(2, 3, 128), (3, 3, 64), (4, 2, 256), (4, 4, 128), (8, 3, 128)])
+@pytest.mark.parametrize("beta1", [0.5, 0.75])
+def test_eq5_rounding_on_the_levels_themselves(bits_m, bits_v, block, beta1):
+    """Eq. 5 where its bracket search is decided by equality: with zero gradients the first moment is
+    beta1 times a level times the scale, so in every block that holds the level 1 the ratio
+    m^ / Delta' lands on a level of the codebook or an ulp beside it (the fractional position is 0, an
+    ulp, or an ulp short of 1), for every level of the random packed state; zero elements give r = +-0.  The
+    sixteen-per-thread kernel counts the levels r reaches with saturated multiply-adds, the general
+    kernel and the oracle compare; all three must agree on every code."""
+    sizes = (2048 * 4 + 3 * block + 5, 2048 * 2)
+    w = synth.workload(1, sizes=sizes)
+    params = [synth.make_param(w, i) for i in range(2)]
+    zero = lambda t: [torch.zeros(n, dtype=torch.bfloat16) for n in sizes]
+    st0 = synth.make_state(sizes, bits_m, bits_v, block, seed=77 + bits_m)
+    hk = dict(lr=1e-3, beta1=beta1, beta2=0.999, weight_decay=0.0, seed=31, round_m=1)
+    run_lockstep(sizes, bits_m, bits_v, block, hk, 3, zero, params, state0=st0, policies=(0, 3, 1),
+                 update_tol=RANDOM_STATE_TOL)
+
+
 @pytest.mark.parametrize("hk", [
     dict(adamw=0, weight_decay=0.1),
     dict(bias_correction=0),
