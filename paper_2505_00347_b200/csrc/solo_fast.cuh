@@ -56,7 +56,7 @@ struct FastSharedT {
     uint4 xin[2][CTA / 8];                  // per group: bits of Delta_m', Delta_v', x_p
     float4 xout[2][CTA / 8];                // per group: 1/Delta_m', 1/Delta_v', 1/log2(alpha'), rounding limit
     uint32_t xflag[2][CTA / 8];             // bit 0: vanishing first moment, bit 1: vanishing second moment
-    uint32_t red[2][16];                    // G = 256: per-warp maxima of |m^| (0..7) and v^ (8..15)
+    uint32_t red[2][24];                    // G = 256: per-warp maxima of |m^| (0..7) and v^ (8..15), minima of v^ (16..23)
     // Two stages for the inputs of a full tile, filled by bulk asynchronous copies (TMA, issued by
     // one thread) one tile ahead of their use; each stage has its own mbarrier.
     struct Stage {
@@ -401,30 +401,39 @@ __device__ __forceinline__ uint32_t select_kth(uint32_t head, const uint32_t* co
 }
 
 // k-th smallest (1-based, duplicates counted) of the CTA's 2048 keys, eight per thread.  Keys are
-// below 2^31, or the all-ones filler of elements that do not exist (k never reaches those).
-// Radix select from the top in levels of 11, 11 and 9 bits with 2048 histogram bins (eight per
-// thread); as soon as the bin that holds the rank has at most 32 keys, those are collected and
-// ranked directly by the first warp, which is the usual case after the first level.  Exact for any
-// input: with many equal keys the levels run on until all 31 bits are fixed.  `hist` is 2096
-// words of shared memory.  Every thread of the CTA calls it; all return the same key.
-__device__ __forceinline__ uint32_t cta_select(const uint32_t (&key)[EPT], int k, uint32_t* hist) {
+// below 2^31, or the all-ones filler of elements that do not exist (k never reaches those); `lo` and
+// `hi` are the smallest and the largest key that exists.
+// Radix select from the top over the bits of key - lo that can be set (those of hi - lo), eleven at a
+// time with 2048 histogram bins (eight per thread): the first level spreads the block's own range of
+// values over all bins, whatever its position and width on the number line (the top bits of the keys
+// themselves, sign and exponent, would put a block's values into a few dozen bins).  As soon as the bin
+// that holds the rank has at most 32 keys, those are collected and ranked directly by the first warp,
+// which is the usual case after the first level.  Exact for any input: with many equal keys the levels
+// run on until every bit is fixed.  `hist` is 2096 words of shared memory.  Every thread of the CTA calls
+// it with the same k, lo and hi; all return the same key.
+__device__ __forceinline__ uint32_t cta_select(const uint32_t (&key)[EPT], int k, uint32_t* hist, uint32_t lo,
+                                               uint32_t hi) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     uint32_t* const scan = hist + 2048;      // [0..7] warp totals, [8] bin, [9] rank in it, [10] its count,
                                              // [11] fill of `list`, [12] the answer
     uint32_t* const list = hist + 2048 + 16; // the keys of a bin with at most 32 of them
+    if (hi == lo) return lo;                 // (uniform) every key that exists is the same
+    int remaining = 32 - __clz(hi - lo);     // bits of key - lo not fixed yet: at most 31
     uint32_t prefix = 0, kk = (uint32_t)k;
 #pragma unroll 1
-    for (int level = 0; level < 3; ++level) {
-        const int shift = level == 0 ? 20 : level == 1 ? 9 : 0;
-        const int width = level == 2 ? 9 : 11;
+    for (;;) {
+        const int width = min(remaining, 11);
+        const int shift = remaining - width;
         __syncthreads();                       // the bins, scan[] and list[] of earlier use are read
         reinterpret_cast<uint4*>(hist)[2 * tid] = make_uint4(0u, 0u, 0u, 0u);
         reinterpret_cast<uint4*>(hist)[2 * tid + 1] = make_uint4(0u, 0u, 0u, 0u);
         if (tid == 0) scan[11] = 0;
         __syncthreads();
 #pragma unroll
-        for (int i = 0; i < EPT; ++i)         // level 0: key >> 31 == 0 leaves the filler out
-            if ((key[i] >> (shift + width)) == prefix) atomicAdd(&hist[(key[i] >> shift) & ((1u << width) - 1u)], 1u);
+        for (int i = 0; i < EPT; ++i) {       // (the filler minus lo is at least 2^31: it matches no prefix)
+            const uint32_t d = key[i] - lo;
+            if ((d >> remaining) == prefix) atomicAdd(&hist[(d >> shift) & ((1u << width) - 1u)], 1u);
+        }
         __syncthreads();
         const uint4 c0 = reinterpret_cast<const uint4*>(hist)[2 * tid];
         const uint4 c1 = reinterpret_cast<const uint4*>(hist)[2 * tid + 1];
@@ -462,11 +471,12 @@ __device__ __forceinline__ uint32_t cta_select(const uint32_t (&key)[EPT], int k
         prefix = (prefix << width) | scan[8];
         kk = scan[9];
         const uint32_t cnt = scan[10];
-        if (level == 2) break;                 // all 31 bits are fixed
+        remaining = shift;
+        if (remaining == 0) break;             // every bit is fixed
         if (cnt <= 32u) {                      // uniform: rank the bin's keys directly
 #pragma unroll
             for (int i = 0; i < EPT; ++i)
-                if ((key[i] >> shift) == prefix) list[atomicAdd(&scan[11], 1u)] = key[i];
+                if (((key[i] - lo) >> remaining) == prefix) list[atomicAdd(&scan[11], 1u)] = key[i];
             __syncthreads();
             if (warp == 0) {
                 const uint32_t my = (uint32_t)lane < cnt ? list[lane] : 0xFFFFFFFFu;
@@ -481,7 +491,7 @@ __device__ __forceinline__ uint32_t cta_select(const uint32_t (&key)[EPT], int k
             return scan[12];
         }
     }
-    return prefix;
+    return lo + prefix;
 }
 
 __device__ __forceinline__ void bar_sync(int id) {
@@ -783,11 +793,19 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
     uint32_t x_p = 0;
     if constexpr (G == CTA) {
         // one block per tile: maxima over the CTA through shared memory, radix select
+        // (and the minimum of v^ over the elements that exist: the select works on the block's own range)
+        uint32_t mn_v = 0xFFFFFFFFu;
+        if (!fixed_base) {
+#pragma unroll
+            for (int i = 0; i < EPT; ++i) mn_v = min(mn_v, (FULL || i < nv) ? __float_as_uint(vh[i]) : 0xFFFFFFFFu);
+            mn_v = __reduce_min_sync(0xffffffffu, mn_v);
+        }
         mx_m = __reduce_max_sync(0xffffffffu, mx_m);
         mx_v = __reduce_max_sync(0xffffffffu, mx_v);
         if (lane == 0) {
             s.red[par][warp] = mx_m;
             s.red[par][8 + warp] = mx_v;
+            s.red[par][16 + warp] = mn_v;
         }
 #pragma unroll
         for (int i = 0; i < EPT; ++i) update(i);
@@ -804,7 +822,8 @@ __device__ __forceinline__ void fast_tile(const StepArgs& a, FastShared<BM, BV>&
                 k = (int)ceil((double)a.p_quantile * (double)nb);
                 k = min(max(k, 1), nb);
             }
-            x_p = cta_select(key, k, &s.sort[0][0]);
+            mn_v = __reduce_min_sync(0xffffffffu, s.red[par][16 + (lane & 7)]);
+            x_p = cta_select(key, k, &s.sort[0][0], mn_v, mx_v);
         }
     } else {
         mx_m = seg_max31<G>(mx_m, hi);
