@@ -57,26 +57,20 @@ static_assert(CTA16 * EPT16 == TILE, "same tile as the other kernels");
 #define SOLO_F16_CTAS_WIDE 6            // the same for every other instantiation
 #endif
 
-// G: lanes per block (4, 8 or 16 for blocks of 64, 128 or 256 elements; 128: the CTA is one block of
-// 2048); NG = 128 / G blocks per tile.
+// G: lanes per block (4, 8 or 16 for blocks of 64, 128 or 256 elements); NG = 128 / G blocks per tile.
 template <int BM, int BV, bool PBF, int G>
 struct Fast16Shared {
     static constexpr int NG = CTA16 / G;
     static constexpr int ROUNDS = G == 4 ? 6 : G == 8 ? 12 : 25;   // rank of the p = 0.1 quantile minus one: 7, 13, 26
     static constexpr int ROWS = ROUNDS < 15 ? ROUNDS : 16;         // G = 16: all fifteen further keys and a sentinel row
-    static constexpr int NT = G == 128 ? 4 : NG;                   // level tables: one per block, or one per warp of the one block
     // Sorted keys of the threads, one column per thread: row j holds the (j+2)-th smallest key.
     // The rounds of popping read rows 0..ROUNDS-1 at most; with 25 rounds a thread can run out of
-    // keys, and row 15 holds a sentinel above every key.  G = 128: the 2048 bins of the radix select.
-    alignas(16) uint32_t sort[ROWS][CTA16];
-    // G = 128: the CTA-wide selection's small state (see cta_select16) and the warps' maxima
-    uint32_t scan[G == 128 ? 16 : 1];
-    uint32_t list[G == 128 ? 32 : 1];
-    uint32_t red[G == 128 ? 8 : 1];
+    // keys, and row 15 holds a sentinel above every key.
+    uint32_t sort[ROWS][CTA16];
     // per block: K_v second-moment levels alpha^k Delta_v and K_m first-moment levels y_k Delta_m.
     // Two arrays, so that the four blocks of a warp occupy distinct banks (up to eight levels).
-    float tab_v[NT][1 << BV];
-    float tab_m[NT][1 << BM];
+    float tab_v[NG][1 << BV];
+    float tab_m[NG][1 << BM];
     // Exchange with the first warp.  One copy is enough: xin is written before the tile's first
     // barrier and read between its two barriers, xout is written between the barriers and read
     // after the second, and nobody writes either again before passing those barriers.
@@ -255,8 +249,7 @@ __device__ __forceinline__ void issue_tile_copy16(const StepArgs& a, Fast16Share
     // 16 bytes more (the state's arrays carry that slack), and read with an offset
     const int64_t bm0 = jb_tile * (2 * G * BM), bv0 = jb_tile * (2 * G * BV);
     const uint32_t bytes_m = 256 * BM + ((bm0 & 15) ? 16u : 0u), bytes_v = 256 * BV + ((bv0 & 15) ? 16u : 0u);
-    // (a single block's scalar lies within the 16 bytes that start at the boundary below it)
-    const uint32_t bytes_s = NG >= 4 ? (NG + ((jb_tile & 3) ? 4u : 0u)) * 4u : 16u;
+    const uint32_t bytes_s = (NG + ((jb_tile & 3) ? 4u : 0u)) * 4u;
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar),
                  "r"((uint32_t)(TILE * (PBF ? 2 : 4) + TILE * 2) + bytes_m + bytes_v + 3u * bytes_s + extra_tx)
                  : "memory");
