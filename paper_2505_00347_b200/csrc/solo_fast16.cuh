@@ -51,10 +51,7 @@ static_assert(CTA16 * EPT16 == TILE, "same tile as the other kernels");
 #define SOLO_F16_M4FMA 1                // 4-bit first moments: two levels of three saturated multiply-adds
 #endif
 #ifndef SOLO_F16_CTAS
-#define SOLO_F16_CTAS 7                 // resident CTAs per SM the plain fp32 kernel for blocks of 64 and 128 is compiled for (72 registers)
-#endif
-#ifndef SOLO_F16_CTAS_WIDE
-#define SOLO_F16_CTAS_WIDE 6            // the same for every other instantiation
+#define SOLO_F16_CTAS 7                 // resident CTAs per SM every instantiation is compiled for (72 registers)
 #endif
 
 // G: lanes per block (4, 8 or 16 for blocks of 64, 128 or 256 elements); NG = 128 / G blocks per tile.
@@ -876,7 +873,7 @@ __device__ __forceinline__ void fast16_tile(const StepArgs& a, Fast16Shared<BM, 
 }
 
 template <int BM, int BV, bool PBF, int G, int MODES>
-__global__ void __launch_bounds__(CTA16, (PBF || G == 16 || MODES != 0) ? SOLO_F16_CTAS_WIDE : SOLO_F16_CTAS) solo_step_fast16_kernel(const StepArgs a) {
+__global__ void __launch_bounds__(CTA16, SOLO_F16_CTAS) solo_step_fast16_kernel(const StepArgs a) {
     constexpr int KM = 1 << BM;
     constexpr bool EXT = MODES == 2;
     using Shared = Fast16Shared<BM, BV, PBF, G>;
