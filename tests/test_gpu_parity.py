@@ -427,6 +427,8 @@ def test_bounded_wait_runs_out_and_nothing_is_stored():
     (2, 3, 128, dict(), 0),
     (2, 3, 128, dict(policy=3), 2048 * 3),
     (2, 4, 128, dict(policy=3, param_dtype=1, param_round=1), 2048 * 2),
+    (4, 3, 128, dict(policy=3, round_m=1, v_codebook=3), 2048 * 3),    # the general kernel takes what is left of each chunk
+    (3, 2, 256, dict(policy=3, v_codebook=1, adamw=0), 2048),
 ])
 def test_host_buffer_entry_point(bits_m, bits_v, block, extra, chunk):
     """solo_multi_step_host (gradients from host memory, parameters copied back, chunked over three
@@ -447,10 +449,12 @@ def test_host_buffer_entry_point(bits_m, bits_v, block, extra, chunk):
     st_hst = B.State(list(sizes), bits_m, bits_v, block)
     for t in (1, 2):
         grads = [synth.make_grad(w, i, t) for i in range(len(sizes))]
-        B.solo_multi_step(B.TensorSet(p_dev, [g.cuda() for g in grads], st_dev), h, t)
         pinned = [g.pin_memory() for g in grads]
+        # (the same kernels on both sides: the general kernel's IEEE division and the faster kernels'
+        # refined reciprocal differ in the last bits of an fp32 parameter)
         B.set_kernel_policy(policy)
         try:
+            B.solo_multi_step(B.TensorSet(p_dev, [g.cuda() for g in grads], st_dev), h, t)
             B.solo_multi_step_host(p_hst, pinned, out if t == 2 else None, st_hst, h, t, chunk_elems=chunk)
             torch.cuda.synchronize()
         finally:
